@@ -1,0 +1,404 @@
+"""Pins for the CPU oracle: every check here compares the oracle with something other than itself -
+a closed form, an invariant of the definitions, a library routine a special case reduces to, a value the
+paper prints, or an independent pure-loop brute force."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import brute, models
+from oracle import s4r_oracle as O
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+def _toy(seed=0, T=48, h_kv=2, G=2, dh=8, r=6, s=3, lowrank=True):
+    rng = _rng(seed)
+    D = h_kv * dh
+    mix = np.linalg.qr(rng.standard_normal((D, D)))[0]
+    sig = np.arange(1, D + 1) ** -0.8 if lowrank else np.ones(D)
+    K = (rng.standard_normal((T, D)) * sig) @ mix.T + 0.05 * rng.standard_normal((T, D))
+    V = (rng.standard_normal((T, D)) * sig) @ mix.T + 0.05 * rng.standard_normal((T, D))
+    K[:s] *= 10
+    V[:s] *= 10
+    q = rng.standard_normal((h_kv * G, dh)) * 2.0
+    BK, _ = O.build_basis(K[s:], r)
+    BV, _ = O.build_basis(V[s:], r)
+    return K, V, q, BK, BV, s
+
+
+# ---------------------------------------------------------------- storage rounding
+
+def test_bf16_rounding_matches_torch_bits():
+    torch = pytest.importorskip("torch")
+    x = _rng(1).standard_normal(20000) * np.exp(_rng(2).uniform(-20, 20, 20000))
+    x32 = x.astype(np.float32).astype(np.float64)          # exactly representable in fp32: no double rounding
+    want = torch.from_numpy(x32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(O.round_to_storage(x32, "bf16"), want)
+
+
+def test_bf16_rounding_ties_to_even_and_ulp():
+    # 1 + 2^-8 is exactly half way between 1 and 1 + 2^-7 -> even mantissa (1.0); 1 + 3*2^-8 -> 1 + 2^-6
+    assert O.round_to_storage(1.0 + 2.0 ** -8, "bf16") == 1.0
+    assert O.round_to_storage(1.0 + 3 * 2.0 ** -8, "bf16") == 1.0 + 2.0 ** -6
+    assert O.storage_ulp(1.5, "bf16") == 2.0 ** -7
+    assert O.storage_ulp(1.5, "f32") == 2.0 ** -23
+
+
+# ---------------------------------------------------------------- P1: basis
+
+def test_basis_orthonormal_and_eckart_young():
+    rng = _rng(3)
+    S = rng.standard_normal((200, 32)) * (np.arange(1, 33) ** -0.7)
+    r = 10
+    B, sv = O.build_basis(S, r)
+    assert np.allclose(B.T @ B, np.eye(r), atol=1e-12)
+    Sn = O.normalize_rows(S)
+    assert np.allclose(np.linalg.norm(Sn, axis=1), 1.0, atol=1e-14)
+    resid = np.linalg.norm(Sn - Sn @ B @ B.T) ** 2
+    assert np.isclose(resid, np.sum(sv[r:] ** 2), rtol=1e-10)
+
+
+def test_basis_matches_gram_eigenvectors():
+    rng = _rng(4)
+    S = rng.standard_normal((120, 24)) * (np.arange(1, 25) ** -1.0)
+    r = 8
+    B, sv = O.build_basis(S, r)
+    Sn = S / np.linalg.norm(S, axis=1, keepdims=True)
+    w, U = np.linalg.eigh(Sn.T @ Sn)
+    U = U[:, ::-1][:, :r]
+    assert np.allclose(np.sqrt(w[::-1][:r]), sv[:r], rtol=1e-10)
+    # same subspace, column by column up to sign
+    assert np.allclose(np.abs(np.sum(U * B, axis=0)), 1.0, atol=1e-8)
+    # sign convention: the largest-magnitude entry of each column is positive
+    assert np.all(B[np.argmax(np.abs(B), axis=0), np.arange(r)] > 0)
+
+
+def test_normalisation_changes_the_basis_only_through_row_scale():
+    # scaling individual rows must not change the basis (that is what Eq. 1 is for)
+    rng = _rng(5)
+    S = rng.standard_normal((80, 16))
+    scale = np.exp(rng.uniform(-3, 3, (80, 1)))
+    B1, _ = O.build_basis(S, 5)
+    B2, _ = O.build_basis(S * scale, 5)
+    assert np.allclose(B1, B2, atol=1e-10)
+
+
+def test_hybrid_sampling_split_and_range():
+    idx = O.hybrid_sample_indices(1000, 100)
+    assert len(idx) == len(set(idx.tolist())) and idx.min() >= 0 and idx.max() == 999
+    assert np.array_equal(idx[-70:], np.arange(930, 1000))          # contiguous recent block, 7:3 split
+    early = idx[:-70]
+    assert len(early) == 30 and early.max() < 930
+    assert np.all(np.diff(early) == 31)                              # evenly spread over the early part
+
+
+# ---------------------------------------------------------------- P2: compress
+
+def test_full_rank_compress_is_exact():
+    K, V, q, _, _, s = _toy(T=40, lowrank=False)
+    D = K.shape[1]
+    BK, _ = O.build_basis(K[s:], D)
+    BV, _ = O.build_basis(V[s:], D)
+    sk, sv_, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    assert np.array_equal(sk, K[:s]) and np.array_equal(sv_, V[:s])
+    assert np.allclose(CK @ BK.T, K[s:], atol=1e-12)
+    assert np.allclose(CV @ BV.T, V[s:], atol=1e-12)
+
+
+def test_low_rank_residual_is_orthogonal_to_basis():
+    K, V, q, BK, BV, s = _toy()
+    _, _, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    assert np.abs(BK.T @ (K[s:] - CK @ BK.T).T).max() < 1e-12
+    assert CK.shape == (K.shape[0] - s, BK.shape[1])
+
+
+def test_compress_is_not_transposed_or_normalised():
+    # a basis made of unit vectors picks out raw channels: C[:, j] = S[:, chan[j]] exactly
+    rng = _rng(6)
+    K = rng.standard_normal((20, 12))
+    V = rng.standard_normal((20, 12))
+    chan = [7, 2, 11]
+    B = np.zeros((12, 3))
+    B[chan, [0, 1, 2]] = 1.0
+    _, _, CK, CV = O.compress(K, V, 2, B, B, "f64")
+    assert np.array_equal(CK, K[2:][:, chan]) and np.array_equal(CV, V[2:][:, chan])
+
+
+def test_compress_rounds_once_to_storage():
+    K, V, q, BK, BV, s = _toy()
+    _, _, CK64, _ = O.compress(K, V, s, BK, BV, "f64")
+    _, _, CKb, _ = O.compress(K, V, s, BK, BV, "bf16")
+    assert np.all(np.abs(CKb - CK64) <= 0.5 * O.storage_ulp(CK64, "bf16") * (1 + 1e-12))
+    assert np.array_equal(O.round_to_storage(CKb, "bf16"), CKb)
+
+
+def test_memory_model_closed_forms():
+    s, L, Dp, r, G, W = 4, 120000, 1024, 204, 4, 32
+    ratio = models.memory_ratio(s, L, Dp, r, G, W)
+    assert math.isclose(ratio, models.memory_s4r(s, L, Dp, r, G, W) / models.memory_full(s, L, Dp), rel_tol=1e-15)
+    assert abs(models.memory_ratio(s, 10 ** 9, Dp, r, G, W) - r / Dp) < 1e-5          # limit r / D'
+    for W_, rho, L_ in [(32, 0.2, 1000), (32, 0.01, 1000), (64, 0.2, 131068)]:
+        assert models.reconstructed_tokens(W_, rho, L_) == max(W_, math.floor(rho * L_))
+        assert models.top_k_from_ratio(rho, L_, W_) + W_ == models.reconstructed_tokens(W_, rho, L_)
+
+
+# ---------------------------------------------------------------- P3: the paper's printed cost example
+
+def _golden(path):
+    out = {}
+    for line in open(path):
+        line = line.split("#")[0].strip()
+        if line:
+            k, v = line.split()
+            out[k] = float(v)
+    return out
+
+
+def test_cost_model_matches_printed_example(golden_dir):
+    g = _golden(golden_dir + "/cost_example.txt")
+    W, r, rho, Dp = int(g["W"]), int(g["r"]), g["rho"], int(g["Dp"])
+    assert models.cost_full_reconstruction(r, Dp, 0) == g["full_rec_const"]
+    sc, rec, att = models.cost_s4r(r, Dp, 1, W, rho)
+    assert sc == g["scoring_per_G"]
+    assert math.isclose(rec, g["reconstruct"], rel_tol=1e-12)
+    assert math.isclose(att, g["attention_per_G"], rel_tol=1e-12)
+    assert round(sc + att) == g["s4r_per_G_rounded"]
+    for G, num, den, ratio in [(1, "ratio_G1_num", "ratio_G1_den", "ratio_G1"),
+                               (4, "ratio_G4_num", "ratio_G4_den", "ratio_G4")]:
+        full = models.cost_full_reconstruction(r, Dp, G)
+        mine = sum(models.cost_s4r(r, Dp, G, W, rho))
+        assert full == g[den]
+        assert abs(mine - g[num]) < 5.0                       # the paper rounds the numerator
+        assert abs(mine / full - g[ratio]) < 6e-4
+
+
+# ---------------------------------------------------------------- P4: latent logits
+
+def test_full_rank_latent_logits_equal_dense_dot_products():
+    K, V, q, _, _, s = _toy(T=30, lowrank=False)
+    D = K.shape[1]
+    h_kv = 2
+    BK, _ = O.build_basis(K[s:], D)
+    _, _, CK, _ = O.compress(K, V, s, BK, BK, "f64")
+    cq = O.project_query(q, BK, h_kv)
+    Z = O.latent_logits(cq[:, None, :], CK)[:, 0, :]
+    # dense definition: sum over KV heads of <q_{kv*G+g}, k_{l,kv}>
+    G, dh = q.shape[0] // h_kv, q.shape[1]
+    want = np.zeros_like(Z)
+    for g in range(G):
+        for kv in range(h_kv):
+            want[g] += K[s:, kv * dh:(kv + 1) * dh] @ q[kv * G + g]
+    assert np.allclose(Z, want / np.sqrt(D), atol=1e-11)
+
+
+def test_group_queries_pairs_each_head_with_its_kv_head():
+    q = np.arange(6 * 4, dtype=float).reshape(6, 4)             # H_q = 6, h_kv = 3, G = 2
+    Qt = O.group_queries(q, 3)
+    assert Qt.shape == (2, 12)
+    assert np.array_equal(Qt[1, 4:8], q[1 * 2 + 1])             # kv = 1, g = 1 -> head 3
+    assert np.array_equal(Qt[0, 8:12], q[2 * 2 + 0])
+
+
+# ---------------------------------------------------------------- P5: relevance, pooling, aggregation
+
+def test_relevance_rows_sum_to_one_and_mask_is_causal():
+    rng = _rng(7)
+    Z = rng.standard_normal((3, 4, 50))
+    A = O.relevance(Z)
+    assert np.allclose(A.sum(axis=1), 1.0, atol=1e-13)
+    # row i of the window cannot see beyond L - W_q + i: the newest position gets mass from the last row only
+    Z1 = Z.copy()
+    Z1[:, :3, 49] += 100.0                                      # masked entries must have no effect
+    assert np.allclose(O.relevance(Z1), A, atol=1e-15)
+    # W_q = 1 reduces to library softmax
+    sp = pytest.importorskip("scipy.special")
+    assert np.allclose(O.relevance(Z[:, 3:4, :]), sp.softmax(Z[:, 3, :], axis=-1), atol=1e-15)
+
+
+def test_ranking_without_pooling_is_argsort_of_logits():
+    rng = _rng(8)
+    cq = rng.standard_normal((1, 1, 6))
+    CK = rng.standard_normal((200, 6))
+    Z = O.latent_logits(cq, CK)
+    A = O.pool_sequence(O.relevance(Z), 1, "max")
+    score = O.aggregate_group(A, "mean")
+    idx, W_eff, k_eff = O.select_indices(score, 10, 25)
+    raw = (CK[:190] @ cq[0, 0])
+    want = np.sort(np.argsort(-raw, kind="stable")[:25])
+    assert np.array_equal(idx[:25][idx[:25] < 190], want) and W_eff == 10 and k_eff == 25
+
+
+@pytest.mark.parametrize("kappa", [1, 3, 7])
+def test_pooling_properties(kappa):
+    nd = pytest.importorskip("scipy.ndimage")
+    rng = _rng(9)
+    A = rng.random((3, 64))
+    mx = O.pool_sequence(A, kappa, "max")
+    av = O.pool_sequence(A, kappa, "avg")
+    assert np.all(mx >= A)
+    assert np.array_equal(mx, nd.maximum_filter1d(A, kappa, axis=1, mode="constant", cval=-np.inf))
+    assert np.allclose(av, nd.uniform_filter1d(A, kappa, axis=1, mode="constant", cval=0.0), atol=1e-15)
+    assert np.array_equal(O.pool_sequence_fast(A, kappa, "max"), mx)
+    assert np.allclose(O.pool_sequence_fast(A, kappa, "avg"), av, rtol=1e-14, atol=0)
+    # interior positions: the sum of avg-pooled values equals the sum of inputs up to edge terms
+    h = kappa // 2
+    edge = sum(A[:, j].sum() * (h - j) / kappa for j in range(h)) + \
+        sum(A[:, 63 - j].sum() * (h - j) / kappa for j in range(h))
+    assert np.isclose(av.sum(), A.sum() - edge, rtol=1e-12)
+
+
+def test_group_aggregation_modes():
+    A = np.array([[1.0, 5.0, 2.0], [3.0, 1.0, 2.0]])
+    assert np.array_equal(O.aggregate_group(A, "mean"), [2.0, 3.0, 2.0])
+    assert np.array_equal(O.aggregate_group(A, "max"), [3.0, 5.0, 2.0])
+
+
+# ---------------------------------------------------------------- P6: selection
+
+def test_selection_properties_and_ties():
+    rng = _rng(10)
+    score = rng.random(300)
+    score[[5, 40, 41, 42]] = 0.99                                # exact ties (as max pooling produces)
+    idx, W_eff, k_eff = O.select_indices(score, 16, 3)
+    assert (W_eff, k_eff) == (16, 3) and len(idx) == 19 and np.all(np.diff(idx) > 0)
+    assert np.array_equal(idx[:3], [5, 40, 41])                  # lower index wins the tie
+    assert np.array_equal(idx[3:], np.arange(284, 300))
+    glob = idx[:3]
+    rest = np.setdiff1d(np.arange(284), glob)
+    assert score[glob].min() >= score[rest].max()
+    # degenerate budgets
+    assert np.array_equal(O.select_indices(score[:10], 16, 3)[0], np.arange(10))      # L < W
+    i2, w2, k2 = O.select_indices(score[:20], 16, 100)                                  # k > candidates
+    assert (w2, k2) == (16, 4) and np.array_equal(i2, np.arange(20))
+    assert O.select_indices(score, 16, 0)[2] == 0
+
+
+def test_selection_band_rule():
+    score = np.array([0.5, 0.4, 0.3000001, 0.3, 0.1, 0.0, 0.0, 0.0])
+    idx, W_eff, k_eff = O.select_indices(score, 2, 3)
+    assert np.array_equal(idx, [0, 1, 2, 6, 7])
+    ok, _ = O.selection_agrees(score, idx, np.array([0, 1, 3, 6, 7]), W_eff, k_eff)      # swap inside the band
+    assert ok
+    assert not O.selection_agrees(score, idx, np.array([0, 1, 4, 6, 7]), W_eff, k_eff)[0]
+    assert not O.selection_agrees(score, idx, np.array([0, 2, 3, 6, 7]), W_eff, k_eff)[0]
+    assert not O.selection_agrees(score, idx, np.array([0, 1, 2, 5, 7]), W_eff, k_eff)[0]  # window incomplete
+    assert not O.selection_agrees(score, idx, np.array([0, 1, 2, 7]), W_eff, k_eff)[0]
+
+
+# ---------------------------------------------------------------- P7: reconstruction + attention
+
+@pytest.mark.parametrize("theta", [0.0, 1.0e4])
+def test_full_budget_equals_dense_attention_over_reconstructed_cache(theta):
+    K, V, q, BK, BV, s = _toy(seed=11)
+    sk, sv_, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    L = CK.shape[0]
+    res = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=4, k=L, kappa=3, theta=theta)
+    assert np.array_equal(res["idx"], np.arange(L))
+    K_all = np.concatenate([sk, CK @ BK.T])
+    V_all = np.concatenate([sv_, CV @ BV.T])
+    want = O.dense_attention(q, K_all, V_all, theta, q_pos=s + L - 1)
+    assert np.allclose(res["out"], want, atol=1e-12)
+
+
+def test_full_rank_full_budget_equals_dense_attention_over_original_kv():
+    sp = pytest.importorskip("scipy.special")
+    K, V, q, _, _, s = _toy(seed=12, T=36, lowrank=False)
+    D = K.shape[1]
+    BK, _ = O.build_basis(K[s:], D)
+    BV, _ = O.build_basis(V[s:], D)
+    sk, sv_, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    res = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=8, k=10 ** 6, theta=0.0)
+    # textbook attention written with library softmax, per head
+    h_kv, dh = 2, q.shape[1]
+    G = q.shape[0] // h_kv
+    for h in range(q.shape[0]):
+        kv = h // G
+        w = sp.softmax(K[:, kv * dh:(kv + 1) * dh] @ q[h] / np.sqrt(dh))
+        assert np.allclose(res["out"][h], w @ V[:, kv * dh:(kv + 1) * dh], atol=1e-11)
+
+
+def test_output_is_convex_combination_and_permutation_invariant():
+    K, V, q, BK, BV, s = _toy(seed=13)
+    sk, sv_, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    res = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=4, k=6, kappa=3, theta=1.0e4)
+    idx = res["idx"]
+    assert len(idx) == 10
+    Vstar = np.concatenate([sv_, CV[idx] @ BV.T])
+    h_kv, dh = 2, q.shape[1]
+    G = q.shape[0] // h_kv
+    for h in range(q.shape[0]):
+        sl = Vstar[:, (h // G) * dh:(h // G + 1) * dh]
+        assert np.all(res["out"][h] <= sl.max(axis=0) + 1e-12) and np.all(res["out"][h] >= sl.min(axis=0) - 1e-12)
+    perm = _rng(0).permutation(len(idx))
+    out2 = O.sparse_attention(q, sk, sv_, CK, CV, BK, BV, idx[perm], 1.0e4)
+    assert np.allclose(out2, res["out"], atol=1e-13)
+
+
+def test_sinks_always_attended_and_local_window_forced():
+    # a huge sink key must dominate the output even with k = 0; the local window is always present
+    K, V, q, BK, BV, s = _toy(seed=14)
+    sk, sv_, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    res = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=5, k=0, theta=0.0)
+    L = CK.shape[0]
+    assert np.array_equal(res["idx"], np.arange(L - 5, L))
+    sk2 = sk.copy()
+    sk2[1, :8] = 50.0 * q[0] / np.linalg.norm(q[0])
+    out = O.sparse_attention(q, sk2, sv_, CK, CV, BK, BV, res["idx"], 0.0)
+    assert np.allclose(out[0], sv_[1, :8], atol=1e-6)
+
+
+# ---------------------------------------------------------------- P8: RoPE
+
+def test_rope_properties():
+    rng = _rng(15)
+    x = rng.standard_normal((5, 16))
+    y = rng.standard_normal((5, 16))
+    pos = np.array([0, 1, 17, 4000, 131071])
+    rx = O.rope_rotate(x, pos, 1.0e4)
+    assert np.allclose(np.linalg.norm(rx, axis=1), np.linalg.norm(x, axis=1), rtol=1e-13)
+    assert np.array_equal(rx[0], x[0])                                      # identity at position 0
+    assert np.array_equal(O.rope_rotate(x, pos, 0.0), x)                    # switch off
+    a = np.sum(O.rope_rotate(x, pos, 1.0e4) * O.rope_rotate(y, pos + 7, 1.0e4), axis=1)
+    b = np.sum(O.rope_rotate(x, pos * 0 + 100, 1.0e4) * O.rope_rotate(y, pos * 0 + 107, 1.0e4), axis=1)
+    assert np.allclose(a, b, atol=1e-9)                                     # depends on p - p' only
+    # explicit 2x2 rotation of the pair (0, d/2) with the base frequency
+    e = np.zeros((1, 16))
+    e[0, 0] = 1.0
+    r1 = O.rope_rotate(e, np.array([3]), 1.0e4)[0]
+    assert np.isclose(r1[0], math.cos(3.0)) and np.isclose(r1[8], math.sin(3.0))
+    e[0, 0], e[0, 1] = 0.0, 1.0
+    r2 = O.rope_rotate(e, np.array([3]), 1.0e4)[0]
+    assert np.isclose(r2[1], math.cos(3.0 * 1.0e4 ** (-2.0 / 16))) and np.isclose(r2[9], math.sin(3.0 * 1.0e4 ** (-2.0 / 16)))
+
+
+# ---------------------------------------------------------------- P9: whole step against the pure-loop brute force
+
+@pytest.mark.parametrize("pool_mode,group_mode,theta,kappa,r",
+                         [("max", "mean", 0.0, 7, 4), ("avg", "max", 1.0e4, 3, 8),
+                          ("max", "max", 5.0e5, 7, 16), ("avg", "mean", 1.0e4, 1, 6)])
+def test_decode_step_matches_brute_force(pool_mode, group_mode, theta, kappa, r):
+    K, V, q, BK, BV, s = _toy(seed=16 + r, T=43, r=r)
+    sk, sv_, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    assert np.allclose(CK, np.array(brute.compress_rows(K.tolist(), s, BK.tolist())), atol=1e-12)
+    res = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=4, k=6, kappa=kappa, pool_mode=pool_mode,
+                        group_mode=group_mode, theta=theta, fast_pool=False)
+    out_b, idx_b, score_b = brute.decode_step(q.tolist(), sk.tolist(), sv_.tolist(), CK.tolist(), CV.tolist(),
+                                              BK.tolist(), BV.tolist(), 4, 6, kappa, pool_mode, group_mode, theta)
+    assert np.allclose(res["score"], score_b, rtol=1e-12, atol=1e-300)
+    assert list(res["idx"]) == idx_b
+    assert np.allclose(res["out"], np.array(out_b), atol=1e-12)
+    res_fast = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=4, k=6, kappa=kappa, pool_mode=pool_mode,
+                             group_mode=group_mode, theta=theta, fast_pool=True)
+    assert np.array_equal(res_fast["idx"], res["idx"]) and np.allclose(res_fast["out"], res["out"], atol=1e-14)
+
+
+def test_query_window_fifo_reduces_to_single_query():
+    K, V, q, BK, BV, s = _toy(seed=30)
+    sk, sv_, CK, CV = O.compress(K, V, s, BK, BV, "f64")
+    cq = O.project_query(q, BK, 2)
+    a = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=4, k=6)
+    b = O.decode_step(q, sk, sv_, CK, CV, BK, BV, W=4, k=6, CQ_window=cq[:, None, :])
+    assert np.array_equal(a["idx"], b["idx"]) and np.allclose(a["out"], b["out"], atol=0)

@@ -1,0 +1,73 @@
+"""The seeded input generators: determinism, shapes, the structure the recipe promises."""
+import numpy as np
+import torch
+
+import workloads as W
+from oracle import s4r_oracle as O
+
+
+def _small(i, **kw):
+    base = dict(context=600, n_sampled=128, batch=1)
+    base.update(kw)
+    return W.scaled_config(W.get_config(i), **base)
+
+
+def test_streams_are_deterministic_and_distinct():
+    c = _small(0)
+    a = W.make_kv(c, 0, 0, "k")
+    assert torch.equal(a, W.make_kv(c, 0, 0, "k"))
+    assert not torch.equal(a, W.make_kv(c, 0, 1, "k"))
+    assert not torch.equal(a, W.make_kv(c, 1, 0, "k"))
+    assert not torch.equal(a, W.make_kv(c, 0, 0, "v"))
+    assert a.dtype == torch.float32 and a.shape == (600, 256)
+    assert W.make_kv(_small(1), 0, 0, "k").dtype == torch.bfloat16
+
+
+def test_sink_rows_are_scaled_and_spectrum_decays():
+    c = _small(0, context=3000)
+    k = W.make_kv(c, 0, 0, "k").double()
+    assert k[:4].norm(dim=1).mean() > 5 * k[4:].norm(dim=1).mean()
+    sv = torch.linalg.svdvals(k[4:])
+    assert sv[0] / sv[63] > 10          # i^-0.8 spectrum: energy concentrates in the leading directions
+
+
+def test_outlier_channels_only_in_config3():
+    c3 = _small(3, context=2000)
+    k = W.make_kv(c3, 0, 0, "k").double()[4:]
+    rms = k.pow(2).mean(0).sqrt()
+    assert (rms > 4 * rms.median()).sum() == round(0.02 * c3.d_kv)
+    k1 = W.make_kv(_small(1, context=2000), 0, 0, "k").double()[4:]
+    rms1 = k1.pow(2).mean(0).sqrt()
+    assert (rms1 > 4 * rms1.median()).sum() == 0
+
+
+def test_query_correlates_with_planted_keys_and_maps_heads():
+    c = _small(0, context=1500)
+    k = W.make_kv(c, 0, 0, "k")
+    q = W.make_query(c, k, 0, 0)
+    assert q.shape == (8, 128)
+    pos = W.planted_positions(c, 0, 0)
+    assert len(pos) == 16 and pos.max() < c.cache_len - c.window
+    qt = torch.from_numpy(O.group_queries(q.double().numpy(), c.n_kv_heads))
+    rows = k[pos + c.sink_count].double()
+    u = (rows / rows.norm(dim=1, keepdim=True)).sum(0)
+    u /= u.norm()
+    cos = (qt @ u) / qt.norm(dim=1)
+    assert torch.allclose(cos, torch.full_like(cos, 0.6), atol=1e-3)
+    assert torch.allclose(qt.norm(dim=1), torch.full((4,), 4.0 * 16.0, dtype=torch.float64), rtol=1e-3)
+
+
+def test_sample_rows_sorted_unique_nonsink():
+    c = _small(1)
+    idx = W.sample_rows(c, 0, 0, "k")
+    assert len(idx) == 128 and idx.min() >= 4 and idx.max() < 600
+    assert torch.all(idx[1:] > idx[:-1])
+
+
+def test_bench_basis_spans_the_oracle_basis():
+    c = _small(0, context=900)
+    k = W.make_kv(c, 0, 0, "k")
+    rows = k[W.sample_rows(c, 0, 0, "k")]
+    b = W.make_bench_basis(rows, 32, torch.float64).numpy()
+    bo, _ = O.build_basis(rows.double().numpy(), 32)
+    assert np.allclose(b, bo, atol=1e-8)

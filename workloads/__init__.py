@@ -1,0 +1,14 @@
+"""Seeded synthetic inputs for the S4R decode hot path.
+
+This package only *makes inputs*: layer geometries, the low-rank-plus-noise
+key/value generator, the correlated query generator and the sampled row
+indices.  It holds none of the arithmetic of the method itself (projection,
+scoring, selection, reconstruction, attention), so both the CUDA library's
+callers and the CPU oracle's callers may use it without sharing any of the
+code under test.
+"""
+from .configs import LayerConfig, CONFIGS, get_config, scaled_config  # noqa: F401
+from .generate import (  # noqa: F401
+    stream_seed, make_kv, make_token, make_query, sample_rows, planted_positions,
+    storage_dtype, make_bench_basis,
+)

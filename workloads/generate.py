@@ -1,0 +1,169 @@
+"""Seeded synthetic K/V, queries and sample indices (torch, CPU or CUDA).
+
+Recipe (stands in for real long-context activations, which need model weights
+and datasets that are not available offline):
+
+* mixing map  M = Q factor of a D'xD' Gaussian matrix, signs fixed so diag(R) > 0
+  (always drawn on the CPU in fp64 so it is identical on every device);
+* latents     z[t, i] = sigma_i * N(0, 1),  sigma_i = i^-alpha, i = 1..D';
+* rows        X = Z M^T + noise_std * N(0, 1);
+* outliers    a seeded set of round(outlier_frac * D') channels is multiplied by outlier_scale;
+* sinks       the first `sink_count` rows are multiplied by sink_scale;
+* query       16 planted non-sink positions outside the local window; u = unit vector of the sum of their
+              normalised key rows; for every group member g a unit Gaussian direction n_g orthogonal to u;
+              Qt[g] = query_scale * sqrt(D') * (c u + sqrt(1-c^2) n_g); query head kv*G+g is slice kv of Qt[g].
+
+Every stream is keyed by (seed, layer, sequence, tensor) through `stream_seed`.
+Random numbers drawn on different devices differ, so a comparison always moves
+the generated *bits* to the other side instead of regenerating them.
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+
+from .configs import LayerConfig
+
+_TENSOR_IDS = {"k": 1, "v": 2, "q": 3, "sample_k": 4, "sample_v": 5, "planted": 6, "mix_k": 7, "mix_v": 8,
+               "outlier_k": 9, "outlier_v": 10, "new_k": 11, "new_v": 12, "new_q": 13}
+
+
+def stream_seed(seed: int, layer: int, seq: int, tensor: str, step: int = 0) -> int:
+    """splitmix64-style mix of the stream key into a 63-bit generator seed."""
+    x = (seed * 0x9E3779B97F4A7C15 + layer * 0xBF58476D1CE4E5B9 + seq * 0x94D049BB133111EB
+         + _TENSOR_IDS[tensor] * 0xD6E8FEB86659FD93 + step * 0xA0761D6478BD642F) & 0xFFFFFFFFFFFFFFFF
+    for _ in range(2):
+        x ^= x >> 30
+        x = (x * 0xBF58476D1CE4E5B9) & 0xFFFFFFFFFFFFFFFF
+        x ^= x >> 27
+        x = (x * 0x94D049BB133111EB) & 0xFFFFFFFFFFFFFFFF
+        x ^= x >> 31
+    return x & 0x7FFFFFFFFFFFFFFF
+
+
+def storage_dtype(cfg: LayerConfig) -> torch.dtype:
+    return torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+
+
+def _cpu_gen(seed: int) -> torch.Generator:
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    return g
+
+
+def _mixing_matrix(cfg: LayerConfig, layer: int, seq: int, tensor: str) -> torch.Tensor:
+    d = cfg.d_kv
+    g = _cpu_gen(stream_seed(cfg.seed, layer, seq, "mix_" + tensor))
+    a = torch.randn(d, d, generator=g, dtype=torch.float64)
+    q, r = torch.linalg.qr(a)
+    return q * torch.sign(torch.diagonal(r))[None, :]
+
+
+def _outlier_channels(cfg: LayerConfig, layer: int, seq: int, tensor: str) -> torch.Tensor:
+    n = int(round(cfg.outlier_frac * cfg.d_kv))
+    if n <= 0:
+        return torch.empty(0, dtype=torch.long)
+    g = _cpu_gen(stream_seed(cfg.seed, layer, seq, "outlier_" + tensor))
+    return torch.randperm(cfg.d_kv, generator=g)[:n].sort().values
+
+
+def make_kv(cfg: LayerConfig, layer: int, seq: int, tensor: str, device="cpu",
+            n_rows: int | None = None, compute_dtype: torch.dtype = torch.float32,
+            chunk: int = 16384) -> torch.Tensor:
+    """[n_rows (default cfg.context), D'] keys ('k') or values ('v') in the storage dtype."""
+    assert tensor in ("k", "v")
+    dev = torch.device(device)
+    t_total = cfg.context if n_rows is None else n_rows
+    d = cfg.d_kv
+    alpha = cfg.alpha_k if tensor == "k" else cfg.alpha_v
+    mix_t = _mixing_matrix(cfg, layer, seq, tensor).t().contiguous().to(device=dev, dtype=compute_dtype)
+    sigma = torch.arange(1, d + 1, dtype=torch.float64).pow(-alpha).to(device=dev, dtype=compute_dtype)
+    chans = _outlier_channels(cfg, layer, seq, tensor).to(dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(stream_seed(cfg.seed, layer, seq, tensor))
+    out = torch.empty(t_total, d, dtype=storage_dtype(cfg), device=dev)
+    for lo in range(0, t_total, chunk):
+        hi = min(t_total, lo + chunk)
+        z = torch.randn(hi - lo, d, generator=gen, dtype=compute_dtype, device=dev) * sigma
+        x = z @ mix_t
+        x += cfg.noise_std * torch.randn(hi - lo, d, generator=gen, dtype=compute_dtype, device=dev)
+        if chans.numel():
+            x[:, chans] *= cfg.outlier_scale
+        if lo < cfg.sink_count:
+            x[: max(0, min(hi, cfg.sink_count) - lo)] *= cfg.sink_scale
+        out[lo:hi] = x.to(out.dtype)
+    return out
+
+
+def make_token(cfg: LayerConfig, layer: int, seq: int, tensor: str, step: int, device="cpu") -> torch.Tensor:
+    """One new decode-time key/value row [D'] (same distribution as the prompt rows, no sink scaling)."""
+    assert tensor in ("k", "v")
+    dev = torch.device(device)
+    d = cfg.d_kv
+    alpha = cfg.alpha_k if tensor == "k" else cfg.alpha_v
+    g = _cpu_gen(stream_seed(cfg.seed, layer, seq, "new_" + tensor, step))
+    z = torch.randn(d, generator=g, dtype=torch.float64) * torch.arange(1, d + 1, dtype=torch.float64).pow(-alpha)
+    x = _mixing_matrix(cfg, layer, seq, tensor) @ z + cfg.noise_std * torch.randn(d, generator=g, dtype=torch.float64)
+    chans = _outlier_channels(cfg, layer, seq, tensor)
+    if chans.numel():
+        x[chans] *= cfg.outlier_scale
+    return x.to(storage_dtype(cfg)).to(dev)
+
+
+def planted_positions(cfg: LayerConfig, layer: int, seq: int, cache_len: int | None = None) -> torch.Tensor:
+    """`n_planted` distinct non-sink indices in [0, L - W) the query is correlated with (sorted, CPU int64)."""
+    length = cfg.cache_len if cache_len is None else cache_len
+    hi = max(1, length - cfg.window)
+    n = min(cfg.n_planted, hi)
+    g = _cpu_gen(stream_seed(cfg.seed, layer, seq, "planted"))
+    return torch.randperm(hi, generator=g)[:n].sort().values
+
+
+def make_query(cfg: LayerConfig, k_seq: torch.Tensor, layer: int, seq: int, step: int = 0,
+               cache_len: int | None = None) -> torch.Tensor:
+    """[H_q, d_h] pre-RoPE query heads correlated (cosine `query_cos`) with the planted keys of `k_seq`.
+
+    `k_seq` is this sequence's key matrix [>= sink_count + max planted + 1, D'] in storage dtype (any device).
+    """
+    dev = k_seq.device
+    d = cfg.d_kv
+    pos = planted_positions(cfg, layer, seq, cache_len).to(dev) + cfg.sink_count
+    rows = k_seq[pos].to(torch.float64)
+    u = (rows / rows.norm(dim=1, keepdim=True).clamp_min(1e-30)).sum(0)
+    u = u / u.norm().clamp_min(1e-30)
+    g = _cpu_gen(stream_seed(cfg.seed, layer, seq, "q" if step == 0 else "new_q", step))
+    n = torch.randn(cfg.group, d, generator=g, dtype=torch.float64).to(dev)
+    n = n - (n @ u)[:, None] * u[None, :]
+    n = n / n.norm(dim=1, keepdim=True)
+    c = cfg.query_cos
+    qt = cfg.query_scale * math.sqrt(d) * (c * u[None, :] + math.sqrt(1.0 - c * c) * n)   # [G, D']
+    # query head kv*G+g is the kv-th head_dim slice of Qt[g]
+    q = qt.view(cfg.group, cfg.n_kv_heads, cfg.head_dim).permute(1, 0, 2).reshape(cfg.n_q_heads, cfg.head_dim)
+    return q.to(storage_dtype(cfg)).contiguous()
+
+
+def sample_rows(cfg: LayerConfig, layer: int, seq: int, tensor: str, prompt_len: int | None = None) -> torch.Tensor:
+    """Sorted absolute row indices in [sink_count, prompt_len): `n_sampled` rows, uniform without replacement."""
+    t_total = cfg.context if prompt_len is None else prompt_len
+    n_nonsink = t_total - cfg.sink_count
+    n = min(cfg.n_sampled, n_nonsink)
+    g = _cpu_gen(stream_seed(cfg.seed, layer, seq, "sample_" + tensor))
+    return (torch.randperm(n_nonsink, generator=g)[:n] + cfg.sink_count).sort().values
+
+
+def make_bench_basis(sampled: torch.Tensor, rank: int, out_dtype: torch.dtype) -> torch.Tensor:
+    """Basis [D', rank] from sampled rows, for callers that have no access to the CPU oracle.
+
+    Setup only (it is an *input* of the library): rows are L2-normalised, the top-`rank` right singular
+    vectors are taken and each column's sign is fixed so its largest-magnitude entry is positive.  Parity
+    tests do not use this function; they take their bases from the oracle's own setup code.
+    """
+    x = sampled.to(torch.float64)
+    x = x / x.norm(dim=1, keepdim=True).clamp_min(1e-12)
+    _, _, vh = torch.linalg.svd(x, full_matrices=False)
+    b = vh[:rank].t().contiguous()
+    idx = b.abs().argmax(dim=0)
+    sign = torch.sign(b[idx, torch.arange(rank, device=b.device)])
+    sign[sign == 0] = 1
+    return (b * sign[None, :]).to(out_dtype)
