@@ -1,0 +1,180 @@
+/*
+ * s4r.h - C ABI of the B200 (sm_100a) library for the S4R decode hot path
+ * (arXiv 2608.00528: low-rank KV-cache compression with latent-space scoring
+ * and sparse reconstruction).
+ *
+ * Citations name the paper's sections; equations of Sec. 3 are unnumbered in
+ * the paper, so "Eq. n" is the n-th displayed equation of Sec. 3 in order of
+ * appearance (Eq. 3: C = S B; Eq. 5: per-step projection; Eq. 6: append;
+ * Eq. 8: latent logits; Eq. 9: softmax; Eq. 11: pooling; Eq. 12: group
+ * aggregation; Eq. 13-15: local window, top-k, union; Eq. 16: sparse
+ * reconstruction; Eq. 17: sink concatenation; Eq. 18: attention with RoPE).
+ *
+ * General rules
+ *   - Unless an argument is documented as HOST memory, every data pointer is a
+ *     DEVICE pointer owned by the caller.  The library never allocates or
+ *     frees device memory, keeps no state between calls and never
+ *     synchronises the stream (except s4r_decode_step_host, see there).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
+ *     work of a call is enqueued on it, in order.
+ *   - Every entry point returns S4R_OK or a negative s4r_status_t.  Misuse
+ *     that the host can see is rejected before anything is launched.
+ *   - `dev_status` (may be NULL) is a device int32 the kernels OR flags into
+ *     (S4R_DEV_*); kernels never trap and never spin without a bound.
+ *   - Tensors are dense, row-major, last index fastest.  Storage type
+ *     (`dtype`) applies to K, V, q, sinks, bases and coefficients alike.
+ *   - There is no CPU fallback and no other GPU architecture: on a device that
+ *     is not compute capability 10.x the calls return S4R_ERR_ARCH.
+ *
+ * Notation (paper, App. A): B batch, H_q query heads, h_kv KV heads,
+ * G = H_q / h_kv, d_h head dimension, D' = h_kv * d_h, r rank, s sink count,
+ * L non-sink cache length INCLUDING the current token (Sec. 3.2.2), W local
+ * window, k global top-k budget.
+ */
+#ifndef S4R_H_
+#define S4R_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  S4R_OK = 0,
+  S4R_ERR_INVALID_ARG = -1, /* NULL pointer, negative size, inconsistent geometry          */
+  S4R_ERR_UNSUPPORTED = -2, /* valid in the paper, not built here (see each call)           */
+  S4R_ERR_WORKSPACE = -3,   /* workspace missing, misaligned (256 B) or too small           */
+  S4R_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, bad stream, ...)   */
+  S4R_ERR_ARCH = -5         /* current device is not sm_100                                 */
+} s4r_status_t;
+
+/* flags OR-ed into *dev_status by kernels */
+#define S4R_DEV_TIMEOUT 1  /* a bounded wait (mbarrier) expired; results of that call are invalid */
+#define S4R_DEV_BOUNDS 2   /* coef_len[b] outside [0, max_len] or cache full on append; clamped   */
+
+#define S4R_F32 0
+#define S4R_BF16 1
+
+#define S4R_POOL_MAX 0
+#define S4R_POOL_AVG 1
+#define S4R_GROUP_MEAN 0
+#define S4R_GROUP_MAX 1
+
+/* Layer geometry, validated on every call.
+ * Supported: head_dim 128 (also 64), G <= 8, rank_k and rank_v multiples of 8 in [8, 512],
+ * rank_k == rank_v not required. */
+typedef struct {
+  int32_t batch;         /* B >= 1                                                        */
+  int32_t n_q_heads;     /* H_q, multiple of n_kv_heads                                    */
+  int32_t n_kv_heads;    /* h_kv                                                           */
+  int32_t head_dim;      /* d_h                                                            */
+  int32_t rank_k;        /* r of the key subspace                                          */
+  int32_t rank_v;        /* r of the value subspace                                        */
+  int32_t sink_count;    /* s >= 0 (Sec. 3.1.1; s = 0 is the "without sinks" ablation)     */
+  int32_t dtype;         /* S4R_BF16 or S4R_F32                                            */
+  int64_t coef_capacity; /* rows allocated per sequence in coef_k and coef_v               */
+} s4r_layer_t;
+
+/* Switches of the relevance estimate (Eq. 9-12); the paper's defaults are
+ * pool_kernel 7, max pooling, mean aggregation. */
+typedef struct {
+  int32_t score_window; /* number of query-coefficient rows scored; only 1 (the current query) is built */
+  int32_t pool_kernel;  /* kappa, odd, 1 = no pooling, <= 31                              */
+  int32_t pool_mode;    /* S4R_POOL_MAX | S4R_POOL_AVG                                    */
+  int32_t group_mode;   /* S4R_GROUP_MEAN | S4R_GROUP_MAX                                 */
+} s4r_score_t;
+
+/* RoPE of Eq. 18: rotate-half pairing (i, i + d_h/2), inv_freq_i = theta^(-2i/d_h), no scaling.
+ * Sink j sits at position j, non-sink row l at s + l, the query at s + L - 1.  theta <= 0: off. */
+typedef struct {
+  float theta;
+  int32_t reserved; /* must be 0 */
+} s4r_rope_t;
+
+/* Bytes of scratch s4r_decode_step / s4r_compress need for this geometry when no sequence is longer
+ * than max_len non-sink rows (compress: max_len = T - s).  0 on invalid arguments.  The workspace
+ * must be 256-byte aligned; its contents are undefined between calls. */
+size_t s4r_workspace_bytes(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k);
+
+/* Prefill-side projection (Sec. 3.1.1 sink split + Eq. 3), per sequence b:
+ *   sink_k[b] = K[b, 0:s], sink_v[b] = V[b, 0:s]            (verbatim copies)
+ *   coef_k[b, 0:T-s] = K[b, s:T] * key_basis[b]              (fp32 accumulate, one rounding to dtype)
+ *   coef_v[b, 0:T-s] = V[b, s:T] * value_basis[b]
+ *   coef_len[b] = T - s
+ * K, V          [B, T, D'] pre-RoPE keys / values of the prompt, T >= s, T - s <= coef_capacity
+ * key_basis     [B, D', rank_k], value_basis [B, D', rank_v]   (Eq. 2; computed by the caller)
+ * norm_stats    reserved, must be NULL: the paper normalises only the sampled rows that build the
+ *               bases (Eq. 1) and projects the raw rows (Eq. 3)
+ * sink_k/v out  [B, s, D'];  coef_k out [B, coef_capacity, rank_k];  coef_v likewise;  coef_len out [B]
+ */
+int s4r_compress(const s4r_layer_t *layer, const void *K, const void *V, int64_t T, const void *key_basis,
+                 const void *value_basis, const void *norm_stats, void *sink_k, void *sink_v, void *coef_k,
+                 void *coef_v, int32_t *coef_len, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                 void *stream);
+
+/* Decode-time cache update (Eq. 5 for K and V, Eq. 6), per sequence b:
+ *   coef_k[b, coef_len[b]] = k_t[b] * key_basis[b];  coef_v likewise;  coef_len[b] += 1
+ * k_t, v_t [B, D'] pre-RoPE.  A full cache (coef_len[b] == coef_capacity) sets S4R_DEV_BOUNDS and
+ * leaves that sequence unchanged. */
+int s4r_append(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *key_basis,
+               const void *value_basis, void *coef_k, void *coef_v, int32_t *coef_len, int32_t *dev_status,
+               void *stream);
+
+/* One decode step of one layer for the whole batch (Sec. 3.2.2-3.2.3), per sequence b with L = coef_len[b]
+ * (the current token already appended):
+ *   1. c^Q[g] = Q~[g] key_basis, Q~[g] = concat over KV heads kv of query head kv*G+g        (Eq. 5)
+ *   2. Z[g, l] = <c^Q[g], coef_k[l]> / sqrt(rank_k), l in [0, L)                              (Eq. 8)
+ *   3. A[g, :] = softmax over l; pooled over kappa neighbours; aggregated over g -> score[l]   (Eq. 9-12)
+ *   4. W_eff = min(window, L); local = [L - W_eff, L); k_eff = min(top_k, L - W_eff);
+ *      global = the k_eff best of score[0 : L - W_eff], ties to the lower index                (Eq. 13-15)
+ *   5. selected rows are reconstructed on chip, K^ = coef_k[sel] key_basis^T, V^ likewise     (Eq. 16),
+ *      joined with the sinks (Eq. 17), rotated (RoPE, if on) and attended                      (Eq. 18)
+ * q             [B, H_q, d_h] pre-RoPE
+ * max_len       host-known upper bound of every coef_len[b] (<= coef_capacity); sizes grids and scratch
+ * window, top_k W >= 0 and k >= 0
+ * out           [B, H_q, d_h], type out_dtype (S4R_F32 or S4R_BF16)
+ * sel_idx       [B, window + top_k] int32: global picks ascending, then the local window ascending, as
+ *               non-sink indices (absolute position = s + index); unused tail = -1.  Sinks are always
+ *               attended and never listed.
+ * sel_count     [B] int32 = W_eff + k_eff
+ * Returns S4R_ERR_UNSUPPORTED for score->score_window != 1. */
+int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
+                    const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,
+                    const void *value_basis, int64_t max_len, int32_t window, int32_t top_k,
+                    const s4r_score_t *score, const s4r_rope_t *rope, void *out, int32_t out_dtype,
+                    int32_t *sel_idx, int32_t *sel_count, void *workspace, size_t workspace_bytes,
+                    int32_t *dev_status, void *stream);
+
+/* Same step for callers whose per-step data lives in HOST memory: q_host, out_host, sel_idx_host and
+ * sel_count_host are host buffers (pinned memory makes the copies asynchronous); q_dev, out_dev,
+ * sel_idx_dev, sel_count_dev are device staging buffers of the same shapes.  The call copies q to the
+ * device, runs s4r_decode_step, copies out / sel_idx / sel_count back and waits for the stream, so the
+ * host buffers are valid on return.  The cache itself (sinks, coefficients, bases) stays on the device:
+ * it is the persistent state of Sec. 3.3, not a per-step input. */
+int s4r_decode_step_host(const s4r_layer_t *layer, const void *q_host, void *q_dev, const void *sink_k,
+                         const void *sink_v, const void *coef_k, const void *coef_v, const int32_t *coef_len,
+                         const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                         int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out_host,
+                         void *out_dev, int32_t out_dtype, int32_t *sel_idx_host, int32_t *sel_idx_dev,
+                         int32_t *sel_count_host, int32_t *sel_count_dev, void *workspace,
+                         size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/* Host helpers (no GPU work). */
+/* Eq. 14: k = max(floor(rho * L) - W, 0). */
+int64_t s4r_top_k_from_ratio(double rho, int64_t L, int32_t window);
+/* Largest rank r (multiple of `multiple`) whose persistent memory ratio of Sec. 3.3,
+ * (s D' + L r + G W r / 2 + D' r) / ((s + L) D'), does not exceed eta; 0 if none. */
+int32_t s4r_rank_for_ratio(double eta, int64_t L, int32_t sink_count, int32_t d_kv, int32_t group,
+                           int32_t query_window, int32_t multiple);
+/* Number of kernel launches the last s4r_decode_step / s4r_compress / s4r_append call on this thread made. */
+int32_t s4r_last_launch_count(void);
+
+const char *s4r_strerror(int status);
+int s4r_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* S4R_H_ */

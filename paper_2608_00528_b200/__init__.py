@@ -1,0 +1,236 @@
+"""Thin Python binding of libs4r.so (the C ABI declared in include/s4r.h).
+
+Argument marshalling only: every step of the S4R path runs in the library's CUDA kernels.  Torch is used
+for device memory and streams.  There is no CPU fallback: importing works without a GPU (the library loads
+and its symbols can be inspected), but every compute call needs a B200 and raises otherwise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import _build
+
+S4R_F32, S4R_BF16 = 0, 1
+POOL_MAX, POOL_AVG = 0, 1
+GROUP_MEAN, GROUP_MAX = 0, 1
+DEV_TIMEOUT, DEV_BOUNDS = 1, 2
+
+EXPORTS = ("s4r_workspace_bytes", "s4r_compress", "s4r_append", "s4r_decode_step", "s4r_decode_step_host",
+           "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_strerror", "s4r_version")
+
+
+class S4RError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} ({status})")
+
+
+class _Layer(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("rank_k", ctypes.c_int32), ("rank_v", ctypes.c_int32),
+                ("sink_count", ctypes.c_int32), ("dtype", ctypes.c_int32), ("coef_capacity", ctypes.c_int64)]
+
+
+class _Score(ctypes.Structure):
+    _fields_ = [("score_window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("pool_mode", ctypes.c_int32),
+                ("group_mode", ctypes.c_int32)]
+
+
+class _Rope(ctypes.Structure):
+    _fields_ = [("theta", ctypes.c_float), ("reserved", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True):
+    """Load libs4r.so (building it first if the sources are newer and nvcc is present)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing and _build.needs_build():
+        try:
+            _build.build()
+        except Exception:
+            if not os.path.exists(_build.LIB):
+                raise
+    if not os.path.exists(_build.LIB):
+        raise ImportError("libs4r.so is missing; run `python -m paper_2608_00528_b200._build`")
+    lib = ctypes.CDLL(_build.LIB)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    lp, sp, rp = ctypes.POINTER(_Layer), ctypes.POINTER(_Score), ctypes.POINTER(_Rope)
+    lib.s4r_workspace_bytes.restype = sz
+    lib.s4r_workspace_bytes.argtypes = [lp, i64, i32, i32]
+    lib.s4r_compress.restype = ctypes.c_int
+    lib.s4r_compress.argtypes = [lp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.s4r_append.restype = ctypes.c_int
+    lib.s4r_append.argtypes = [lp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.s4r_decode_step.restype = ctypes.c_int
+    lib.s4r_decode_step.argtypes = [lp, vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, sp, rp, vp, i32, vp, vp, vp,
+                                    sz, vp, vp]
+    lib.s4r_decode_step_host.restype = ctypes.c_int
+    lib.s4r_decode_step_host.argtypes = [lp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, sp, rp, vp, vp, i32,
+                                         vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.s4r_top_k_from_ratio.restype = i64
+    lib.s4r_top_k_from_ratio.argtypes = [ctypes.c_double, i64, i32]
+    lib.s4r_rank_for_ratio.restype = i32
+    lib.s4r_rank_for_ratio.argtypes = [ctypes.c_double, i64, i32, i32, i32, i32, i32]
+    lib.s4r_last_launch_count.restype = i32
+    lib.s4r_last_launch_count.argtypes = []
+    lib.s4r_strerror.restype = ctypes.c_char_p
+    lib.s4r_strerror.argtypes = [ctypes.c_int]
+    lib.s4r_version.restype = ctypes.c_int
+    lib.s4r_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def strerror(status: int) -> str:
+    return load().s4r_strerror(int(status)).decode()
+
+
+def version() -> int:
+    return load().s4r_version()
+
+
+def top_k_from_ratio(rho: float, cache_len: int, window: int) -> int:
+    return int(load().s4r_top_k_from_ratio(float(rho), int(cache_len), int(window)))
+
+
+def rank_for_ratio(eta: float, cache_len: int, sink_count: int, d_kv: int, group: int, query_window: int,
+                   multiple: int = 8) -> int:
+    return int(load().s4r_rank_for_ratio(float(eta), int(cache_len), int(sink_count), int(d_kv), int(group),
+                                         int(query_window), int(multiple)))
+
+
+def last_launch_count() -> int:
+    return int(load().s4r_last_launch_count())
+
+
+@dataclass
+class Layer:
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    rank_k: int
+    rank_v: int
+    sink_count: int
+    dtype: int                 # S4R_BF16 | S4R_F32
+    coef_capacity: int
+
+    def c(self) -> _Layer:
+        return _Layer(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.rank_k, self.rank_v,
+                      self.sink_count, self.dtype, self.coef_capacity)
+
+    @property
+    def d_kv(self) -> int:
+        return self.n_kv_heads * self.head_dim
+
+    @property
+    def torch_dtype(self) -> torch.dtype:
+        return torch.bfloat16 if self.dtype == S4R_BF16 else torch.float32
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return ctypes.c_void_p(t)
+    assert t.is_contiguous(), "tensors passed to libs4r must be contiguous"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _need_cuda(*tensors):
+    if not torch.cuda.is_available():
+        raise RuntimeError("libs4r needs a CUDA device (sm_100); there is no CPU fallback")
+    for t in tensors:
+        if t is not None and not isinstance(t, int) and not t.is_cuda:
+            raise ValueError("expected CUDA tensors")
+
+
+def workspace_bytes(layer: Layer, max_len: int, window: int, top_k: int) -> int:
+    return int(load().s4r_workspace_bytes(ctypes.byref(layer.c()), int(max_len), int(window), int(top_k)))
+
+
+def alloc_workspace(layer: Layer, max_len: int, window: int, top_k: int, device="cuda") -> torch.Tensor:
+    n = workspace_bytes(layer, max_len, window, top_k)
+    if n == 0:
+        raise S4RError(-1, "s4r_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def compress(layer: Layer, K, V, key_basis, value_basis, sink_k, sink_v, coef_k, coef_v, coef_len,
+             workspace=None, dev_status=None, stream=None, norm_stats=None):
+    """s4r_compress: K, V [B, T, D'] -> sinks, coefficient caches, coef_len (all preallocated by the caller)."""
+    _need_cuda(K, V, key_basis, value_basis, coef_k, coef_v, coef_len)
+    T = K.shape[1]
+    rc = load().s4r_compress(ctypes.byref(layer.c()), _ptr(K), _ptr(V), int(T), _ptr(key_basis), _ptr(value_basis),
+                             _ptr(norm_stats), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k), _ptr(coef_v),
+                             _ptr(coef_len), _ptr(workspace), 0 if workspace is None else workspace.numel(),
+                             _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_compress")
+
+
+def append(layer: Layer, k_t, v_t, key_basis, value_basis, coef_k, coef_v, coef_len, dev_status=None, stream=None):
+    """s4r_append: project one new key/value row per sequence and append it to the coefficient caches."""
+    _need_cuda(k_t, v_t, key_basis, value_basis, coef_k, coef_v, coef_len)
+    rc = load().s4r_append(ctypes.byref(layer.c()), _ptr(k_t), _ptr(v_t), _ptr(key_basis), _ptr(value_basis),
+                           _ptr(coef_k), _ptr(coef_v), _ptr(coef_len), _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_append")
+
+
+def _score_rope(pool_kernel, pool_mode, group_mode, score_window, theta):
+    return _Score(score_window, pool_kernel, pool_mode, group_mode), _Rope(float(theta), 0)
+
+
+def decode_step(layer: Layer, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis, max_len: int,
+                window: int, top_k: int, out, sel_idx, sel_count, workspace, *, pool_kernel: int = 7,
+                pool_mode: int = POOL_MAX, group_mode: int = GROUP_MEAN, score_window: int = 1,
+                rope_theta: float = 0.0, dev_status=None, stream=None):
+    """s4r_decode_step: writes `out` [B, H_q, d_h], `sel_idx` [B, window + top_k] and `sel_count` [B]."""
+    _need_cuda(q, coef_k, coef_v, coef_len, key_basis, value_basis, out, sel_idx, sel_count, workspace)
+    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, score_window, rope_theta)
+    out_dtype = S4R_BF16 if out.dtype == torch.bfloat16 else S4R_F32
+    rc = load().s4r_decode_step(ctypes.byref(layer.c()), _ptr(q), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k),
+                                _ptr(coef_v), _ptr(coef_len), _ptr(key_basis), _ptr(value_basis), int(max_len),
+                                int(window), int(top_k), ctypes.byref(sc), ctypes.byref(rp), _ptr(out), out_dtype,
+                                _ptr(sel_idx), _ptr(sel_count), _ptr(workspace), workspace.numel(),
+                                _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_decode_step")
+
+
+def decode_step_host(layer: Layer, q_host, q_dev, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,
+                     max_len: int, window: int, top_k: int, out_host, out_dev, sel_idx_host, sel_idx_dev,
+                     sel_count_host, sel_count_dev, workspace, *, pool_kernel: int = 7, pool_mode: int = POOL_MAX,
+                     group_mode: int = GROUP_MEAN, score_window: int = 1, rope_theta: float = 0.0, dev_status=None,
+                     stream=None):
+    """s4r_decode_step_host: q / out / sel_idx / sel_count live in host memory; returns after the results landed."""
+    _need_cuda(q_dev, coef_k, coef_v, coef_len, key_basis, value_basis, out_dev, sel_idx_dev, sel_count_dev, workspace)
+    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, score_window, rope_theta)
+    out_dtype = S4R_BF16 if out_dev.dtype == torch.bfloat16 else S4R_F32
+    rc = load().s4r_decode_step_host(
+        ctypes.byref(layer.c()), _ptr(q_host), _ptr(q_dev), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k), _ptr(coef_v),
+        _ptr(coef_len), _ptr(key_basis), _ptr(value_basis), int(max_len), int(window), int(top_k), ctypes.byref(sc),
+        ctypes.byref(rp), _ptr(out_host), _ptr(out_dev), out_dtype, _ptr(sel_idx_host), _ptr(sel_idx_dev),
+        _ptr(sel_count_host), _ptr(sel_count_dev), _ptr(workspace), workspace.numel(), _ptr(dev_status),
+        _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_decode_step_host")

@@ -1,0 +1,232 @@
+// C ABI of the S4R library: argument validation, workspace plan, kernel dispatch.  See include/s4r.h.
+#include <math.h>
+#include <string.h>
+
+#include "s4r_internal.h"
+
+namespace s4r {
+
+static bool layer_ok(const s4r_layer_t *l, Layer *out) {
+  if (!l) return false;
+  if (l->batch < 1 || l->n_q_heads < 1 || l->n_kv_heads < 1 || l->head_dim < 1) return false;
+  if (l->n_q_heads % l->n_kv_heads) return false;
+  if (l->rank_k < 1 || l->rank_v < 1 || l->sink_count < 0 || l->coef_capacity < 0) return false;
+  if (l->dtype != S4R_BF16 && l->dtype != S4R_F32) return false;
+  out->B = l->batch; out->Hq = l->n_q_heads; out->Hkv = l->n_kv_heads; out->dh = l->head_dim;
+  out->rk = l->rank_k; out->rv = l->rank_v; out->s = l->sink_count; out->dtype = l->dtype;
+  out->G = l->n_q_heads / l->n_kv_heads; out->D = l->n_kv_heads * l->head_dim; out->cap = l->coef_capacity;
+  return true;
+}
+
+static int layer_supported(const Layer &ly) {
+  if (ly.dh != 128 && ly.dh != 64) return S4R_ERR_UNSUPPORTED;
+  if (ly.G > kMaxGroup) return S4R_ERR_UNSUPPORTED;
+  if (ly.rk % 8 || ly.rv % 8 || ly.rk > 512 || ly.rv > 512) return S4R_ERR_UNSUPPORTED;
+  if (ly.s > 64) return S4R_ERR_UNSUPPORTED;
+  if (ly.cap > 0x7fffffffLL - 4096 || ly.B > 65535 || ly.Hkv > 65535 || ly.Hq > 65535) return S4R_ERR_UNSUPPORTED;
+  return S4R_OK;
+}
+
+static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k, DecodePlan *p) {
+  if (max_len < 0 || window < 0 || top_k < 0) return false;
+  if ((int64_t)window + top_k > 0x3fffffff) return false;
+  p->max_len = max_len;
+  p->z_stride = (int64_t)align_up((size_t)(max_len > 0 ? max_len : 1), 4);
+  p->n_scan_chunks = (int)((max_len + kScanRows - 1) / kScanRows);
+  if (p->n_scan_chunks < 1) p->n_scan_chunks = 1;
+  p->att_tok = kAttTok;
+  p->n_att_tiles = (window + top_k + p->att_tok - 1) / p->att_tok;
+  int cl = 1;
+  while (cl < kMaxCluster && max_len > (int64_t)cl * 8192) cl *= 2;
+  p->cluster = cl;
+  size_t off = 0;
+  p->off_cq = off;      off = align_up(off + sizeof(float) * ly.B * ly.G * ly.rk, 256);
+  p->off_z = off;       off = align_up(off + sizeof(float) * ly.B * ly.G * p->z_stride, 256);
+  p->off_part = off;    off = align_up(off + sizeof(float2) * ly.B * p->n_scan_chunks * kMaxGroup, 256);
+  p->off_score = off;   off = align_up(off + sizeof(float) * ly.B * p->z_stride, 256);
+  p->off_att = off;     off = align_up(off + sizeof(float) * ly.B * ly.Hq * (size_t)p->n_att_tiles * ly.dh, 256);
+  p->off_att_ms = off;  off = align_up(off + sizeof(float2) * ly.B * ly.Hq * (size_t)p->n_att_tiles, 256);
+  p->off_basis_t = off;
+  p->total = off > 256 ? off : 256;
+  return true;
+}
+
+static int check_arch() {
+  static int cached[64];  // 0 unknown, 1 ok, 2 wrong architecture
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return S4R_ERR_CUDA;
+  if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev] == 1 ? S4R_OK : S4R_ERR_ARCH;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return S4R_ERR_CUDA;
+  if (dev >= 0 && dev < 64) cached[dev] = (major == 10) ? 1 : 2;
+  return major == 10 ? S4R_OK : S4R_ERR_ARCH;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace s4r
+
+using namespace s4r;
+
+extern "C" {
+
+size_t s4r_workspace_bytes(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k) {
+  Layer ly;
+  DecodePlan p;
+  if (!layer_ok(layer, &ly) || layer_supported(ly) != S4R_OK) return 0;
+  if (!plan_decode(ly, max_len, window, top_k, &p)) return 0;
+  return p.total;
+}
+
+int s4r_compress(const s4r_layer_t *layer, const void *K, const void *V, int64_t T, const void *key_basis,
+                 const void *value_basis, const void *norm_stats, void *sink_k, void *sink_v, void *coef_k,
+                 void *coef_v, int32_t *coef_len, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                 void *stream) {
+  (void)workspace; (void)workspace_bytes; (void)dev_status;
+  launch_counter() = 0;
+  Layer ly;
+  if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
+  if (int rc = layer_supported(ly)) return rc;
+  if (norm_stats != nullptr) return S4R_ERR_INVALID_ARG;
+  if (!K || !V || !key_basis || !value_basis || !coef_k || !coef_v || !coef_len) return S4R_ERR_INVALID_ARG;
+  if (ly.s > 0 && (!sink_k || !sink_v)) return S4R_ERR_INVALID_ARG;
+  if (T < ly.s || T - ly.s > ly.cap) return S4R_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(key_basis) || !aligned16(value_basis) || !aligned16(coef_k) ||
+      !aligned16(coef_v))
+    return S4R_ERR_INVALID_ARG;
+  if (int rc = check_arch()) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (launch_compress_generic(ly, K, key_basis, ly.rk, sink_k, coef_k, T, st) != cudaSuccess) return S4R_ERR_CUDA;
+  if (launch_compress_generic(ly, V, value_basis, ly.rv, sink_v, coef_v, T, st) != cudaSuccess) return S4R_ERR_CUDA;
+  if (launch_set_len(ly, coef_len, T, st) != cudaSuccess) return S4R_ERR_CUDA;
+  return S4R_OK;
+}
+
+int s4r_append(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *key_basis,
+               const void *value_basis, void *coef_k, void *coef_v, int32_t *coef_len, int32_t *dev_status,
+               void *stream) {
+  launch_counter() = 0;
+  Layer ly;
+  if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
+  if (int rc = layer_supported(ly)) return rc;
+  if (!k_t || !v_t || !key_basis || !value_basis || !coef_k || !coef_v || !coef_len) return S4R_ERR_INVALID_ARG;
+  if (!aligned16(key_basis) || !aligned16(value_basis) || !aligned16(coef_k) || !aligned16(coef_v))
+    return S4R_ERR_INVALID_ARG;
+  if (int rc = check_arch()) return rc;
+  if (launch_append(ly, k_t, v_t, key_basis, value_basis, coef_k, coef_v, coef_len, dev_status,
+                    (cudaStream_t)stream) != cudaSuccess)
+    return S4R_ERR_CUDA;
+  return S4R_OK;
+}
+
+int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
+                    const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,
+                    const void *value_basis, int64_t max_len, int32_t window, int32_t top_k,
+                    const s4r_score_t *score, const s4r_rope_t *rope, void *out, int32_t out_dtype,
+                    int32_t *sel_idx, int32_t *sel_count, void *workspace, size_t workspace_bytes,
+                    int32_t *dev_status, void *stream) {
+  launch_counter() = 0;
+  StepArgs a;
+  if (!layer_ok(layer, &a.ly)) return S4R_ERR_INVALID_ARG;
+  const Layer &ly = a.ly;
+  if (int rc = layer_supported(ly)) return rc;
+  if (!q || !coef_k || !coef_v || !coef_len || !key_basis || !value_basis || !out || !sel_idx || !sel_count)
+    return S4R_ERR_INVALID_ARG;
+  if (ly.s > 0 && (!sink_k || !sink_v)) return S4R_ERR_INVALID_ARG;
+  if (out_dtype != S4R_F32 && out_dtype != S4R_BF16) return S4R_ERR_INVALID_ARG;
+  if (max_len < 0 || max_len > ly.cap || window < 0 || top_k < 0) return S4R_ERR_INVALID_ARG;
+  s4r_score_t sc = {1, 7, S4R_POOL_MAX, S4R_GROUP_MEAN};
+  if (score) sc = *score;
+  if (sc.score_window < 1 || sc.pool_kernel < 1 || (sc.pool_kernel & 1) == 0) return S4R_ERR_INVALID_ARG;
+  if (sc.pool_mode != S4R_POOL_MAX && sc.pool_mode != S4R_POOL_AVG) return S4R_ERR_INVALID_ARG;
+  if (sc.group_mode != S4R_GROUP_MEAN && sc.group_mode != S4R_GROUP_MAX) return S4R_ERR_INVALID_ARG;
+  if (sc.score_window != 1) return S4R_ERR_UNSUPPORTED;
+  if (sc.pool_kernel > 2 * kMaxPoolHalf + 1) return S4R_ERR_UNSUPPORTED;
+  if (rope && rope->reserved != 0) return S4R_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(coef_k) || !aligned16(coef_v) || !aligned16(key_basis) || !aligned16(value_basis))
+    return S4R_ERR_INVALID_ARG;
+  if (!plan_decode(ly, max_len, window, top_k, &a.plan)) return S4R_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < a.plan.total)
+    return S4R_ERR_WORKSPACE;
+  if (int rc = check_arch()) return rc;
+  a.q = q; a.sink_k = sink_k; a.sink_v = sink_v; a.coef_k = coef_k; a.coef_v = coef_v; a.coef_len = coef_len;
+  a.basis_k = key_basis; a.basis_v = value_basis; a.window = window; a.top_k = top_k; a.kappa = sc.pool_kernel;
+  a.pool_mode = sc.pool_mode; a.group_mode = sc.group_mode; a.theta = rope ? rope->theta : 0.f; a.out = out;
+  a.out_dtype = out_dtype; a.sel_idx = sel_idx; a.sel_count = sel_count; a.ws = (char *)workspace;
+  a.dev_status = dev_status; a.stream = (cudaStream_t)stream;
+  if (launch_qproj(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (launch_scan_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (launch_select(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (launch_attend_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (launch_merge(a) != cudaSuccess) return S4R_ERR_CUDA;
+  return S4R_OK;
+}
+
+int s4r_decode_step_host(const s4r_layer_t *layer, const void *q_host, void *q_dev, const void *sink_k,
+                         const void *sink_v, const void *coef_k, const void *coef_v, const int32_t *coef_len,
+                         const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                         int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out_host,
+                         void *out_dev, int32_t out_dtype, int32_t *sel_idx_host, int32_t *sel_idx_dev,
+                         int32_t *sel_count_host, int32_t *sel_count_dev, void *workspace,
+                         size_t workspace_bytes, int32_t *dev_status, void *stream) {
+  Layer ly;
+  if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
+  if (!q_host || !q_dev || !out_host || !out_dev || !sel_idx_host || !sel_idx_dev || !sel_count_host ||
+      !sel_count_dev || window < 0 || top_k < 0)
+    return S4R_ERR_INVALID_ARG;
+  if (out_dtype != S4R_F32 && out_dtype != S4R_BF16) return S4R_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t esz = ly.dtype == S4R_BF16 ? 2 : 4, osz = out_dtype == S4R_BF16 ? 2 : 4;
+  const size_t nq = (size_t)ly.B * ly.Hq * ly.dh;
+  if (cudaMemcpyAsync(q_dev, q_host, nq * esz, cudaMemcpyHostToDevice, st) != cudaSuccess) return S4R_ERR_CUDA;
+  int rc = s4r_decode_step(layer, q_dev, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis, max_len,
+                           window, top_k, score, rope, out_dev, out_dtype, sel_idx_dev, sel_count_dev, workspace,
+                           workspace_bytes, dev_status, stream);
+  if (rc != S4R_OK) return rc;
+  if (cudaMemcpyAsync(out_host, out_dev, nq * osz, cudaMemcpyDeviceToHost, st) != cudaSuccess) return S4R_ERR_CUDA;
+  if (cudaMemcpyAsync(sel_idx_host, sel_idx_dev, sizeof(int32_t) * ly.B * ((size_t)window + top_k),
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return S4R_ERR_CUDA;
+  if (cudaMemcpyAsync(sel_count_host, sel_count_dev, sizeof(int32_t) * ly.B, cudaMemcpyDeviceToHost, st) !=
+      cudaSuccess)
+    return S4R_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return S4R_ERR_CUDA;
+  return S4R_OK;
+}
+
+int64_t s4r_top_k_from_ratio(double rho, int64_t L, int32_t window) {
+  if (!(rho >= 0.0) || L < 0) return 0;
+  int64_t m = (int64_t)floor(rho * (double)L) - window;
+  return m > 0 ? m : 0;
+}
+
+int32_t s4r_rank_for_ratio(double eta, int64_t L, int32_t sink_count, int32_t d_kv, int32_t group,
+                           int32_t query_window, int32_t multiple) {
+  if (multiple < 1 || d_kv < 1 || L < 0 || sink_count < 0) return 0;
+  // (s D' + L r + G W r / 2 + D' r) / ((s + L) D') <= eta   <=>   r <= (eta (s + L) D' - s D') / (L + G W / 2 + D')
+  const double num = eta * (double)(sink_count + L) * d_kv - (double)sink_count * d_kv;
+  const double den = (double)L + 0.5 * group * query_window + d_kv;
+  if (num <= 0 || den <= 0) return 0;
+  int64_t r = (int64_t)floor(num / den);
+  r -= r % multiple;
+  if (r > d_kv) r = d_kv - d_kv % multiple;
+  return r > 0 ? (int32_t)r : 0;
+}
+
+int32_t s4r_last_launch_count(void) { return launch_counter(); }
+
+const char *s4r_strerror(int status) {
+  switch (status) {
+    case S4R_OK: return "ok";
+    case S4R_ERR_INVALID_ARG: return "invalid argument";
+    case S4R_ERR_UNSUPPORTED: return "unsupported configuration";
+    case S4R_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case S4R_ERR_CUDA: return "CUDA runtime error";
+    case S4R_ERR_ARCH: return "device is not sm_100";
+    default: return "unknown status";
+  }
+}
+
+int s4r_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,108 @@
+// Shared device/host helpers of the S4R library: storage-type loads, reductions, RoPE angles, launch plan.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/s4r.h"
+
+namespace s4r {
+
+constexpr int kMaxGroup = 8;       // G <= 8
+constexpr int kMaxPoolHalf = 15;   // kappa <= 31
+constexpr int kScanRows = 1024;    // rows of C^K per scan CTA (also the granularity of the softmax partials)
+constexpr int kAttTok = 32;        // selected rows per CTA in the generic reconstruct+attend kernel
+constexpr int kSelThreads = 1024;  // threads per CTA of the selection kernel (one position each per tile)
+constexpr int kMaxCluster = 8;     // portable cluster size
+
+// ---- storage-type helpers -------------------------------------------------------------------------
+
+template <typename T>
+struct Store;
+
+template <>
+struct Store<float> {
+  static constexpr int kVec = 4;  // elements per 16-byte vector
+  __device__ static inline float ld(const float *p) { return __ldg(p); }
+  __device__ static inline void ld_vec(const float *p, float (&v)[4]) {
+    float4 t = __ldg(reinterpret_cast<const float4 *>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+  __device__ static inline void st(float *p, float v) { *p = v; }
+};
+
+template <>
+struct Store<__nv_bfloat16> {
+  static constexpr int kVec = 8;
+  __device__ static inline float ld(const __nv_bfloat16 *p) {
+    return __bfloat162float(*p);
+  }
+  __device__ static inline void ld_vec(const __nv_bfloat16 *p, float (&v)[8]) {
+    uint4 t = __ldg(reinterpret_cast<const uint4 *>(p));
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static inline void st(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+// ---- reductions -----------------------------------------------------------------------------------
+
+__device__ inline float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ inline float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// online-softmax pair (m, s): s = sum exp(x - m)
+__device__ inline void ms_merge(float &m, float &s, float m2, float s2) {
+  float mn = fmaxf(m, m2);
+  if (mn == -INFINITY) { m = mn; s = 0.f; return; }
+  s = s * __expf(m - mn) + s2 * __expf(m2 - mn);
+  m = mn;
+}
+
+// ---- RoPE ------------------------------------------------------------------------------------------
+
+// inverse frequency of pair index i (0 <= i < d_h/2): theta^(-2i/d_h), in fp64
+__device__ inline double rope_inv_freq(int i, int head_dim, float theta) {
+  return exp2(-(2.0 * (double)i / (double)head_dim) * log2((double)theta));
+}
+
+// sin/cos of pos * inv_freq with the argument reduced in fp64 (positions reach 2^17 and beyond, where an
+// fp32 product has lost the fraction bits that matter)
+__device__ inline void rope_sincos(int pos, double inv_freq, float &sn, float &cs) {
+  const double kInv2Pi = 0.15915494309189533576888;
+  const double k2PiHi = 6.28318530717958623200;
+  const double k2PiLo = 2.44929359829470635445e-16;
+  double a = (double)pos * inv_freq;
+  double k = rint(a * kInv2Pi);
+  double red = fma(-k, k2PiHi, a);
+  red = fma(-k, k2PiLo, red);
+  sincosf((float)red, &sn, &cs);
+}
+
+// ---- host-side plan of one decode step -------------------------------------------------------------
+
+struct DecodePlan {
+  int64_t max_len;      // host-known bound of L
+  int64_t z_stride;     // floats per (b, g) row of Z
+  int n_scan_chunks;    // CTAs per sequence in the scan
+  int n_att_tiles;      // row tiles per sequence in the attention kernel
+  int cluster;          // CTAs per sequence in the selection kernel
+  int att_tok;          // selected rows per attention tile
+  size_t off_cq, off_z, off_part, off_score, off_att, off_att_ms, off_basis_t, total;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace s4r

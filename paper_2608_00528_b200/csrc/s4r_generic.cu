@@ -1,0 +1,895 @@
+// Generic kernels of the S4R decode step and prefill projection: any supported geometry, fp32 or bf16
+// storage, fp32 arithmetic on the CUDA cores.  They are the whole path for fp32 storage and the reference
+// implementation that the specialised sm_100a kernels (TMA / tcgen05) replace for bf16 storage.
+#include <cooperative_groups.h>
+
+#include "s4r_internal.h"
+
+namespace cg = cooperative_groups;
+
+namespace s4r {
+
+int &launch_counter() {
+  static thread_local int n = 0;
+  return n;
+}
+
+#define S4R_LAUNCH_CHECK()                      \
+  do {                                          \
+    ++launch_counter();                         \
+    cudaError_t e__ = cudaGetLastError();       \
+    if (e__ != cudaSuccess) return e__;         \
+  } while (0)
+
+__device__ inline int clamp_len(const int32_t *coef_len, int b, int64_t max_len, int32_t *dev_status) {
+  int L = coef_len[b];
+  if (L < 0 || (int64_t)L > max_len) {
+    if (dev_status && threadIdx.x == 0) atomicOr(dev_status, S4R_DEV_BOUNDS);
+    L = L < 0 ? 0 : (int)max_len;
+  }
+  return L;
+}
+
+// ======================================================================================================
+// Query projection (Eq. 5):  cq[b][g][c] = sum_d Qt[g][d] * B^K[b][d][c],  Qt[g][d] = q[b][(d/dh)*G+g][d%dh]
+// grid (ceil(r/32), B), block 256 = 32 columns x 8 row groups; row groups are summed in a fixed order.
+// ======================================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256) k_qproj(const T *__restrict__ q, const T *__restrict__ basis,
+                                               float *__restrict__ cq, int D, int r, int G, int dh, int Hq) {
+  extern __shared__ float xs[];  // [G][D]
+  __shared__ float red[8][kMaxGroup][32];
+  const int b = blockIdx.y;
+  const int col = blockIdx.x * 32 + (threadIdx.x & 31);
+  const int rg = threadIdx.x >> 5;
+  for (int i = threadIdx.x; i < G * D; i += 256) {
+    int g = i / D, d = i - g * D;
+    xs[i] = Store<T>::ld(q + ((size_t)b * Hq + (size_t)(d / dh) * G + g) * dh + (d % dh));
+  }
+  __syncthreads();
+  float acc[kMaxGroup];
+#pragma unroll
+  for (int g = 0; g < kMaxGroup; ++g) acc[g] = 0.f;
+  if (col < r) {
+    const T *bp = basis + (size_t)b * D * r + col;
+    for (int d = rg; d < D; d += 8) {
+      float bv = Store<T>::ld(bp + (size_t)d * r);
+#pragma unroll
+      for (int g = 0; g < kMaxGroup; ++g)
+        if (g < G) acc[g] = fmaf(xs[g * D + d], bv, acc[g]);
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < kMaxGroup; ++g) red[rg][g][threadIdx.x & 31] = acc[g];
+  __syncthreads();
+  if (rg == 0 && col < r) {
+    for (int g = 0; g < G; ++g) {
+      float s = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) s += red[k][g][threadIdx.x & 31];
+      cq[((size_t)b * G + g) * r + col] = s;
+    }
+  }
+}
+
+template <typename T>
+static cudaError_t qproj_t(const StepArgs &a) {
+  const Layer &ly = a.ly;
+  size_t smem = (size_t)ly.G * ly.D * sizeof(float);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k_qproj<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid((ly.rk + 31) / 32, ly.B);
+  k_qproj<T><<<grid, 256, smem, a.stream>>>((const T *)a.q, (const T *)a.basis_k, (float *)(a.ws + a.plan.off_cq),
+                                            ly.D, ly.rk, ly.G, ly.dh, ly.Hq);
+  S4R_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+cudaError_t launch_qproj(const StepArgs &a) {
+  return a.ly.dtype == S4R_BF16 ? qproj_t<__nv_bfloat16>(a) : qproj_t<float>(a);
+}
+
+// ======================================================================================================
+// Latent scoring (Eq. 8): Z[b][g][l] = <cq[b][g], C^K[b][l]> / sqrt(r), plus per-chunk softmax partials
+// (max, sum exp) of Eq. 9.  grid (n_chunks, B), block 256; 8 lanes share a row, 4 rows per warp pass.
+// ======================================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256) k_scan(const T *__restrict__ coef_k, const int32_t *__restrict__ coef_len,
+                                              const float *__restrict__ cq, float *__restrict__ Z,
+                                              float2 *__restrict__ part, int r, int G, int64_t cap,
+                                              int64_t max_len, int64_t z_stride, int n_chunks, float inv_sqrt_r,
+                                              int32_t *dev_status) {
+  constexpr int V = Store<T>::kVec;
+  __shared__ __align__(16) float cqs[kMaxGroup * 512];
+  __shared__ float red[8];
+  const int b = blockIdx.y, chunk = blockIdx.x;
+  const int L = clamp_len(coef_len, b, max_len, dev_status);
+  const int row0 = chunk * kScanRows;
+  const int row1 = min(L, row0 + kScanRows);
+  if (row0 >= L) {
+    if (threadIdx.x < G) part[((size_t)b * n_chunks + chunk) * kMaxGroup + threadIdx.x] = make_float2(-INFINITY, 0.f);
+    return;
+  }
+  for (int i = threadIdx.x; i < G * r; i += 256) cqs[i] = cq[(size_t)b * G * r + i];
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane & 7, slot = lane >> 3;
+  const int nvec = r / V;
+  const T *base = coef_k + (size_t)b * cap * r;
+  float *zb = Z + (size_t)b * G * z_stride;
+  for (int row = row0 + warp * 4 + slot; row < row0 + kScanRows; row += 32) {
+    const bool live = row < row1;
+    float acc[kMaxGroup];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) acc[g] = 0.f;
+    if (live) {
+      const T *rp = base + (size_t)row * r;
+      for (int c = sub; c < nvec; c += 8) {
+        float v[V];
+        Store<T>::ld_vec(rp + c * V, v);
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g) {
+          if (g < G) {
+            const float *cp = cqs + g * r + c * V;
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[g] = fmaf(v[e], cp[e], acc[g]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) {
+      if (g < G) {
+        float s = acc[g];
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        s += __shfl_xor_sync(0xffffffffu, s, 4);
+        if (live && sub == 0) zb[(size_t)g * z_stride + row] = s * inv_sqrt_r;
+      }
+    }
+  }
+  __syncthreads();
+  // softmax partials of this chunk, from the values just written (same block: visible after the barrier)
+  for (int g = 0; g < G; ++g) {
+    const float *zr = zb + (size_t)g * z_stride;
+    float m = -INFINITY;
+    for (int row = row0 + threadIdx.x; row < row1; row += 256) m = fmaxf(m, zr[row]);
+    m = warp_max(m);
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    m = red[0];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) m = fmaxf(m, red[k]);
+    __syncthreads();
+    float s = 0.f;
+    for (int row = row0 + threadIdx.x; row < row1; row += 256) s += expf(zr[row] - m);
+    s = warp_sum(s);
+    if (lane == 0) red[warp] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) t += red[k];
+      part[((size_t)b * n_chunks + chunk) * kMaxGroup + g] = make_float2(m, t);
+    }
+    __syncthreads();
+  }
+}
+
+cudaError_t launch_scan_generic(const StepArgs &a) {
+  const Layer &ly = a.ly;
+  dim3 grid(a.plan.n_scan_chunks, ly.B);
+  float *Z = (float *)(a.ws + a.plan.off_z);
+  float2 *part = (float2 *)(a.ws + a.plan.off_part);
+  const float *cq = (const float *)(a.ws + a.plan.off_cq);
+  float isr = (float)(1.0 / sqrt((double)ly.rk));
+  if (ly.dtype == S4R_BF16)
+    k_scan<__nv_bfloat16><<<grid, 256, 0, a.stream>>>((const __nv_bfloat16 *)a.coef_k, a.coef_len, cq, Z, part, ly.rk,
+                                                      ly.G, ly.cap, a.plan.max_len, a.plan.z_stride,
+                                                      a.plan.n_scan_chunks, isr, a.dev_status);
+  else
+    k_scan<float><<<grid, 256, 0, a.stream>>>((const float *)a.coef_k, a.coef_len, cq, Z, part, ly.rk, ly.G, ly.cap,
+                                              a.plan.max_len, a.plan.z_stride, a.plan.n_scan_chunks, isr,
+                                              a.dev_status);
+  S4R_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+// ======================================================================================================
+// Relevance + selection (Eq. 9-15).  One thread-block cluster per sequence; each CTA owns a contiguous
+// slice of the cache.  Scores are softmax probabilities (>= 0), so their fp32 bit patterns order like the
+// values; the k-th largest candidate is found by a 3-pass radix select (11 + 11 + 10 bits) whose
+// histograms are summed across the cluster through distributed shared memory, and the winners are written
+// in ascending index order (equal scores: lower index first).
+// ======================================================================================================
+struct SelParams {
+  const float *Z;
+  const float2 *part;
+  const int32_t *coef_len;
+  float *score;
+  int32_t *sel_idx, *sel_count;
+  int G, n_chunks, window, top_k, kappa, pool_mode, group_mode;
+  int64_t max_len, z_stride;
+  int32_t *dev_status;
+};
+
+// exclusive prefix sum over the block (kSelThreads threads); returns the exclusive value, total in *total
+__device__ inline unsigned block_excl_scan(unsigned v, unsigned *s_warp, unsigned *total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    unsigned t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    unsigned w = s_warp[lane];
+    unsigned winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    s_warp[lane] = winc - w;       // exclusive offset of each warp
+    if (lane == 31) s_warp[32] = winc;  // grand total
+  }
+  __syncthreads();
+  unsigned res = s_warp[warp] + inc - v;
+  *total = s_warp[32];
+  __syncthreads();
+  return res;
+}
+
+// Sum the per-CTA histograms of the cluster and locate the bin that holds the k_rem-th largest element
+// (bins are scanned from the top).  Returns the bin; *above = number of elements in higher bins.
+__device__ inline unsigned find_bin(cg::cluster_group &cluster, unsigned *s_hist, unsigned *s_warp, unsigned *s_bc,
+                                    int nbins, unsigned k_rem, unsigned *above) {
+  const int CL = cluster.num_blocks();
+  cluster.sync();  // every CTA's histogram is complete
+  const int t = threadIdx.x;
+  const int b0 = nbins - 1 - 2 * t, b1 = nbins - 2 - 2 * t;
+  unsigned c0 = 0, c1 = 0;
+  for (int rk = 0; rk < CL; ++rk) {
+    const unsigned *h = cluster.map_shared_rank(s_hist, rk);
+    if (b0 >= 0) c0 += h[b0];
+    if (b1 >= 0) c1 += h[b1];
+  }
+  unsigned total;
+  unsigned excl = block_excl_scan(c0 + c1, s_warp, &total);
+  if (b0 >= 0 && excl < k_rem && k_rem <= excl + c0) {
+    s_bc[0] = (unsigned)b0;
+    s_bc[1] = excl;
+  } else if (b1 >= 0 && excl + c0 < k_rem && k_rem <= excl + c0 + c1) {
+    s_bc[0] = (unsigned)b1;
+    s_bc[1] = excl + c0;
+  }
+  cluster.sync();  // remote reads done before anyone clears its histogram; also a block barrier for s_bc
+  *above = s_bc[1];
+  return s_bc[0];
+}
+
+__global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int CL = cluster.num_blocks();
+  const int rank = cluster.block_rank();
+  const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int HALO = 16;
+  __shared__ float s_p[kMaxGroup][kSelThreads + 2 * HALO];
+  __shared__ unsigned s_hist[2048];
+  __shared__ float s_M[kMaxGroup], s_iS[kMaxGroup];
+  __shared__ unsigned s_warp[33];
+  __shared__ unsigned s_bc[2];
+  __shared__ unsigned s_cnt[2];
+
+  const int L = clamp_len(p.coef_len, b, p.max_len, p.dev_status);
+  const int W_eff = min(p.window, L);
+  const int n_cand = L - W_eff;
+  const int k_eff = min(p.top_k, n_cand);
+  int32_t *out_idx = p.sel_idx + (size_t)b * (p.window + p.top_k);
+
+  if (rank == 0) {  // local window (Eq. 13), padding and count
+    for (int j = tid; j < W_eff; j += kSelThreads) out_idx[k_eff + j] = n_cand + j;
+    for (int j = k_eff + W_eff + tid; j < p.window + p.top_k; j += kSelThreads) out_idx[j] = -1;
+    if (tid == 0) p.sel_count[b] = k_eff + W_eff;
+  }
+  if (k_eff == 0) return;  // uniform over the cluster: nothing to rank
+
+  // ---- softmax normalisers of Eq. 9 from the scan's per-chunk partials
+  const int used_chunks = (L + kScanRows - 1) / kScanRows;
+  if (warp < p.G) {
+    const float2 *pp = p.part + (size_t)b * p.n_chunks * kMaxGroup + warp;
+    float m = -INFINITY;
+    for (int c = lane; c < used_chunks; c += 32) m = fmaxf(m, pp[(size_t)c * kMaxGroup].x);
+    m = warp_max(m);
+    float s = 0.f;
+    for (int c = lane; c < used_chunks; c += 32) {
+      float2 v = pp[(size_t)c * kMaxGroup];
+      s += v.y * expf(v.x - m);
+    }
+    s = warp_sum(s);
+    if (lane == 0) {
+      s_M[warp] = m;
+      s_iS[warp] = 1.f / s;
+    }
+  }
+  for (int i = tid; i < 2048; i += kSelThreads) s_hist[i] = 0;
+  __syncthreads();
+
+  // ---- scores of this CTA's slice (Eq. 9-12) + first histogram
+  int per = (L + CL - 1) / CL;
+  per = (per + 3) & ~3;
+  const int begin = min(L, rank * per), end = min(L, begin + per);
+  const int half = p.kappa >> 1;
+  const float *zb = p.Z + (size_t)b * p.G * p.z_stride;
+  float *score = p.score + (size_t)b * p.z_stride;
+  const float inv_kappa = 1.f / (float)p.kappa, inv_G = 1.f / (float)p.G;
+  for (int l0 = begin; l0 < end; l0 += kSelThreads) {
+    for (int g = 0; g < p.G; ++g) {
+      const float M = s_M[g], iS = s_iS[g];
+      for (int i = tid; i < kSelThreads + 2 * HALO; i += kSelThreads) {
+        int l = l0 - HALO + i;
+        s_p[g][i] = (l >= 0 && l < L) ? expf(zb[(size_t)g * p.z_stride + l] - M) * iS : 0.f;
+      }
+    }
+    __syncthreads();
+    const int l = l0 + tid;
+    if (l < end) {
+      float agg = 0.f;
+      for (int g = 0; g < p.G; ++g) {
+        const float *row = &s_p[g][HALO + tid];
+        float v;
+        if (p.pool_mode == S4R_POOL_MAX) {
+          v = row[0];
+          for (int j = 1; j <= half; ++j) v = fmaxf(v, fmaxf(row[-j], row[j]));
+        } else {
+          v = row[-half];
+          for (int j = -half + 1; j <= half; ++j) v += row[j];
+          v *= inv_kappa;
+        }
+        agg = (p.group_mode == S4R_GROUP_MEAN) ? agg + v : fmaxf(agg, v);
+      }
+      if (p.group_mode == S4R_GROUP_MEAN) agg *= inv_G;
+      score[l] = agg;
+      if (l < n_cand) atomicAdd(&s_hist[__float_as_uint(agg) >> 21], 1u);
+    }
+    __syncthreads();
+  }
+
+  // ---- radix select of the k_eff-th largest candidate score
+  const int c_end = min(end, n_cand);
+  unsigned k_rem = (unsigned)k_eff, above;
+  const unsigned bin1 = find_bin(cluster, s_hist, s_warp, s_bc, 2048, k_rem, &above);
+  k_rem -= above;
+  for (int i = tid; i < 2048; i += kSelThreads) s_hist[i] = 0;
+  __syncthreads();
+  for (int l = begin + tid; l < c_end; l += kSelThreads) {
+    unsigned v = __float_as_uint(score[l]);
+    if ((v >> 21) == bin1) atomicAdd(&s_hist[(v >> 10) & 0x7ffu], 1u);
+  }
+  const unsigned bin2 = find_bin(cluster, s_hist, s_warp, s_bc, 2048, k_rem, &above);
+  k_rem -= above;
+  const unsigned pre2 = (bin1 << 11) | bin2;
+  for (int i = tid; i < 2048; i += kSelThreads) s_hist[i] = 0;
+  __syncthreads();
+  for (int l = begin + tid; l < c_end; l += kSelThreads) {
+    unsigned v = __float_as_uint(score[l]);
+    if ((v >> 10) == pre2) atomicAdd(&s_hist[v & 0x3ffu], 1u);
+  }
+  const unsigned bin3 = find_bin(cluster, s_hist, s_warp, s_bc, 1024, k_rem, &above);
+  k_rem -= above;  // how many candidates equal to the threshold are taken (lowest indices first)
+  const unsigned tau = (pre2 << 10) | bin3;
+
+  // ---- per-CTA counts, exchanged through distributed shared memory
+  if (tid < 2) s_cnt[tid] = 0;
+  __syncthreads();
+  {
+    unsigned ngt = 0, neq = 0;
+    for (int l = begin + tid; l < c_end; l += kSelThreads) {
+      unsigned v = __float_as_uint(score[l]);
+      ngt += v > tau;
+      neq += v == tau;
+    }
+    ngt = __reduce_add_sync(0xffffffffu, ngt);
+    neq = __reduce_add_sync(0xffffffffu, neq);
+    if (lane == 0) {
+      atomicAdd(&s_cnt[0], ngt);
+      atomicAdd(&s_cnt[1], neq);
+    }
+  }
+  cluster.sync();
+  unsigned gt_before = 0, eq_before = 0;
+  for (int rk = 0; rk < rank; ++rk) {
+    const unsigned *c = cluster.map_shared_rank(s_cnt, rk);
+    gt_before += c[0];
+    eq_before += c[1];
+  }
+  unsigned out_pos = gt_before + min(eq_before, k_rem);
+  unsigned eq_seen = eq_before;
+
+  // ---- ordered compaction of the winners
+  for (int l0 = begin; l0 < c_end; l0 += kSelThreads) {
+    const int l = l0 + tid;
+    unsigned v = (l < c_end) ? __float_as_uint(score[l]) : 0u;
+    const bool in = l < c_end;
+    const unsigned is_eq = in && v == tau;
+    unsigned tot_eq, tot_take;
+    unsigned eq_rank = eq_seen + block_excl_scan(is_eq, s_warp, &tot_eq);
+    const unsigned take = in && (v > tau || (is_eq && eq_rank < k_rem));
+    unsigned pos = out_pos + block_excl_scan(take, s_warp, &tot_take);
+    if (take) out_idx[pos] = l;
+    out_pos += tot_take;
+    eq_seen += tot_eq;
+  }
+  cluster.sync();  // no CTA leaves while a peer may still read its shared memory
+}
+
+cudaError_t launch_select(const StepArgs &a) {
+  SelParams p;
+  p.Z = (const float *)(a.ws + a.plan.off_z);
+  p.part = (const float2 *)(a.ws + a.plan.off_part);
+  p.coef_len = a.coef_len;
+  p.score = (float *)(a.ws + a.plan.off_score);
+  p.sel_idx = a.sel_idx;
+  p.sel_count = a.sel_count;
+  p.G = a.ly.G;
+  p.n_chunks = a.plan.n_scan_chunks;
+  p.window = a.window;
+  p.top_k = a.top_k;
+  p.kappa = a.kappa;
+  p.pool_mode = a.pool_mode;
+  p.group_mode = a.group_mode;
+  p.max_len = a.plan.max_len;
+  p.z_stride = a.plan.z_stride;
+  p.dev_status = a.dev_status;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.plan.cluster, a.ly.B);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = a.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = a.plan.cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, k_select, p);
+  if (e != cudaSuccess) return e;
+  S4R_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+// ======================================================================================================
+// Sparse reconstruction + attention (Eq. 16-18), generic version.  grid (tiles, h_kv, B), block d_h threads.
+// Thread i owns channel i of the KV head: it reconstructs K^[t][i] and V^[t][i] for the tile's rows, so the
+// reconstructed rows exist only in registers / shared memory.  Each CTA writes flash-style partials
+// (max, sum, unnormalised output) per query head; k_merge joins tiles and sinks.
+// ======================================================================================================
+struct AttParams {
+  const void *q, *sink_k, *sink_v, *coef_k, *coef_v, *basis_k, *basis_v;
+  const int32_t *coef_len, *sel_idx, *sel_count;
+  float *part_o;   // [B][Hq][tiles][dh]
+  float2 *part_ms; // [B][Hq][tiles]
+  void *out;
+  int out_dtype;
+  int Hq, Hkv, G, dh, D, rk, rv, s, n_tiles, sel_stride, att_tok;
+  int64_t cap, max_len;
+  float theta;
+  int32_t *dev_status;
+};
+
+// rotated and pre-scaled query channel i of head h (RoPE at the query position, times 1/sqrt(d_h))
+template <typename T>
+__device__ inline float rotated_query(const T *q, int b, int h, int i, int Hq, int dh, float theta, int q_pos,
+                                      double inv_freq) {
+  const T *qp = q + ((size_t)b * Hq + h) * dh;
+  float v = Store<T>::ld(qp + i);
+  if (theta > 0.f) {
+    const int half = dh >> 1;
+    float o = Store<T>::ld(qp + (i < half ? i + half : i - half));
+    float sn, cs;
+    rope_sincos(q_pos, inv_freq, sn, cs);
+    v = (i < half) ? v * cs - o * sn : v * cs + o * sn;
+  }
+  return v * rsqrtf((float)dh);
+}
+
+template <typename T>
+__device__ inline void load_rows_f32(float *dst, const T *coef_b, const int *rows, int nt, int r) {
+  constexpr int V = Store<T>::kVec;
+  const int nvec = r / V;
+  for (int i = threadIdx.x; i < kAttTok * nvec; i += blockDim.x) {
+    int t = i / nvec, c = i - t * nvec;
+    float v[V];
+    if (t < nt) {
+      Store<T>::ld_vec(coef_b + (size_t)rows[t] * r + c * V, v);
+    } else {
+#pragma unroll
+      for (int e = 0; e < V; ++e) v[e] = 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < V; ++e) dst[t * r + c * V + e] = v[e];
+  }
+}
+
+template <typename T>
+__device__ inline void reconstruct_channel(float (&acc)[kAttTok], const float *Cs, const T *brow, int r) {
+  constexpr int V = Store<T>::kVec;
+#pragma unroll
+  for (int t = 0; t < kAttTok; ++t) acc[t] = 0.f;
+  for (int j = 0; j < r; j += V) {
+    float bv[V];
+    Store<T>::ld_vec(brow + j, bv);
+#pragma unroll
+    for (int t = 0; t < kAttTok; ++t) {
+      const float4 *cp = reinterpret_cast<const float4 *>(Cs + t * r + j);
+#pragma unroll
+      for (int e4 = 0; e4 < V / 4; ++e4) {
+        float4 c = cp[e4];
+        acc[t] = fmaf(bv[4 * e4 + 0], c.x, acc[t]);
+        acc[t] = fmaf(bv[4 * e4 + 1], c.y, acc[t]);
+        acc[t] = fmaf(bv[4 * e4 + 2], c.z, acc[t]);
+        acc[t] = fmaf(bv[4 * e4 + 3], c.w, acc[t]);
+      }
+    }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_attend(AttParams p) {
+  extern __shared__ __align__(16) float smem[];
+  const int dh = p.dh, G = p.G;
+  const int rmax = max(p.rk, p.rv);
+  float *Cs = smem;                         // [kAttTok][rmax]
+  float *Ks = Cs + kAttTok * rmax;          // [kAttTok][dh + 1]
+  float *qs = Ks + kAttTok * (dh + 1);      // [G][dh + 1]
+  float *lg = qs + kMaxGroup * (dh + 1);    // [kAttTok][G]  logits, then probabilities
+  int *rows = reinterpret_cast<int *>(lg + kAttTok * kMaxGroup);  // [kAttTok]
+  const int tile = blockIdx.x, kv = blockIdx.y, b = blockIdx.z, i = threadIdx.x;
+  const int count = min(p.sel_count[b], p.sel_stride);
+  const int t0 = tile * kAttTok;
+  if (t0 >= count) return;
+  const int nt = min(kAttTok, count - t0);
+  const int L = clamp_len(p.coef_len, b, p.max_len, nullptr);
+  if (i < kAttTok) {
+    int rix = (i < nt) ? p.sel_idx[(size_t)b * p.sel_stride + t0 + i] : 0;
+    rows[i] = min(max(rix, 0), max(L - 1, 0));
+  }
+  const int half = dh >> 1;
+  const double inv_freq = p.theta > 0.f ? rope_inv_freq(i % half, dh, p.theta) : 0.0;
+  for (int g = 0; g < G; ++g)
+    qs[g * (dh + 1) + i] = rotated_query((const T *)p.q, b, kv * G + g, i, p.Hq, dh, p.theta, p.s + L - 1, inv_freq);
+  __syncthreads();
+
+  // ---- K^ = C^K[rows] (B^K)^T for this KV head (Eq. 16)
+  float acc[kAttTok];
+  load_rows_f32(Cs, (const T *)p.coef_k + (size_t)b * p.cap * p.rk, rows, nt, p.rk);
+  __syncthreads();
+  reconstruct_channel(acc, Cs, (const T *)p.basis_k + ((size_t)b * p.D + (size_t)kv * dh + i) * p.rk, p.rk);
+#pragma unroll
+  for (int t = 0; t < kAttTok; ++t) Ks[t * (dh + 1) + i] = acc[t];
+  __syncthreads();
+  if (p.theta > 0.f) {  // RoPE at the original positions s + row
+    const int partner = i < half ? i + half : i - half;
+#pragma unroll 4
+    for (int t = 0; t < kAttTok; ++t) {
+      float sn, cs;
+      rope_sincos(p.s + rows[t], inv_freq, sn, cs);
+      float o = Ks[t * (dh + 1) + partner];
+      acc[t] = (i < half) ? acc[t] * cs - o * sn : acc[t] * cs + o * sn;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < kAttTok; ++t) Ks[t * (dh + 1) + i] = acc[t];
+    __syncthreads();
+  }
+  // ---- logits of Eq. 18 for the G heads of this KV head
+  for (int pr = i; pr < kAttTok * G; pr += dh) {
+    const int t = pr / G, g = pr - t * G;
+    const float *kr = Ks + t * (dh + 1), *qr = qs + g * (dh + 1);
+    float d = 0.f;
+    for (int c = 0; c < dh; ++c) d = fmaf(qr[c], kr[c], d);
+    lg[t * kMaxGroup + g] = (t < nt) ? d : -INFINITY;
+  }
+  __syncthreads();
+  {
+    const int warp = i >> 5, lane = i & 31, nwarp = dh >> 5;
+    for (int g = warp; g < G; g += nwarp) {
+      float v = lg[lane * kMaxGroup + g];
+      float m = warp_max(v);
+      float e = (v == -INFINITY) ? 0.f : expf(v - m);
+      float s = warp_sum(e);
+      lg[lane * kMaxGroup + g] = e;
+      if (lane == 0)
+        p.part_ms[((size_t)b * p.Hq + kv * G + g) * p.n_tiles + tile] = make_float2(m, s);
+    }
+  }
+  __syncthreads();
+  // ---- V^ = C^V[rows] (B^V)^T and the weighted sum
+  load_rows_f32(Cs, (const T *)p.coef_v + (size_t)b * p.cap * p.rv, rows, nt, p.rv);
+  __syncthreads();
+  reconstruct_channel(acc, Cs, (const T *)p.basis_v + ((size_t)b * p.D + (size_t)kv * dh + i) * p.rv, p.rv);
+  for (int g = 0; g < G; ++g) {
+    float o = 0.f;
+#pragma unroll
+    for (int t = 0; t < kAttTok; ++t) o = fmaf(lg[t * kMaxGroup + g], acc[t], o);
+    p.part_o[(((size_t)b * p.Hq + kv * G + g) * p.n_tiles + tile) * dh + i] = o;
+  }
+}
+
+static AttParams make_att_params(const StepArgs &a) {
+  AttParams p;
+  const Layer &ly = a.ly;
+  p.q = a.q; p.sink_k = a.sink_k; p.sink_v = a.sink_v; p.coef_k = a.coef_k; p.coef_v = a.coef_v;
+  p.basis_k = a.basis_k; p.basis_v = a.basis_v; p.coef_len = a.coef_len; p.sel_idx = a.sel_idx;
+  p.sel_count = a.sel_count;
+  p.part_o = (float *)(a.ws + a.plan.off_att);
+  p.part_ms = (float2 *)(a.ws + a.plan.off_att_ms);
+  p.out = a.out; p.out_dtype = a.out_dtype;
+  p.Hq = ly.Hq; p.Hkv = ly.Hkv; p.G = ly.G; p.dh = ly.dh; p.D = ly.D; p.rk = ly.rk; p.rv = ly.rv; p.s = ly.s;
+  p.n_tiles = a.plan.n_att_tiles; p.sel_stride = a.window + a.top_k; p.att_tok = a.plan.att_tok;
+  p.cap = ly.cap; p.max_len = a.plan.max_len; p.theta = a.theta; p.dev_status = a.dev_status;
+  return p;
+}
+
+template <typename T>
+static cudaError_t attend_t(const StepArgs &a) {
+  AttParams p = make_att_params(a);
+  if (p.n_tiles == 0) return cudaSuccess;
+  const Layer &ly = a.ly;
+  const int rmax = ly.rk > ly.rv ? ly.rk : ly.rv;
+  size_t smem = sizeof(float) * ((size_t)kAttTok * rmax + (size_t)kAttTok * (ly.dh + 1) +
+                                 (size_t)kMaxGroup * (ly.dh + 1) + (size_t)kAttTok * kMaxGroup) +
+                sizeof(int) * kAttTok;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k_attend<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid(p.n_tiles, ly.Hkv, ly.B);
+  k_attend<T><<<grid, ly.dh, smem, a.stream>>>(p);
+  S4R_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+cudaError_t launch_attend_generic(const StepArgs &a) {
+  return a.ly.dtype == S4R_BF16 ? attend_t<__nv_bfloat16>(a) : attend_t<float>(a);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Merge of the tile partials with the sink tokens (Eq. 17-18).  grid (H_q, B), block d_h threads.
+// Sinks are kept in storage precision and handled in fp32 here.
+// ------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) k_merge(AttParams p) {
+  __shared__ float s_red[8];
+  __shared__ float s_log[64];
+  const int h = blockIdx.x, b = blockIdx.y, i = threadIdx.x, dh = p.dh;
+  const int kv = h / p.G, half = dh >> 1, lane = i & 31, warp = i >> 5, nwarp = dh >> 5;
+  const int L = clamp_len(p.coef_len, b, p.max_len, nullptr);
+  const int count = min(p.sel_count[b], p.sel_stride);
+  const int tiles = (count + p.att_tok - 1) / p.att_tok;
+  const double inv_freq = p.theta > 0.f ? rope_inv_freq(i % half, dh, p.theta) : 0.0;
+  const float qi = rotated_query((const T *)p.q, b, h, i, p.Hq, dh, p.theta, p.s + L - 1, inv_freq);
+  // sink logits
+  for (int j = 0; j < p.s; ++j) {
+    const T *kp = (const T *)p.sink_k + ((size_t)b * p.s + j) * p.D + (size_t)kv * dh;
+    float v = Store<T>::ld(kp + i);
+    if (p.theta > 0.f) {
+      float o = Store<T>::ld(kp + (i < half ? i + half : i - half));
+      float sn, cs;
+      rope_sincos(j, inv_freq, sn, cs);
+      v = (i < half) ? v * cs - o * sn : v * cs + o * sn;
+    }
+    float d = warp_sum(qi * v);
+    if (lane == 0) s_red[warp] = d;
+    __syncthreads();
+    if (i == 0) {
+      float t = 0.f;
+      for (int k = 0; k < nwarp; ++k) t += s_red[k];
+      s_log[j] = t;
+    }
+    __syncthreads();
+  }
+  const float2 *ms = p.part_ms + ((size_t)b * p.Hq + h) * p.n_tiles;
+  const float *po = p.part_o + ((size_t)b * p.Hq + h) * p.n_tiles * dh;
+  float M = -INFINITY;
+  for (int t = 0; t < tiles; ++t) M = fmaxf(M, ms[t].x);
+  for (int j = 0; j < p.s; ++j) M = fmaxf(M, s_log[j]);
+  float den = 0.f, num = 0.f;
+  for (int t = 0; t < tiles; ++t) {
+    float2 v = ms[t];
+    float w = expf(v.x - M);
+    den = fmaf(v.y, w, den);
+    num = fmaf(po[(size_t)t * dh + i], w, num);
+  }
+  for (int j = 0; j < p.s; ++j) {
+    float w = expf(s_log[j] - M);
+    den += w;
+    num = fmaf(Store<T>::ld((const T *)p.sink_v + ((size_t)b * p.s + j) * p.D + (size_t)kv * dh + i), w, num);
+  }
+  const float o = (tiles + p.s > 0 && den > 0.f) ? num / den : 0.f;
+  const size_t oi = ((size_t)b * p.Hq + h) * dh + i;
+  if (p.out_dtype == S4R_F32)
+    ((float *)p.out)[oi] = o;
+  else
+    ((__nv_bfloat16 *)p.out)[oi] = __float2bfloat16_rn(o);
+}
+
+cudaError_t launch_merge(const StepArgs &a) {
+  AttParams p = make_att_params(a);
+  dim3 grid(a.ly.Hq, a.ly.B);
+  if (a.ly.dtype == S4R_BF16)
+    k_merge<__nv_bfloat16><<<grid, a.ly.dh, 0, a.stream>>>(p);
+  else
+    k_merge<float><<<grid, a.ly.dh, 0, a.stream>>>(p);
+  S4R_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+// ======================================================================================================
+// Prefill projection (Eq. 3), generic tiled version: C[t - s][c] = sum_d X[t][d] * Bm[d][c] for rows t >= s;
+// rows t < s are copied to the sink buffer (Sec. 3.1.1).  grid (ceil(r/64), ceil((T-s)/64), B), block 256.
+// ======================================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256) k_compress(const T *__restrict__ X, const T *__restrict__ basis,
+                                                  T *__restrict__ coef, int64_t T_rows, int s, int D, int r,
+                                                  int64_t cap) {
+  __shared__ float As[16][64 + 4];
+  __shared__ float Bs[16][64 + 4];
+  const int b = blockIdx.z;
+  const int64_t n_rows = T_rows - s;
+  const int64_t row0 = (int64_t)blockIdx.y * 64;
+  const int col0 = blockIdx.x * 64;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const T *Xb = X + ((size_t)b * T_rows + s) * D;
+  const T *Bb = basis + (size_t)b * D * r;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  const int a_row = threadIdx.x >> 2, a_k = (threadIdx.x & 3) * 4;
+  const int b_k = threadIdx.x >> 4, b_col = (threadIdx.x & 15) * 4;
+  for (int k0 = 0; k0 < D; k0 += 16) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      int64_t rr = row0 + a_row;
+      As[a_k + e][a_row] = (rr < n_rows) ? Store<T>::ld(Xb + (size_t)rr * D + k0 + a_k + e) : 0.f;
+      int cc = col0 + b_col + e;
+      Bs[b_k][b_col + e] = (cc < r) ? Store<T>::ld(Bb + (size_t)(k0 + b_k) * r + cc) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        av[e] = As[kk][ty * 4 + e];
+        bv[e] = Bs[kk][tx * 4 + e];
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int64_t rr = row0 + ty * 4 + i;
+    if (rr >= n_rows) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int cc = col0 + tx * 4 + j;
+      if (cc < r) Store<T>::st(coef + ((size_t)b * cap + rr) * r + cc, acc[i][j]);
+    }
+  }
+}
+
+template <typename T>
+__global__ void k_copy_sinks(const T *__restrict__ X, T *__restrict__ sink, int64_t T_rows, int s, int D) {
+  const int b = blockIdx.x;
+  for (int i = threadIdx.x; i < s * D; i += blockDim.x) sink[(size_t)b * s * D + i] = X[(size_t)b * T_rows * D + i];
+}
+
+__global__ void k_set_len(int32_t *coef_len, int B, int32_t v) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < B) coef_len[i] = v;
+}
+
+template <typename T>
+static cudaError_t compress_t(const Layer &ly, const void *X, const void *basis, int r, void *sink, void *coef,
+                              int64_t n_tok, cudaStream_t st) {
+  if (ly.s > 0) {
+    k_copy_sinks<T><<<ly.B, 256, 0, st>>>((const T *)X, (T *)sink, n_tok, ly.s, ly.D);
+    S4R_LAUNCH_CHECK();
+  }
+  const int64_t n = n_tok - ly.s;
+  if (n > 0) {
+    dim3 grid((r + 63) / 64, (unsigned)((n + 63) / 64), ly.B);
+    k_compress<T><<<grid, 256, 0, st>>>((const T *)X, (const T *)basis, (T *)coef, n_tok, ly.s, ly.D, r, ly.cap);
+    S4R_LAUNCH_CHECK();
+  }
+  return cudaSuccess;
+}
+cudaError_t launch_compress_generic(const Layer &ly, const void *X, const void *basis, int r, void *sink,
+                                    void *coef, int64_t T, cudaStream_t st) {
+  return ly.dtype == S4R_BF16 ? compress_t<__nv_bfloat16>(ly, X, basis, r, sink, coef, T, st)
+                              : compress_t<float>(ly, X, basis, r, sink, coef, T, st);
+}
+cudaError_t launch_set_len(const Layer &ly, int32_t *coef_len, int64_t T, cudaStream_t st) {
+  k_set_len<<<(ly.B + 127) / 128, 128, 0, st>>>(coef_len, ly.B, (int32_t)(T - ly.s));
+  S4R_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+// ======================================================================================================
+// Cache update (Eq. 5-6): one new coefficient row per sequence for K and V, then coef_len += 1.
+// grid (ceil(rmax/32), B, 2), block 256 = 32 columns x 8 row groups.
+// ======================================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256) k_append(const T *__restrict__ k_t, const T *__restrict__ v_t,
+                                                const T *__restrict__ basis_k, const T *__restrict__ basis_v,
+                                                T *__restrict__ coef_k, T *__restrict__ coef_v,
+                                                const int32_t *__restrict__ coef_len, int D, int rk, int rv,
+                                                int64_t cap, int32_t *dev_status) {
+  extern __shared__ float xs[];  // [D]
+  __shared__ float red[8][32];
+  const int b = blockIdx.y, which = blockIdx.z;
+  const int r = which ? rv : rk;
+  const T *x = (which ? v_t : k_t) + (size_t)b * D;
+  const T *basis = (which ? basis_v : basis_k) + (size_t)b * D * r;
+  T *coef = (which ? coef_v : coef_k) + (size_t)b * cap * r;
+  const int len = coef_len[b];
+  if (len < 0 || len >= cap) {
+    if (dev_status && threadIdx.x == 0 && blockIdx.x == 0 && which == 0) atomicOr(dev_status, S4R_DEV_BOUNDS);
+    return;
+  }
+  const int col = blockIdx.x * 32 + (threadIdx.x & 31), rg = threadIdx.x >> 5;
+  if (blockIdx.x * 32 >= r) return;
+  for (int i = threadIdx.x; i < D; i += 256) xs[i] = Store<T>::ld(x + i);
+  __syncthreads();
+  float acc = 0.f;
+  if (col < r)
+    for (int d = rg; d < D; d += 8) acc = fmaf(xs[d], Store<T>::ld(basis + (size_t)d * r + col), acc);
+  red[rg][threadIdx.x & 31] = acc;
+  __syncthreads();
+  if (rg == 0 && col < r) {
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x & 31];
+    Store<T>::st(coef + (size_t)len * r + col, s);
+  }
+}
+
+__global__ void k_bump_len(int32_t *coef_len, int B, int64_t cap) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < B) {
+    int v = coef_len[i];
+    if (v >= 0 && v < cap) coef_len[i] = v + 1;
+  }
+}
+
+cudaError_t launch_append(const Layer &ly, const void *k_t, const void *v_t, const void *basis_k,
+                          const void *basis_v, void *coef_k, void *coef_v, int32_t *coef_len, int32_t *dev_status,
+                          cudaStream_t st) {
+  const int rmax = ly.rk > ly.rv ? ly.rk : ly.rv;
+  dim3 grid((rmax + 31) / 32, ly.B, 2);
+  size_t smem = (size_t)ly.D * sizeof(float);
+  if (ly.dtype == S4R_BF16)
+    k_append<__nv_bfloat16><<<grid, 256, smem, st>>>(
+        (const __nv_bfloat16 *)k_t, (const __nv_bfloat16 *)v_t, (const __nv_bfloat16 *)basis_k,
+        (const __nv_bfloat16 *)basis_v, (__nv_bfloat16 *)coef_k, (__nv_bfloat16 *)coef_v, coef_len, ly.D, ly.rk, ly.rv,
+        ly.cap, dev_status);
+  else
+    k_append<float><<<grid, 256, smem, st>>>((const float *)k_t, (const float *)v_t, (const float *)basis_k,
+                                             (const float *)basis_v, (float *)coef_k, (float *)coef_v, coef_len, ly.D,
+                                             ly.rk, ly.rv, ly.cap, dev_status);
+  S4R_LAUNCH_CHECK();
+  k_bump_len<<<(ly.B + 127) / 128, 128, 0, st>>>(coef_len, ly.B, ly.cap);
+  S4R_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+}  // namespace s4r

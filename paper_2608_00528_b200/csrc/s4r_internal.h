@@ -1,0 +1,44 @@
+// Internal launch interface between the C ABI (s4r_api.cu) and the kernel files.
+#pragma once
+
+#include "s4r_common.cuh"
+
+namespace s4r {
+
+struct Layer {
+  int B, Hq, Hkv, dh, rk, rv, s, dtype, G, D;
+  int64_t cap;
+};
+
+struct StepArgs {
+  Layer ly;
+  const void *q, *sink_k, *sink_v, *coef_k, *coef_v, *basis_k, *basis_v;
+  const int32_t *coef_len;
+  int window, top_k, kappa, pool_mode, group_mode;
+  float theta;
+  void *out;
+  int out_dtype;
+  int32_t *sel_idx, *sel_count;
+  char *ws;
+  int32_t *dev_status;
+  cudaStream_t stream;
+  DecodePlan plan;
+};
+
+// launch counter of the calling host thread (kernels enqueued by the current API call)
+int &launch_counter();
+
+// generic (any supported geometry, fp32 or bf16 storage, CUDA-core arithmetic in fp32)
+cudaError_t launch_qproj(const StepArgs &a);
+cudaError_t launch_scan_generic(const StepArgs &a);
+cudaError_t launch_select(const StepArgs &a);
+cudaError_t launch_attend_generic(const StepArgs &a);
+cudaError_t launch_merge(const StepArgs &a);
+cudaError_t launch_compress_generic(const Layer &ly, const void *X, const void *basis, int r, void *sink,
+                                    void *coef, int64_t T, cudaStream_t st);
+cudaError_t launch_set_len(const Layer &ly, int32_t *coef_len, int64_t T, cudaStream_t st);
+cudaError_t launch_append(const Layer &ly, const void *k_t, const void *v_t, const void *basis_k,
+                          const void *basis_v, void *coef_k, void *coef_v, int32_t *coef_len,
+                          int32_t *dev_status, cudaStream_t st);
+
+}  // namespace s4r

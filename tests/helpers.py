@@ -1,0 +1,145 @@
+"""Shared machinery of the parity tests: build one seeded problem, run the oracle on it, run the library on it,
+compare by the rules of the benchmark definition.  Only tests (and the smoke check) import this file."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import workloads as W
+from oracle import s4r_oracle as O
+
+TOL = {"f32": 1e-4, "bf16": 1e-2}       # max relative output error (per-head inf-norm relative), from the benchmark
+BAND = 1e-3                              # relative tie band around the k-th score inside which index sets may differ
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu", torch.float64).numpy()
+
+
+def from_np(a: np.ndarray, dtype: torch.dtype, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).to(dtype).to(device)
+
+
+class Problem:
+    """Inputs of one layer for the whole batch: the oracle's fp64 views and the device tensors, same bits."""
+
+    def __init__(self, cfg: W.LayerConfig, layer: int = 0, gen_device="cpu", device="cpu", capacity: int | None = None,
+                 full_rank: bool = False):
+        self.cfg = cfg
+        self.layer = layer
+        st = W.storage_dtype(cfg)
+        self.st = st
+        B, s, D = cfg.batch, cfg.sink_count, cfg.d_kv
+        self.L = cfg.cache_len
+        self.cap = capacity if capacity is not None else self.L
+        self.K, self.V, self.q = [], [], []
+        self.BK, self.BV, self.CK, self.CV = [], [], [], []
+        for b in range(B):
+            k = W.make_kv(cfg, layer, b, "k", device=gen_device)
+            v = W.make_kv(cfg, layer, b, "v", device=gen_device)
+            q = W.make_query(cfg, k, layer, b)
+            rk = D if full_rank else cfg.rank_k
+            rv = D if full_rank else cfg.rank_v
+            bk, _ = O.build_basis(to_np(k[W.sample_rows(cfg, layer, b, "k").to(k.device)]), rk)
+            bv, _ = O.build_basis(to_np(v[W.sample_rows(cfg, layer, b, "v").to(v.device)]), rv)
+            bk = O.round_to_storage(bk, cfg.dtype)
+            bv = O.round_to_storage(bv, cfg.dtype)
+            kn, vn = to_np(k), to_np(v)
+            _, _, ck, cv = O.compress(kn, vn, s, bk, bv, cfg.dtype)
+            self.K.append(k.cpu()); self.V.append(v.cpu()); self.q.append(to_np(q))
+            self.BK.append(bk); self.BV.append(bv); self.CK.append(ck); self.CV.append(cv)
+        self.device = torch.device(device)
+
+    # ---- device tensors (uploaded lazily so that CPU-only tests can use the oracle side alone)
+    def upload(self):
+        cfg, dev, st = self.cfg, self.device, self.st
+        B, s = cfg.batch, cfg.sink_count
+        rk, rv = self.BK[0].shape[1], self.BV[0].shape[1]
+        self.d_K = torch.stack(self.K).to(dev)
+        self.d_V = torch.stack(self.V).to(dev)
+        self.d_q = torch.stack([from_np(q, st, dev) for q in self.q])
+        self.d_BK = torch.stack([from_np(b, st, dev) for b in self.BK])
+        self.d_BV = torch.stack([from_np(b, st, dev) for b in self.BV])
+        self.d_sink_k = self.d_K[:, :s].contiguous()
+        self.d_sink_v = self.d_V[:, :s].contiguous()
+        self.d_CK = torch.zeros(B, self.cap, rk, dtype=st, device=dev)
+        self.d_CV = torch.zeros(B, self.cap, rv, dtype=st, device=dev)
+        for b in range(B):
+            self.d_CK[b, :self.L] = from_np(self.CK[b], st, dev)
+            self.d_CV[b, :self.L] = from_np(self.CV[b], st, dev)
+        self.d_len = torch.full((B,), self.L, dtype=torch.int32, device=dev)
+        return self
+
+    def layer_desc(self):
+        import paper_2608_00528_b200 as s4r
+        cfg = self.cfg
+        return s4r.Layer(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, self.BK[0].shape[1],
+                         self.BV[0].shape[1], cfg.sink_count, s4r.S4R_BF16 if cfg.dtype == "bf16" else s4r.S4R_F32,
+                         self.cap)
+
+    def oracle_step(self, b: int, W_: int | None = None, k: int | None = None, theta: float | None = None,
+                    kappa: int | None = None, pool_mode: str | None = None, group_mode: str | None = None,
+                    L: int | None = None):
+        cfg = self.cfg
+        L = self.L if L is None else L
+        s = cfg.sink_count
+        return O.decode_step(self.q[b], to_np(self.K[b][:s]), to_np(self.V[b][:s]), self.CK[b][:L], self.CV[b][:L],
+                             self.BK[b], self.BV[b], cfg.window if W_ is None else W_, cfg.top_k if k is None else k,
+                             kappa=cfg.pool_kernel if kappa is None else kappa,
+                             pool_mode=cfg.pool_mode if pool_mode is None else pool_mode,
+                             group_mode=cfg.group_mode if group_mode is None else group_mode,
+                             theta=cfg.rope_theta if theta is None else theta)
+
+    def oracle_attention_on(self, b: int, idx, theta: float | None = None, L: int | None = None):
+        cfg = self.cfg
+        L = self.L if L is None else L
+        s = cfg.sink_count
+        return O.sparse_attention(self.q[b], to_np(self.K[b][:s]), to_np(self.V[b][:s]), self.CK[b][:L], self.CV[b][:L],
+                                  self.BK[b], self.BV[b], idx, cfg.rope_theta if theta is None else theta)
+
+
+def run_gpu_step(p: Problem, W_: int | None = None, k: int | None = None, theta: float | None = None,
+                 kappa: int | None = None, pool_mode: str | None = None, group_mode: str | None = None,
+                 out_dtype: torch.dtype | None = None, max_len: int | None = None):
+    import paper_2608_00528_b200 as s4r
+    cfg = p.cfg
+    W_ = cfg.window if W_ is None else W_
+    k = cfg.top_k if k is None else k
+    theta = cfg.rope_theta if theta is None else theta
+    ly = p.layer_desc()
+    max_len = p.cap if max_len is None else max_len
+    ws = s4r.alloc_workspace(ly, max_len, W_, k, p.device)
+    out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=out_dtype or torch.float32, device=p.device)
+    sel_buf = torch.full((cfg.batch * (W_ + k) + 1,), -7, dtype=torch.int32, device=p.device)
+    sel = sel_buf[:cfg.batch * (W_ + k)].view(cfg.batch, W_ + k)
+    cnt = torch.full((cfg.batch,), -7, dtype=torch.int32, device=p.device)
+    status = torch.zeros(1, dtype=torch.int32, device=p.device)
+    pm = {"max": s4r.POOL_MAX, "avg": s4r.POOL_AVG}[cfg.pool_mode if pool_mode is None else pool_mode]
+    gm = {"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode if group_mode is None else group_mode]
+    s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, max_len, W_, k,
+                    out, sel_buf, cnt, ws, pool_kernel=cfg.pool_kernel if kappa is None else kappa, pool_mode=pm,
+                    group_mode=gm, rope_theta=theta, dev_status=status)
+    torch.cuda.synchronize()
+    return out, sel, cnt, int(status.item())
+
+
+def check_step(p: Problem, out, sel, cnt, seqs=None, tol: float | None = None, **step_kw):
+    """Selection parity by the tie-band rule, then output parity against the oracle's attention evaluated on
+    the library's own index set.  Returns the worst output error seen."""
+    cfg = p.cfg
+    tol = TOL[cfg.dtype] if tol is None else tol
+    worst = 0.0
+    oracle_kw = {k_: v for k_, v in step_kw.items() if k_ in ("W_", "k", "theta", "kappa", "pool_mode", "group_mode", "L")}
+    for b in (range(cfg.batch) if seqs is None else seqs):
+        res = p.oracle_step(b, **oracle_kw)
+        n = int(cnt[b].item())
+        got = sel[b, :n].cpu().numpy().astype(np.int64)
+        assert n == res["W_eff"] + res["k_eff"], f"seq {b}: sel_count {n} != {res['W_eff'] + res['k_eff']}"
+        assert np.all(sel[b, n:].cpu().numpy() == -1), f"seq {b}: tail of sel_idx not -1"
+        ok, msg = O.selection_agrees(res["score"], res["idx"], got, res["W_eff"], res["k_eff"], BAND)
+        assert ok, f"seq {b}: selection mismatch: {msg}"
+        ref = p.oracle_attention_on(b, np.sort(got), theta=oracle_kw.get("theta"), L=oracle_kw.get("L"))
+        err = O.output_error(to_np(out[b]), ref)
+        assert err <= tol, f"seq {b}: output error {err:.3e} > {tol:.1e}"
+        worst = max(worst, err)
+    return worst

@@ -1,0 +1,84 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header declares, rejects bad arguments
+before touching a device, and its host helpers match the closed forms of the paper."""
+import ctypes
+import math
+import os
+import re
+
+import pytest
+
+import paper_2608_00528_b200 as s4r
+from oracle import models
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "s4r.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(s4r_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = s4r.load()
+    names = _declared_symbols()
+    assert set(names) == set(s4r.EXPORTS), names
+    for n in names:
+        assert getattr(lib, n) is not None
+    assert s4r.version() >= 100
+    assert s4r.strerror(0) == "ok" and "workspace" in s4r.strerror(-3)
+
+
+def test_workspace_bytes_and_validation_need_no_gpu():
+    ly = s4r.Layer(8, 32, 8, 128, 192, 192, 4, s4r.S4R_BF16, 131068)
+    n = s4r.workspace_bytes(ly, 131068, 128, 2048)
+    assert n > 8 * 4 * 131068 * 4 and n % 256 == 0
+    assert s4r.workspace_bytes(s4r.Layer(8, 30, 8, 128, 192, 192, 4, 1, 10), 10, 1, 1) == 0      # H_q % h_kv != 0
+    assert s4r.workspace_bytes(ly, -1, 128, 2048) == 0
+    lib = s4r.load()
+    c = ly.c()
+    one = ctypes.c_void_p(256)
+    sc = s4r._Score(1, 7, 0, 0)
+    rp = s4r._Rope(0.0, 0)
+    args = [ctypes.byref(c), one, one, one, one, one, one, one, one, 131068, 128, 2048, ctypes.byref(sc),
+            ctypes.byref(rp), one, 0, one, one, one, n, None, None]
+    bad = list(args); bad[1] = None                                  # q == NULL
+    assert lib.s4r_decode_step(*bad) == -1
+    bad = list(args); bad[9] = 131069                                # max_len > capacity
+    assert lib.s4r_decode_step(*bad) == -1
+    bad = list(args); bad[19] = n - 1                                # workspace too small
+    assert lib.s4r_decode_step(*bad) == -3
+    sc2 = s4r._Score(4, 7, 0, 0); bad = list(args); bad[12] = ctypes.byref(sc2)   # W_q > 1 not built
+    assert lib.s4r_decode_step(*bad) == -2
+    sc3 = s4r._Score(1, 6, 0, 0); bad = list(args); bad[12] = ctypes.byref(sc3)   # even pooling kernel
+    assert lib.s4r_decode_step(*bad) == -1
+    odd = s4r.Layer(8, 32, 8, 128, 100, 192, 4, 1, 131068).c()                   # rank not a multiple of 8
+    bad = list(args); bad[0] = ctypes.byref(odd)
+    assert lib.s4r_decode_step(*bad) == -2
+    # compress: norm_stats must be NULL, T >= s
+    cargs = [ctypes.byref(c), one, one, 1000, one, one, None, one, one, one, one, one, None, 0, None, None]
+    bad = list(cargs); bad[6] = one
+    assert lib.s4r_compress(*bad) == -1
+    bad = list(cargs); bad[3] = 3
+    assert lib.s4r_compress(*bad) == -1
+
+
+def test_compute_calls_fail_loudly_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    ly = s4r.Layer(1, 8, 2, 128, 64, 64, 4, s4r.S4R_F32, 16)
+    t = torch.zeros(4)
+    with pytest.raises(RuntimeError):
+        s4r.decode_step(ly, t, t, t, t, t, t, t, t, 16, 4, 4, t, t, t, t)
+
+
+def test_host_helpers_match_closed_forms():
+    for rho, L, W in [(0.2, 131068, 64), (0.2, 100, 64), (0.15, 32764, 32), (0.0, 10, 4)]:
+        assert s4r.top_k_from_ratio(rho, L, W) == models.top_k_from_ratio(rho, L, W)
+    for eta, L, s, Dp, G, Wq in [(0.2, 120000, 4, 1024, 4, 32), (0.3, 32000, 4, 512, 7, 4), (0.4, 8000, 0, 1024, 4, 1)]:
+        r = s4r.rank_for_ratio(eta, L, s, Dp, G, Wq, 1)
+        assert models.memory_ratio(s, L, Dp, r, G, Wq) <= eta < models.memory_ratio(s, L, Dp, r + 1, G, Wq)
+        r8 = s4r.rank_for_ratio(eta, L, s, Dp, G, Wq, 8)
+        assert r8 % 8 == 0 and r - 8 < r8 <= r
+    assert abs(s4r.rank_for_ratio(0.2, 10 ** 9, 4, 1024, 4, 32, 1) - math.floor(0.2 * 1024)) <= 1   # limit r / D'

@@ -1,0 +1,229 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import s4r_oracle as O
+from tests.helpers import Problem, run_gpu_step, check_step, to_np, from_np, TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def _s4r():
+    import paper_2608_00528_b200 as s4r
+    return s4r
+
+
+def _cfg(i, **kw):
+    return W.scaled_config(W.get_config(i), **kw)
+
+
+# ------------------------------------------------------------------ decode step
+
+@pytest.mark.parametrize("theta", [None, 0.0])
+def test_decode_config0_fp32(theta):
+    p = Problem(_cfg(0), device="cuda").upload()
+    out, sel, cnt, status = run_gpu_step(p, theta=theta)
+    assert status == 0
+    err = check_step(p, out, sel, cnt, theta=theta)
+    print(f"cfg0 theta={theta}: max rel err {err:.3e}")
+
+
+@pytest.mark.parametrize("theta", [None, 0.0])
+def test_decode_llama_shape_bf16_8k(theta):
+    # config 1's layer at a context that spans several scan chunks and a ragged tail, batch 2
+    p = Problem(_cfg(1, context=8192 + 333, batch=2), device="cuda").upload()
+    out, sel, cnt, status = run_gpu_step(p, theta=theta)
+    assert status == 0
+    err = check_step(p, out, sel, cnt, theta=theta)
+    print(f"llama 8k theta={theta}: max rel err {err:.3e}")
+
+
+def test_decode_qwen_shape_bf16_8k_group7():
+    p = Problem(_cfg(3, context=8192 + 77, batch=2, top_k=512), device="cuda").upload()
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status == 0
+    check_step(p, out, sel, cnt)
+
+
+def test_decode_config1_full_size():
+    p = Problem(_cfg(1), gen_device="cuda", device="cuda").upload()
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status == 0
+    err = check_step(p, out, sel, cnt)
+    print(f"cfg1: max rel err {err:.3e}")
+    out_b, sel_b, cnt_b, _ = run_gpu_step(p, out_dtype=torch.bfloat16)
+    assert torch.equal(sel_b, sel)                                           # run-to-run determinism of selection
+    assert (out_b.float() - out).abs().max() <= 2.0 ** -8 * out.abs().max() * 1.01
+
+
+@pytest.mark.parametrize("pool_mode,group_mode,kappa", [("avg", "mean", 7), ("max", "max", 7), ("avg", "max", 3),
+                                                        ("max", "mean", 1), ("max", "mean", 31)])
+def test_decode_score_switches(pool_mode, group_mode, kappa):
+    p = Problem(_cfg(0, context=3000), device="cuda").upload()
+    kw = dict(pool_mode=pool_mode, group_mode=group_mode, kappa=kappa)
+    out, sel, cnt, status = run_gpu_step(p, **kw)
+    assert status == 0
+    check_step(p, out, sel, cnt, **kw)
+
+
+@pytest.mark.parametrize("Wn,k", [(64, 0), (0, 100), (5000, 10), (64, 10 ** 6), (0, 0), (1, 1), (2000, 1990)])
+def test_decode_degenerate_budgets(Wn, k):
+    # k = 0, W = 0, W > L, k > candidates (everything selected), nothing but sinks
+    p = Problem(_cfg(0, context=2500), device="cuda").upload()
+    k_arg = min(k, 4000)
+    out, sel, cnt, status = run_gpu_step(p, W_=Wn, k=k_arg)
+    assert status == 0
+    check_step(p, out, sel, cnt, W_=Wn, k=k_arg)
+
+
+def test_full_budget_equals_dense_attention_over_reconstructed_cache():
+    cfg = _cfg(0, context=1500)
+    p = Problem(cfg, device="cuda").upload()
+    out, sel, cnt, _ = run_gpu_step(p, W_=16, k=2000)
+    s = cfg.sink_count
+    K_all = np.concatenate([to_np(p.K[0][:s]), p.CK[0] @ p.BK[0].T])
+    V_all = np.concatenate([to_np(p.V[0][:s]), p.CV[0] @ p.BV[0].T])
+    want = O.dense_attention(p.q[0], K_all, V_all, cfg.rope_theta, q_pos=s + p.L - 1)
+    assert O.output_error(to_np(out[0]), want) <= TOL["f32"]
+    assert int(cnt[0]) == p.L and np.array_equal(np.sort(sel[0, :p.L].cpu().numpy()), np.arange(p.L))
+
+
+def test_decode_without_sinks_and_ragged_lengths():
+    cfg = _cfg(1, context=5000, batch=3, sink_count=0, top_k=300)
+    p = Problem(cfg, device="cuda", capacity=5100).upload()
+    lens = [5000, 1234, 37]
+    p.d_len = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status == 0
+    for b, L in enumerate(lens):
+        check_step(p, out, sel, cnt, seqs=[b], L=L)
+
+
+def test_empty_cache_attends_to_sinks_only():
+    cfg = _cfg(0, context=600)
+    p = Problem(cfg, device="cuda").upload()
+    p.d_len.zero_()
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status == 0 and int(cnt[0]) == 0 and bool((sel == -1).all())
+    s = cfg.sink_count
+    ref = O.sparse_attention(p.q[0], to_np(p.K[0][:s]), to_np(p.V[0][:s]), p.CK[0][:0], p.CV[0][:0], p.BK[0], p.BV[0],
+                             np.empty(0, dtype=np.int64), cfg.rope_theta)
+    assert O.output_error(to_np(out[0]), ref) <= TOL["f32"]
+
+
+def test_length_beyond_max_len_is_flagged_and_clamped():
+    s4r = _s4r()
+    p = Problem(_cfg(0, context=800), device="cuda").upload()
+    p.d_len.fill_(10 ** 6)
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status & s4r.DEV_BOUNDS
+    p.d_len.fill_(p.L)
+    out2, sel2, cnt2, status2 = run_gpu_step(p)
+    assert status2 == 0 and torch.equal(sel, sel2)          # clamped to max_len == the true length here
+
+
+def test_small_rank_head_dim_64_and_asymmetric_ranks():
+    cfg = _cfg(0, context=1200, head_dim=64, n_kv_heads=4, n_q_heads=8, rank_k=8, rank_v=40, top_k=100)
+    p = Problem(cfg, device="cuda").upload()
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status == 0
+    check_step(p, out, sel, cnt)
+
+
+def test_decode_step_host_entry_point():
+    s4r = _s4r()
+    cfg = _cfg(0, context=2000)
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+    n = cfg.window + cfg.top_k
+    q_h = p.d_q.cpu().pin_memory()
+    out_h = torch.empty(1, cfg.n_q_heads, cfg.head_dim).pin_memory()
+    sel_h = torch.empty(1, n, dtype=torch.int32).pin_memory()
+    cnt_h = torch.empty(1, dtype=torch.int32).pin_memory()
+    q_d = torch.empty_like(p.d_q)
+    out_d = torch.empty(1, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel_d = torch.empty(1, n, dtype=torch.int32, device="cuda")
+    cnt_d = torch.empty(1, dtype=torch.int32, device="cuda")
+    s4r.decode_step_host(ly, q_h, q_d, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                         cfg.window, cfg.top_k, out_h, out_d, sel_h, sel_d, cnt_h, cnt_d, ws,
+                         rope_theta=cfg.rope_theta)
+    out, sel, cnt, _ = run_gpu_step(p)
+    assert torch.equal(out_h, out.cpu()) and torch.equal(sel_h, sel.cpu()) and torch.equal(cnt_h, cnt.cpu())
+
+
+# ------------------------------------------------------------------ compress and append
+
+def _check_coefficients(got: torch.Tensor, want: np.ndarray, dtype: str, absdot: np.ndarray):
+    """`absdot` = sum_d |x_d| |b_d| per coefficient: the library accumulates in fp32 (unit roundoff 2^-24 per
+    operation, D' <= 1024 terms), the oracle in fp64, so the two pre-rounding values differ by at most about
+    2^-18 * absdot; after rounding to storage they agree to that plus one storage ulp."""
+    g = to_np(got)
+    acc_err = 2.0 ** -18 * absdot
+    if dtype == "bf16":
+        bad = np.abs(g - want) > O.storage_ulp(want, "bf16") * 1.0001 + acc_err
+        assert not bad.any(), f"{bad.sum()} coefficients differ by more than 1 ulp + accumulation error"
+        assert (g != want).mean() < 0.02
+    else:
+        assert (np.abs(g - want) <= O.storage_ulp(want, "f32") + acc_err).all()
+
+
+def _absdot(x: torch.Tensor, basis: np.ndarray) -> np.ndarray:
+    return np.abs(to_np(x)) @ np.abs(basis)
+
+
+@pytest.mark.parametrize("ci,ctx,B", [(0, 1500, 2), (1, 2000 + 13, 2), (3, 1100, 1)])
+def test_compress_matches_oracle(ci, ctx, B):
+    s4r = _s4r()
+    cfg = _cfg(ci, context=ctx, batch=B)
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    s = cfg.sink_count
+    sk = torch.zeros_like(p.d_sink_k); sv = torch.zeros_like(p.d_sink_v)
+    ck = torch.zeros_like(p.d_CK); cv = torch.zeros_like(p.d_CV)
+    ln = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+    s4r.compress(ly, p.d_K, p.d_V, p.d_BK, p.d_BV, sk, sv, ck, cv, ln, workspace=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(sk, p.d_K[:, :s]) and torch.equal(sv, p.d_V[:, :s])
+    assert ln.tolist() == [ctx - s] * B
+    for b in range(B):
+        _check_coefficients(ck[b, :p.L], p.CK[b], cfg.dtype, _absdot(p.K[b][s:], p.BK[b]))
+        _check_coefficients(cv[b, :p.L], p.CV[b], cfg.dtype, _absdot(p.V[b][s:], p.BV[b]))
+
+
+def test_compress_full_rank_reconstructs_the_input():
+    s4r = _s4r()
+    cfg = _cfg(0, context=700, n_sampled=600)
+    p = Problem(cfg, device="cuda", full_rank=True).upload()
+    ly = p.layer_desc()
+    ck = torch.zeros_like(p.d_CK); cv = torch.zeros_like(p.d_CV)
+    ln = torch.zeros(1, dtype=torch.int32, device="cuda")
+    s4r.compress(ly, p.d_K, p.d_V, p.d_BK, p.d_BV, torch.zeros_like(p.d_sink_k), torch.zeros_like(p.d_sink_v), ck, cv, ln)
+    rec = to_np(ck[0]) @ p.BK[0].T
+    ref = to_np(p.K[0][cfg.sink_count:])
+    assert np.abs(rec - ref).max() <= 1e-4 * np.abs(ref).max()
+
+
+def test_append_matches_oracle_and_respects_capacity():
+    s4r = _s4r()
+    cfg = _cfg(1, context=900, batch=2)
+    p = Problem(cfg, device="cuda", capacity=cfg.cache_len + 2).upload()
+    ly = p.layer_desc()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for step in range(3):
+        kt = torch.stack([W.make_token(cfg, 0, b, "k", step + 1, "cuda") for b in range(2)])
+        vt = torch.stack([W.make_token(cfg, 0, b, "v", step + 1, "cuda") for b in range(2)])
+        s4r.append(ly, kt, vt, p.d_BK, p.d_BV, p.d_CK, p.d_CV, p.d_len, dev_status=status)
+        torch.cuda.synchronize()
+        if step < 2:
+            assert status.item() == 0 and p.d_len.tolist() == [p.L + step + 1] * 2
+            for b in range(2):
+                want = O.project_token(to_np(kt[b]), p.BK[b], "bf16")
+                _check_coefficients(p.d_CK[b, p.L + step][None], want[None], "bf16", _absdot(kt[b][None], p.BK[b]))
+                want = O.project_token(to_np(vt[b]), p.BV[b], "bf16")
+                _check_coefficients(p.d_CV[b, p.L + step][None], want[None], "bf16", _absdot(vt[b][None], p.BV[b]))
+        else:
+            assert status.item() & s4r.DEV_BOUNDS and p.d_len.tolist() == [p.L + 2] * 2
