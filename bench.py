@@ -1,0 +1,368 @@
+"""Benchmark of the S4R decode hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+
+One "step" = one pass of the decode path for one layer over the whole batch: the cache update (s4r_append)
+followed by s4r_decode_step (query projection, latent scoring, relevance, selection, sparse reconstruction,
+attention).  The prefill projection (s4r_compress) builds the cache during set-up and is timed separately
+(`compress` in the JSON line).  Workload: the 128K-context Llama-3.1-8B-shaped layer with batch 8 on which the
+headline metric is quoted (coefficients 0.8 GB, far larger than L2, so nothing is carried between steps).
+With N > 1 every rank runs its own batch of sequences (weak scaling, no collective on the data path).
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import workloads as W  # noqa: E402
+
+METRIC = "decode steps/sec at 128K context (one layer, whole batch)"
+UNIT = "steps/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_cache(cfg, s4r, device, capacity):
+    """Synthetic prompt -> bases (set-up) -> s4r_compress.  Returns the device-resident cache and timings."""
+    st = W.storage_dtype(cfg)
+    B, s, D = cfg.batch, cfg.sink_count, cfg.d_kv
+    ly = s4r.Layer(B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rank_k, cfg.rank_v, s,
+                   s4r.S4R_BF16 if cfg.dtype == "bf16" else s4r.S4R_F32, capacity)
+    K = torch.empty(B, cfg.context, D, dtype=st, device=device)
+    V = torch.empty_like(K)
+    BK = torch.empty(B, D, cfg.rank_k, dtype=st, device=device)
+    BV = torch.empty(B, D, cfg.rank_v, dtype=st, device=device)
+    q = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=st, device=device)
+    rank_off = int(os.environ.get("RANK", "0")) * B          # every rank draws its own sequences
+    for b in range(B):
+        K[b] = W.make_kv(cfg, 0, rank_off + b, "k", device=device)
+        V[b] = W.make_kv(cfg, 0, rank_off + b, "v", device=device)
+        BK[b] = W.make_bench_basis(K[b][W.sample_rows(cfg, 0, rank_off + b, "k").to(device)], cfg.rank_k, st)
+        BV[b] = W.make_bench_basis(V[b][W.sample_rows(cfg, 0, rank_off + b, "v").to(device)], cfg.rank_v, st)
+        q[b] = W.make_query(cfg, K[b], 0, rank_off + b)
+    sink_k = torch.empty(B, s, D, dtype=st, device=device)
+    sink_v = torch.empty_like(sink_k)
+    CK = torch.zeros(B, capacity, cfg.rank_k, dtype=st, device=device)
+    CV = torch.zeros(B, capacity, cfg.rank_v, dtype=st, device=device)
+    ln = torch.zeros(B, dtype=torch.int32, device=device)
+    ws = s4r.alloc_workspace(ly, capacity, cfg.window, cfg.top_k, device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s4r.compress(ly, K, V, BK, BV, sink_k, sink_v, CK, CV, ln, workspace=ws)       # warm-up
+    torch.cuda.synchronize()
+    e0.record()
+    s4r.compress(ly, K, V, BK, BV, sink_k, sink_v, CK, CV, ln, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    compress_ms = e0.elapsed_time(e1)
+    compress_launches = s4r.last_launch_count()
+    del K, V
+    torch.cuda.empty_cache()
+    return dict(ly=ly, BK=BK, BV=BV, q=q, sink_k=sink_k, sink_v=sink_v, CK=CK, CV=CV, len=ln, ws=ws,
+                compress_ms=compress_ms, compress_launches=compress_launches)
+
+
+def cpu_baseline(cfg, repeats=3):
+    """The fp64 oracle, as it stands, on one sequence of the workload, timed on this host's cores."""
+    import numpy as np
+    from oracle import s4r_oracle as O
+    cores = len(os.sched_getaffinity(0))
+    torch.set_num_threads(cores)
+    s = cfg.sink_count
+    k = W.make_kv(cfg, 0, 0, "k", device="cpu")
+    v = W.make_kv(cfg, 0, 0, "v", device="cpu")
+    q = W.make_query(cfg, k, 0, 0).double().numpy()
+    bk, _ = O.build_basis(k[W.sample_rows(cfg, 0, 0, "k")].double().numpy(), cfg.rank_k)
+    bv, _ = O.build_basis(v[W.sample_rows(cfg, 0, 0, "v")].double().numpy(), cfg.rank_v)
+    bk, bv = O.round_to_storage(bk, cfg.dtype), O.round_to_storage(bv, cfg.dtype)
+    kn, vn = k.double().numpy(), v.double().numpy()
+    del k, v
+    t0 = time.perf_counter()
+    sk, sv, ck, cv = O.compress(kn, vn, s, bk, bv, cfg.dtype)
+    t_compress = time.perf_counter() - t0
+    del kn, vn
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.decode_step(q, sk, sv, ck, cv, bk, bv, cfg.window, cfg.top_k, kappa=cfg.pool_kernel,
+                      pool_mode=cfg.pool_mode, group_mode=cfg.group_mode, theta=cfg.rope_theta)
+        times.append(time.perf_counter() - t0)
+    times.sort()
+    t_seq = times[len(times) // 2]
+    return {"value": 1.0 / (t_seq * cfg.batch), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"1 of {cfg.batch} sequences of the workload, median of {repeats} decode steps "
+                      f"({t_seq * 1e3:.0f} ms per sequence-step), scaled to the batch; oracle compress of that "
+                      f"sequence took {t_compress:.1f} s (not in the metric)",
+            "ms_per_sequence_step": t_seq * 1e3}
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    base = cpu_baseline(cfg, repeats=max(1, args.steps))
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / base["value"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "batch": cfg.batch, "context": cfg.context},
+            "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--context", type=int, default=None, help="override the context length (profiling only)")
+    ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = W.get_config(args.config)
+    over = {}
+    if args.context:
+        over["context"] = args.context
+    if args.batch:
+        over["batch"] = args.batch
+    if over:
+        cfg = W.scaled_config(cfg, **over)
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+
+    import paper_2608_00528_b200 as s4r
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    K_steps, Wm = args.steps, max(args.warmup, 3)
+    n_append = 2 * (K_steps + Wm) + 8
+    capacity = cfg.cache_len + n_append
+    c = build_cache(cfg, s4r, device, capacity)
+    ly, B = c["ly"], cfg.batch
+    st = W.storage_dtype(cfg)
+    n_sel = cfg.window + cfg.top_k
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=device)
+    sel = torch.empty(B, n_sel, dtype=torch.int32, device=device)
+    cnt = torch.empty(B, dtype=torch.int32, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    # per-step inputs: one new (k_t, v_t, q) triple per step, cycled from a small pool
+    pool = 4
+    kt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "k", i + 1, device) for b in range(B)]) for i in range(pool)])
+    vt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "v", i + 1, device) for b in range(B)]) for i in range(pool)])
+    qs = torch.stack([c["q"] * (1.0 + 0.01 * i) for i in range(pool)]).to(st)
+    kw = dict(pool_kernel=cfg.pool_kernel, pool_mode={"max": s4r.POOL_MAX, "avg": s4r.POOL_AVG}[cfg.pool_mode],
+              group_mode={"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode], rope_theta=cfg.rope_theta,
+              dev_status=status)
+
+    launches = [0]
+
+    def step(i):
+        j = i % pool
+        s4r.append(ly, kt[j], vt[j], c["BK"], c["BV"], c["CK"], c["CV"], c["len"], dev_status=status)
+        launches[0] += s4r.last_launch_count()
+        s4r.decode_step(ly, qs[j], c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"], capacity,
+                        cfg.window, cfg.top_k, out, sel, cnt, c["ws"], **kw)
+        launches[0] += s4r.last_launch_count()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(Wm):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches[0] = 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for i in range(K_steps):
+        step(Wm + i)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    gpu_launches = launches[0]
+    if dist is not None:
+        t = torch.tensor([ms_total], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / K_steps
+
+    # ---- per-stage device times of the same steps (second pass; events recorded inside the library on the
+    #      launching stream), for the roofline of the dominant kernel
+    s4r.stage_timing(True)
+    stage_sum = {}
+    n_prof = K_steps
+    for i in range(n_prof):
+        c["len"].fill_(cfg.cache_len + Wm + K_steps)      # keep the cache length of the timed region
+        step(i)
+        for k_, v_ in s4r.stage_times().items():
+            stage_sum[k_] = stage_sum.get(k_, 0.0) + v_
+    s4r.stage_timing(False)
+    stage_ms = {k_: v_ / n_prof for k_, v_ in stage_sum.items()}
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the host-buffer entry point: q from pinned host memory, results read back
+    c["len"].fill_(cfg.cache_len)
+    q_h = [qs[j].cpu().pin_memory() for j in range(pool)]
+    kt_h = [kt[j].cpu().pin_memory() for j in range(pool)]
+    vt_h = [vt[j].cpu().pin_memory() for j in range(pool)]
+    out_h = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32).pin_memory()
+    sel_h = torch.empty(B, n_sel, dtype=torch.int32).pin_memory()
+    cnt_h = torch.empty(B, dtype=torch.int32).pin_memory()
+    q_d, kt_d, vt_d = torch.empty_like(qs[0]), torch.empty_like(kt[0]), torch.empty_like(vt[0])
+
+    def step_e2e(i):
+        j = i % pool
+        kt_d.copy_(kt_h[j], non_blocking=True)
+        vt_d.copy_(vt_h[j], non_blocking=True)
+        s4r.append(ly, kt_d, vt_d, c["BK"], c["BV"], c["CK"], c["CV"], c["len"], dev_status=status)
+        s4r.decode_step_host(ly, q_h[j], q_d, c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"],
+                             capacity, cfg.window, cfg.top_k, out_h, out, sel_h, sel, cnt_h, cnt, c["ws"], **kw)
+
+    for i in range(3):
+        step_e2e(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(K_steps):
+        step_e2e(3 + i)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    esz = cfg.elem_bytes
+    h2d = B * (cfg.n_q_heads * cfg.head_dim + 2 * cfg.d_kv) * esz
+    d2h = B * (cfg.n_q_heads * cfg.head_dim * 4 + n_sel * 4 + 4)
+    dev_flags = int(status.item())
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (latent scoring): algorithmic bytes = the key-coefficient cache
+    L_now = cfg.cache_len + Wm + K_steps
+    scan_bytes = B * L_now * cfg.rank_k * esz
+    peak, peak_kind = _peaks()
+    scan_ms = stage_ms.get("latent_scoring", float("nan"))
+    achieved = scan_bytes / (scan_ms * 1e-3) / 1e9
+    m = cfg.window + cfg.top_k
+    step_bytes = B * (L_now * cfg.rank_k + m * (cfg.rank_k + cfg.rank_v) + 2 * cfg.sink_count * cfg.d_kv) * esz
+    line = {
+        "metric": METRIC, "value": world * 1e3 / ms_step, "unit": UNIT, "n_gpus": world, "steps": K_steps,
+        "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "batch_per_gpu": B, "global_batch": B * world, "context": cfg.context,
+                   "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
+                   "rank": cfg.rank_k, "window": cfg.window, "top_k": cfg.top_k, "sinks": cfg.sink_count,
+                   "rope_theta": cfg.rope_theta, "step": "s4r_append + s4r_decode_step",
+                   "l2": "inputs larger than L2 (key coefficients %.0f MB per step)" % (scan_bytes / 1e6),
+                   "parallelism": f"dp{world} (independent sequences, no collective)"},
+        "roofline": {"bound": "hbm", "kernel": "latent_scoring", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                     "bytes_per_launch": scan_bytes, "ms_per_launch": scan_ms},
+        "step_roofline": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_bytes / (ms_step * 1e-3) / 1e9,
+                          "frac_of_8TBs": step_bytes / (ms_step * 1e-3) / 8e12,
+                          "frac_of_measured_copy": step_bytes / (ms_step * 1e-3) / 1e9 / peak},
+        "stage_ms": stage_ms,
+        "compress": {"ms": c["compress_ms"], "tokens_per_s": B * (cfg.context - cfg.sink_count) / (c["compress_ms"] * 1e-3),
+                     "launches": c["compress_launches"]},
+        "e2e": {"value": world * K_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": gpu_launches, "clocks": clocks, "dev_status": dev_flags,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = {k: v for k, v in cpu_baseline(cfg).items() if k != "ms_per_sequence_step"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

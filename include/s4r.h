@@ -13,8 +13,9 @@
  * General rules
  *   - Unless an argument is documented as HOST memory, every data pointer is a
  *     DEVICE pointer owned by the caller.  The library never allocates or
- *     frees device memory, keeps no state between calls and never
- *     synchronises the stream (except s4r_decode_step_host, see there).
+ *     frees device memory, keeps no state between calls (except the opt-in
+ *     stage timing below) and never synchronises the stream (except
+ *     s4r_decode_step_host and s4r_stage_times, see there).
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *     work of a call is enqueued on it, in order.
  *   - Every entry point returns S4R_OK or a negative s4r_status_t.  Misuse
@@ -170,6 +171,17 @@ int32_t s4r_rank_for_ratio(double eta, int64_t L, int32_t sink_count, int32_t d_
                            int32_t query_window, int32_t multiple);
 /* Number of kernel launches the last s4r_decode_step / s4r_compress / s4r_append call on this thread made. */
 int32_t s4r_last_launch_count(void);
+
+/* Opt-in per-stage timing for benchmarks (the only state the library keeps; off by default).
+ * s4r_stage_timing(1) makes every later s4r_decode_step on this host thread record CUDA events on its
+ * stream around its stages; s4r_stage_timing(0) switches it off again.  s4r_stage_times waits for the events
+ * of the last step and writes up to n elapsed times in milliseconds, in stage order: 0 query projection
+ * (Eq. 5), 1 latent scoring (Eq. 8), 2 relevance + selection (Eq. 9-15), 3 sparse reconstruction +
+ * attention over the selected rows (Eq. 16-18), 4 merge with the sinks (Eq. 17-18).  Returns the number of
+ * stages written, or a negative s4r_status_t. */
+#define S4R_N_STAGES 5
+int s4r_stage_timing(int enable);
+int s4r_stage_times(float *ms_out, int n);
 
 const char *s4r_strerror(int status);
 int s4r_version(void);

@@ -20,7 +20,9 @@ GROUP_MEAN, GROUP_MAX = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_compress", "s4r_append", "s4r_decode_step", "s4r_decode_step_host",
-           "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_strerror", "s4r_version")
+           "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
+           "s4r_stage_times", "s4r_strerror", "s4r_version")
+STAGES = ("query_projection", "latent_scoring", "selection", "reconstruct_attend", "merge")
 
 
 class S4RError(RuntimeError):
@@ -85,6 +87,10 @@ def load(build_if_missing: bool = True):
     lib.s4r_rank_for_ratio.argtypes = [ctypes.c_double, i64, i32, i32, i32, i32, i32]
     lib.s4r_last_launch_count.restype = i32
     lib.s4r_last_launch_count.argtypes = []
+    lib.s4r_stage_timing.restype = ctypes.c_int
+    lib.s4r_stage_timing.argtypes = [ctypes.c_int]
+    lib.s4r_stage_times.restype = ctypes.c_int
+    lib.s4r_stage_times.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int]
     lib.s4r_strerror.restype = ctypes.c_char_p
     lib.s4r_strerror.argtypes = [ctypes.c_int]
     lib.s4r_version.restype = ctypes.c_int
@@ -113,6 +119,21 @@ def rank_for_ratio(eta: float, cache_len: int, sink_count: int, d_kv: int, group
 
 def last_launch_count() -> int:
     return int(load().s4r_last_launch_count())
+
+
+def stage_timing(enable: bool) -> None:
+    rc = load().s4r_stage_timing(1 if enable else 0)
+    if rc != 0:
+        raise S4RError(rc, "s4r_stage_timing")
+
+
+def stage_times() -> dict:
+    """Milliseconds per stage of the last decode step on this thread (waits for that step)."""
+    buf = (ctypes.c_float * len(STAGES))()
+    rc = load().s4r_stage_times(buf, len(STAGES))
+    if rc < 0:
+        raise S4RError(rc, "s4r_stage_times")
+    return {STAGES[i]: float(buf[i]) for i in range(rc)}
 
 
 @dataclass

@@ -62,6 +62,22 @@ static int check_arch() {
   return major == 10 ? S4R_OK : S4R_ERR_ARCH;
 }
 
+struct StageTimer {
+  bool enabled = false, created = false, recorded = false;
+  cudaEvent_t ev[S4R_N_STAGES + 1];
+};
+static StageTimer &stage_timer() {
+  static thread_local StageTimer t;
+  return t;
+}
+static inline void stage_mark(int i, cudaStream_t st) {
+  StageTimer &t = stage_timer();
+  if (t.enabled) {
+    cudaEventRecord(t.ev[i], st);
+    if (i == S4R_N_STAGES) t.recorded = true;
+  }
+}
+
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace s4r
@@ -154,11 +170,17 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
   a.pool_mode = sc.pool_mode; a.group_mode = sc.group_mode; a.theta = rope ? rope->theta : 0.f; a.out = out;
   a.out_dtype = out_dtype; a.sel_idx = sel_idx; a.sel_count = sel_count; a.ws = (char *)workspace;
   a.dev_status = dev_status; a.stream = (cudaStream_t)stream;
+  stage_mark(0, a.stream);
   if (launch_qproj(a) != cudaSuccess) return S4R_ERR_CUDA;
+  stage_mark(1, a.stream);
   if (launch_scan_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  stage_mark(2, a.stream);
   if (launch_select(a) != cudaSuccess) return S4R_ERR_CUDA;
+  stage_mark(3, a.stream);
   if (launch_attend_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  stage_mark(4, a.stream);
   if (launch_merge(a) != cudaSuccess) return S4R_ERR_CUDA;
+  stage_mark(5, a.stream);
   return S4R_OK;
 }
 
@@ -214,6 +236,29 @@ int32_t s4r_rank_for_ratio(double eta, int64_t L, int32_t sink_count, int32_t d_
 }
 
 int32_t s4r_last_launch_count(void) { return launch_counter(); }
+
+int s4r_stage_timing(int enable) {
+  StageTimer &t = stage_timer();
+  if (enable && !t.created) {
+    for (int i = 0; i <= S4R_N_STAGES; ++i)
+      if (cudaEventCreate(&t.ev[i]) != cudaSuccess) return S4R_ERR_CUDA;
+    t.created = true;
+  }
+  t.enabled = enable != 0;
+  t.recorded = false;
+  return S4R_OK;
+}
+
+int s4r_stage_times(float *ms_out, int n) {
+  StageTimer &t = stage_timer();
+  if (!ms_out || n < 0) return S4R_ERR_INVALID_ARG;
+  if (!t.created || !t.recorded) return S4R_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(t.ev[S4R_N_STAGES]) != cudaSuccess) return S4R_ERR_CUDA;
+  int m = n < S4R_N_STAGES ? n : S4R_N_STAGES;
+  for (int i = 0; i < m; ++i)
+    if (cudaEventElapsedTime(&ms_out[i], t.ev[i], t.ev[i + 1]) != cudaSuccess) return S4R_ERR_CUDA;
+  return m;
+}
 
 const char *s4r_strerror(int status) {
   switch (status) {

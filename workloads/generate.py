@@ -19,6 +19,7 @@ the generated *bits* to the other side instead of regenerating them.
 """
 from __future__ import annotations
 
+import functools
 import math
 
 import torch
@@ -52,6 +53,7 @@ def _cpu_gen(seed: int) -> torch.Generator:
     return g
 
 
+@functools.lru_cache(maxsize=64)
 def _mixing_matrix(cfg: LayerConfig, layer: int, seq: int, tensor: str) -> torch.Tensor:
     d = cfg.d_kv
     g = _cpu_gen(stream_seed(cfg.seed, layer, seq, "mix_" + tensor))
