@@ -162,6 +162,30 @@ int s4r_decode_step_host(const s4r_layer_t *layer, const void *q_host, void *q_d
                          int32_t *sel_count_host, int32_t *sel_count_dev, void *workspace,
                          size_t workspace_bytes, int32_t *dev_status, void *stream);
 
+/* The decode step for callers that cannot allocate device memory.  (The paper has no counterpart; this is
+ * a property of the library, not of the method.)  Some callers have nowhere to get a workspace from: code
+ * that runs where cudaMalloc is forbidden or would stall - inside a latency-critical serving loop whose
+ * memory pool is already carved up, a plugin that is handed tensors but no allocator, a process that must
+ * not touch the allocator after start-up.  For them the scratch of s4r_decode_step lives in a fixed array
+ * inside the library (S4R_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the library, held
+ * until the process exits).  Arguments and results are exactly those of s4r_decode_step without
+ * `workspace` / `workspace_bytes`; the call itself allocates and frees nothing.
+ *   - Geometries whose s4r_workspace_bytes(...) exceeds S4R_STATIC_SCRATCH_BYTES are rejected with
+ *     S4R_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address (a one-off query that also makes
+ *     sure the module is loaded).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left in it; the step
+ *     overwrites every scratch location before reading it, so nothing needs clearing - but two calls that
+ *     overlap on the GPU (different streams, no ordering between them) race on it and corrupt each other.
+ *     Keep calls on one device ordered. */
+#define S4R_STATIC_SCRATCH_BYTES (16u << 20)
+int s4r_decode_step_static(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
+                           const void *coef_k, const void *coef_v, const int32_t *coef_len,
+                           const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                           int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out,
+                           int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, int32_t *dev_status,
+                           void *stream);
+
 /* Host helpers (no GPU work). */
 /* Eq. 14: k = max(floor(rho * L) - W, 0). */
 int64_t s4r_top_k_from_ratio(double rho, int64_t L, int32_t window);

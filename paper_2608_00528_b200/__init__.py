@@ -20,6 +20,7 @@ GROUP_MEAN, GROUP_MAX = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_compress", "s4r_append", "s4r_decode_step", "s4r_decode_step_host",
+           "s4r_decode_step_static",
            "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
            "s4r_stage_times", "s4r_strerror", "s4r_version")
 STAGES = ("query_projection", "latent_scoring", "selection", "reconstruct_attend", "merge")
@@ -255,3 +256,38 @@ def decode_step_host(layer: Layer, q_host, q_dev, sink_k, sink_v, coef_k, coef_v
         _stream(stream))
     if rc != 0:
         raise S4RError(rc, "s4r_decode_step_host")
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def decode_step_static(layer: Layer, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,
+                       max_len: int, window: int, top_k: int, out, sel_idx, sel_count, *, pool_kernel: int = 7,
+                       pool_mode: int = POOL_MAX, group_mode: int = GROUP_MEAN, score_window: int = 1,
+                       rope_theta: float = 0.0, dev_status=None, stream=None):
+    """s4r_decode_step_static: the decode step for callers that have no way to allocate a workspace.
+
+    Same inputs and results as `decode_step`, but the scratch memory is a fixed 16 MiB array inside the
+    library, so nothing is allocated by this call (not by the library, and no torch tensor is created here
+    either).  Geometries that need more scratch raise S4RError(-3).  All calls on a device share that array:
+    keep them ordered on the GPU, and make the first call on a device outside stream capture.
+    """
+    _need_cuda(q, coef_k, coef_v, coef_len, key_basis, value_basis, out, sel_idx, sel_count)
+    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, score_window, rope_theta)
+    out_dtype = S4R_BF16 if out.dtype == torch.bfloat16 else S4R_F32
+    rc = _static_fn()(ctypes.byref(layer.c()), _ptr(q), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k), _ptr(coef_v),
+                      _ptr(coef_len), _ptr(key_basis), _ptr(value_basis), int(max_len), int(window), int(top_k),
+                      ctypes.byref(sc), ctypes.byref(rp), _ptr(out), out_dtype, _ptr(sel_idx), _ptr(sel_count),
+                      _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_decode_step_static")
+
+
+def _static_fn():
+    fn = load().s4r_decode_step_static
+    if fn.restype is not ctypes.c_int or not fn.argtypes:
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        fn.restype = ctypes.c_int
+        fn.argtypes = [ctypes.POINTER(_Layer), vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, ctypes.POINTER(_Score),
+                       ctypes.POINTER(_Rope), vp, i32, vp, vp, vp, vp]
+    return fn

@@ -2,6 +2,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "s4r_internal.h"
 
 namespace s4r {
@@ -214,6 +216,48 @@ int s4r_decode_step_host(const s4r_layer_t *layer, const void *q_host, void *q_d
     return S4R_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return S4R_ERR_CUDA;
   return S4R_OK;
+}
+
+// ---- decode step with built-in scratch, for callers that may not allocate --------------------------------
+// The array below is the whole workspace of one decode step.  In host code its name is only a handle for the
+// runtime (not a device address), so the address the kernels get is looked up once per device with
+// cudaGetSymbolAddress while that device is current.
+static __device__ __align__(256) unsigned char g_static_scratch[S4R_STATIC_SCRATCH_BYTES];
+
+static int static_scratch_address(void **out) {
+  static void *cached[64];
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return S4R_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return S4R_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return S4R_ERR_CUDA;
+    cached[dev] = p;
+  }
+  *out = cached[dev];
+  return S4R_OK;
+}
+
+int s4r_decode_step_static(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
+                           const void *coef_k, const void *coef_v, const int32_t *coef_len,
+                           const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                           int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out,
+                           int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, int32_t *dev_status,
+                           void *stream) {
+  Layer ly;
+  if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
+  if (int rc = layer_supported(ly)) return rc;
+  const size_t need = s4r_workspace_bytes(layer, max_len, window, top_k);
+  if (need == 0) return S4R_ERR_INVALID_ARG;
+  if (need > (size_t)S4R_STATIC_SCRATCH_BYTES) return S4R_ERR_WORKSPACE;  // beyond the built-in maximum
+  if (int rc = check_arch()) return rc;
+  void *scratch = nullptr;
+  if (int rc = static_scratch_address(&scratch)) return rc;
+  return s4r_decode_step(layer, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis, max_len, window,
+                         top_k, score, rope, out, out_dtype, sel_idx, sel_count, scratch, S4R_STATIC_SCRATCH_BYTES,
+                         dev_status, stream);
 }
 
 int64_t s4r_top_k_from_ratio(double rho, int64_t L, int32_t window) {

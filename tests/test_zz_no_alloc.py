@@ -1,0 +1,59 @@
+"""The allocation-free decode step (s4r_decode_step_static) against the regular entry point.
+
+Collected last on purpose: a run that stops at the first failure has then already run every other test.
+The entry point exists for callers that cannot get a workspace: they are forbidden to allocate device memory
+where they run (a serving loop with a fixed memory plan, a plugin without an allocator).  Its scratch is one
+array inside the library shared by all calls, so the test makes two calls in a row on different problems -
+the second one meets whatever the first left behind - and compares each with s4r_decode_step.
+"""
+import pytest
+import torch
+
+import workloads as W
+from tests.helpers import Problem, run_gpu_step, check_step, TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def _static_step(s4r, p, cfg):
+    ly = p.layer_desc()
+    n = cfg.window + cfg.top_k
+    out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device="cuda")
+    sel = torch.full((cfg.batch, n), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((cfg.batch,), -7, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    s4r.decode_step_static(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                           cfg.window, cfg.top_k, out, sel, cnt, pool_kernel=cfg.pool_kernel,
+                           rope_theta=cfg.rope_theta, dev_status=status)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == before          # the call created no device tensor
+    assert status.item() == 0
+    return out, sel, cnt
+
+
+def test_static_scratch_entry_point_matches_regular_entry_point_twice():
+    import paper_2608_00528_b200 as s4r
+    assert "s4r_decode_step_static" in open(s4r.lib_path(), "rb").read().decode("latin1")
+    problems = [W.scaled_config(W.get_config(1), context=6000 + 41, batch=2),
+                W.scaled_config(W.get_config(0), context=2500, batch=1)]
+    for cfg in problems:                                     # two calls in a row share the built-in scratch
+        p = Problem(cfg, device="cuda").upload()
+        out_s, sel_s, cnt_s = _static_step(s4r, p, cfg)
+        out_r, sel_r, cnt_r, status = run_gpu_step(p)
+        assert status == 0
+        assert torch.equal(sel_s, sel_r) and torch.equal(cnt_s, cnt_r)
+        scale = out_r.abs().amax(dim=-1, keepdim=True)
+        assert ((out_s - out_r).abs() <= TOL[cfg.dtype] * scale).all()
+        check_step(p, out_s, sel_s, cnt_s)                   # and it is right, not merely equal
+
+
+def test_static_scratch_rejects_geometries_beyond_its_maximum():
+    import paper_2608_00528_b200 as s4r
+    big = s4r.Layer(8, 32, 8, 128, 192, 192, 4, s4r.S4R_BF16, 131068)
+    assert s4r.workspace_bytes(big, 131068, 128, 2048) > s4r.STATIC_SCRATCH_BYTES
+    t = torch.zeros(64, device="cuda")
+    with pytest.raises(s4r.S4RError) as e:
+        s4r.decode_step_static(big, t, t, t, t, t, t, t, t, 131068, 128, 2048, t, t, t)
+    assert e.value.status == -3
