@@ -42,9 +42,11 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   while (cl < kMaxCluster && max_len > (int64_t)cl * 8192) cl *= 2;
   p->cluster = cl;
   size_t off = 0;
-  p->off_cq = off;      off = align_up(off + sizeof(float) * ly.B * ly.G * ly.rk, 256);
+  p->n_parts = p->n_scan_chunks;
+  p->parts_cap = p->n_scan_chunks > kMaxParts ? p->n_scan_chunks : kMaxParts;
+  p->off_cq = off;      off = align_up(off + sizeof(float) * ly.B * kQSlices * ly.G * ly.rk, 256);
   p->off_z = off;       off = align_up(off + sizeof(float) * ly.B * ly.G * p->z_stride, 256);
-  p->off_part = off;    off = align_up(off + sizeof(float2) * ly.B * p->n_scan_chunks * kMaxGroup, 256);
+  p->off_part = off;    off = align_up(off + sizeof(float2) * ly.B * p->parts_cap * kMaxGroup, 256);
   p->off_score = off;   off = align_up(off + sizeof(float) * ly.B * p->z_stride, 256);
   p->off_att = off;     off = align_up(off + sizeof(float) * ly.B * ly.Hq * (size_t)p->n_att_tiles * ly.dh, 256);
   p->off_att_ms = off;  off = align_up(off + sizeof(float2) * ly.B * ly.Hq * (size_t)p->n_att_tiles, 256);
@@ -172,10 +174,19 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
   a.pool_mode = sc.pool_mode; a.group_mode = sc.group_mode; a.theta = rope ? rope->theta : 0.f; a.out = out;
   a.out_dtype = out_dtype; a.sel_idx = sel_idx; a.sel_count = sel_count; a.ws = (char *)workspace;
   a.dev_status = dev_status; a.stream = (cudaStream_t)stream;
+  bool fast_scan = scan_fast_supported(ly);
+  if (fast_scan) {
+    const int parts = scan_fast_parts(ly);
+    if (parts < 1 || parts > a.plan.parts_cap) fast_scan = false; else a.plan.n_parts = parts;
+  }
   stage_mark(0, a.stream);
   if (launch_qproj(a) != cudaSuccess) return S4R_ERR_CUDA;
   stage_mark(1, a.stream);
-  if (launch_scan_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (fast_scan) {
+    if (launch_scan_sm100(a) != cudaSuccess) return S4R_ERR_CUDA;
+  } else {
+    if (launch_scan_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  }
   stage_mark(2, a.stream);
   if (launch_select(a) != cudaSuccess) return S4R_ERR_CUDA;
   stage_mark(3, a.stream);

@@ -15,6 +15,8 @@ constexpr int kScanRows = 1024;    // rows of C^K per scan CTA (also the granula
 constexpr int kAttTok = 32;        // selected rows per CTA in the generic reconstruct+attend kernel
 constexpr int kSelThreads = 1024;  // threads per CTA of the selection kernel (one position each per tile)
 constexpr int kMaxCluster = 8;     // portable cluster size
+constexpr int kQSlices = 8;        // D' is split into this many slices by the query projection (partials summed by readers)
+constexpr int kMaxParts = 256;     // upper bound of softmax partials per sequence written by a scan kernel
 
 // ---- storage-type helpers -------------------------------------------------------------------------
 
@@ -96,7 +98,9 @@ __device__ inline void rope_sincos(int pos, double inv_freq, float &sn, float &c
 struct DecodePlan {
   int64_t max_len;      // host-known bound of L
   int64_t z_stride;     // floats per (b, g) row of Z
-  int n_scan_chunks;    // CTAs per sequence in the scan
+  int n_scan_chunks;    // CTAs per sequence in the generic scan (1024 rows each)
+  int n_parts;          // softmax partials per sequence the chosen scan kernel writes (set at dispatch)
+  int parts_cap;        // partials allocated per sequence
   int n_att_tiles;      // row tiles per sequence in the attention kernel
   int cluster;          // CTAs per sequence in the selection kernel
   int att_tok;          // selected rows per attention tile

@@ -32,18 +32,21 @@ __device__ inline int clamp_len(const int32_t *coef_len, int b, int64_t max_len,
 
 // ======================================================================================================
 // Query projection (Eq. 5):  cq[b][g][c] = sum_d Qt[g][d] * B^K[b][d][c],  Qt[g][d] = q[b][(d/dh)*G+g][d%dh]
-// grid (ceil(r/32), B), block 256 = 32 columns x 8 row groups; row groups are summed in a fixed order.
+// grid (ceil(r/32), B, kQSlices): each CTA covers D'/kQSlices rows of the basis and writes a partial
+// cq_part[b][slice][g][c]; readers add the kQSlices partials in slice order (deterministic).
+// block 256 = 32 columns x 8 row groups; row groups are summed in a fixed order.
 // ======================================================================================================
 template <typename T>
 __global__ void __launch_bounds__(256) k_qproj(const T *__restrict__ q, const T *__restrict__ basis,
-                                               float *__restrict__ cq, int D, int r, int G, int dh, int Hq) {
-  extern __shared__ float xs[];  // [G][D]
+                                               float *__restrict__ cq_part, int D, int r, int G, int dh, int Hq) {
+  extern __shared__ float xs[];  // [G][D / kQSlices]
   __shared__ float red[8][kMaxGroup][32];
-  const int b = blockIdx.y;
+  const int b = blockIdx.y, slice = blockIdx.z;
+  const int Ds = D / kQSlices, d0 = slice * Ds;
   const int col = blockIdx.x * 32 + (threadIdx.x & 31);
   const int rg = threadIdx.x >> 5;
-  for (int i = threadIdx.x; i < G * D; i += 256) {
-    int g = i / D, d = i - g * D;
+  for (int i = threadIdx.x; i < G * Ds; i += 256) {
+    int g = i / Ds, d = d0 + (i - g * Ds);
     xs[i] = Store<T>::ld(q + ((size_t)b * Hq + (size_t)(d / dh) * G + g) * dh + (d % dh));
   }
   __syncthreads();
@@ -51,12 +54,12 @@ __global__ void __launch_bounds__(256) k_qproj(const T *__restrict__ q, const T 
 #pragma unroll
   for (int g = 0; g < kMaxGroup; ++g) acc[g] = 0.f;
   if (col < r) {
-    const T *bp = basis + (size_t)b * D * r + col;
-    for (int d = rg; d < D; d += 8) {
+    const T *bp = basis + ((size_t)b * D + d0) * r + col;
+    for (int d = rg; d < Ds; d += 8) {
       float bv = Store<T>::ld(bp + (size_t)d * r);
 #pragma unroll
       for (int g = 0; g < kMaxGroup; ++g)
-        if (g < G) acc[g] = fmaf(xs[g * D + d], bv, acc[g]);
+        if (g < G) acc[g] = fmaf(xs[g * Ds + d], bv, acc[g]);
     }
   }
 #pragma unroll
@@ -67,7 +70,7 @@ __global__ void __launch_bounds__(256) k_qproj(const T *__restrict__ q, const T 
       float s = 0.f;
 #pragma unroll
       for (int k = 0; k < 8; ++k) s += red[k][g][threadIdx.x & 31];
-      cq[((size_t)b * G + g) * r + col] = s;
+      cq_part[(((size_t)b * kQSlices + slice) * G + g) * r + col] = s;
     }
   }
 }
@@ -75,12 +78,8 @@ __global__ void __launch_bounds__(256) k_qproj(const T *__restrict__ q, const T 
 template <typename T>
 static cudaError_t qproj_t(const StepArgs &a) {
   const Layer &ly = a.ly;
-  size_t smem = (size_t)ly.G * ly.D * sizeof(float);
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k_qproj<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-  }
-  dim3 grid((ly.rk + 31) / 32, ly.B);
+  size_t smem = (size_t)ly.G * (ly.D / kQSlices) * sizeof(float);
+  dim3 grid((ly.rk + 31) / 32, ly.B, kQSlices);
   k_qproj<T><<<grid, 256, smem, a.stream>>>((const T *)a.q, (const T *)a.basis_k, (float *)(a.ws + a.plan.off_cq),
                                             ly.D, ly.rk, ly.G, ly.dh, ly.Hq);
   S4R_LAUNCH_CHECK();
@@ -111,7 +110,12 @@ __global__ void __launch_bounds__(256) k_scan(const T *__restrict__ coef_k, cons
     if (threadIdx.x < G) part[((size_t)b * n_chunks + chunk) * kMaxGroup + threadIdx.x] = make_float2(-INFINITY, 0.f);
     return;
   }
-  for (int i = threadIdx.x; i < G * r; i += 256) cqs[i] = cq[(size_t)b * G * r + i];
+  for (int i = threadIdx.x; i < G * r; i += 256) {
+    float t = 0.f;
+#pragma unroll
+    for (int sl = 0; sl < kQSlices; ++sl) t += cq[((size_t)b * kQSlices + sl) * G * r + i];
+    cqs[i] = t;
+  }
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane & 7, slot = lane >> 3;
   const int nvec = r / V;
@@ -297,7 +301,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
   if (k_eff == 0) return;  // uniform over the cluster: nothing to rank
 
   // ---- softmax normalisers of Eq. 9 from the scan's per-chunk partials
-  const int used_chunks = (L + kScanRows - 1) / kScanRows;
+  const int used_chunks = p.n_chunks;  // every partial is defined; empty ones are (-inf, 0)
   if (warp < p.G) {
     const float2 *pp = p.part + (size_t)b * p.n_chunks * kMaxGroup + warp;
     float m = -INFINITY;
@@ -306,7 +310,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
     float s = 0.f;
     for (int c = lane; c < used_chunks; c += 32) {
       float2 v = pp[(size_t)c * kMaxGroup];
-      s += v.y * expf(v.x - m);
+      if (v.y > 0.f) s += v.y * expf(v.x - m);
     }
     s = warp_sum(s);
     if (lane == 0) {
@@ -434,7 +438,7 @@ cudaError_t launch_select(const StepArgs &a) {
   p.sel_idx = a.sel_idx;
   p.sel_count = a.sel_count;
   p.G = a.ly.G;
-  p.n_chunks = a.plan.n_scan_chunks;
+  p.n_chunks = a.plan.n_parts;
   p.window = a.window;
   p.top_k = a.top_k;
   p.kappa = a.kappa;

@@ -32,6 +32,12 @@ int &launch_counter();
 cudaError_t launch_qproj(const StepArgs &a);
 cudaError_t launch_scan_generic(const StepArgs &a);
 cudaError_t launch_select(const StepArgs &a);
+
+// sm_100a specialisations for bf16 storage (TMA + tcgen05)
+bool scan_fast_supported(const Layer &ly);
+int scan_fast_parts(const Layer &ly);  // CTAs (= softmax partials) per sequence; 0 on error
+cudaError_t launch_scan_sm100(const StepArgs &a);
+
 cudaError_t launch_attend_generic(const StepArgs &a);
 cudaError_t launch_merge(const StepArgs &a);
 cudaError_t launch_compress_generic(const Layer &ly, const void *X, const void *basis, int r, void *sink,
