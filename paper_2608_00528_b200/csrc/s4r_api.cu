@@ -36,7 +36,7 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   p->z_stride = (int64_t)align_up((size_t)(max_len > 0 ? max_len : 1), 4);
   p->n_scan_chunks = (int)((max_len + kScanRows - 1) / kScanRows);
   if (p->n_scan_chunks < 1) p->n_scan_chunks = 1;
-  p->att_tok = kAttTok;
+  p->att_tok = att_fast_supported(ly) ? 128 : kAttTok;
   p->n_att_tiles = (window + top_k + p->att_tok - 1) / p->att_tok;
   int cl = 1;
   while (cl < kMaxCluster && max_len > (int64_t)cl * 8192) cl *= 2;
@@ -190,7 +190,11 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
   stage_mark(2, a.stream);
   if (launch_select(a) != cudaSuccess) return S4R_ERR_CUDA;
   stage_mark(3, a.stream);
-  if (launch_attend_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (att_fast_supported(ly)) {
+    if (launch_attend_sm100(a) != cudaSuccess) return S4R_ERR_CUDA;
+  } else {
+    if (launch_attend_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+  }
   stage_mark(4, a.stream);
   if (launch_merge(a) != cudaSuccess) return S4R_ERR_CUDA;
   stage_mark(5, a.stream);

@@ -1,0 +1,401 @@
+// Sparse reconstruction + attention (Eq. 16-18) for bf16 caches on sm_100a, fused so that the reconstructed
+// keys and values never leave the chip.
+//
+// One CTA owns a tile of 128 selected rows of one sequence and a range of KV heads.  It gathers the rows'
+// key and value coefficients once into 128-byte-swizzled shared memory, then for every KV head
+//   K^[tokens x d_h]   = C^K[rows] (B^K slice)^T      (tcgen05.mma, A = gathered rows, B = basis slice)
+//   V^^T[d_h x tokens] = (B^V slice) C^V[rows]^T      (tcgen05.mma, A = basis slice, B = gathered rows)
+// with the basis slices streamed through a TMA ring in 64-column blocks and the fp32 results held in tensor
+// memory (2 x 2 accumulators of 128 columns, so the tensor pipe runs one head ahead of the epilogue).
+// The epilogue warps read K^ row-per-thread, apply RoPE from a per-tile sin/cos table, form the logits of
+// the G query heads in fp32, take the tile softmax, then read V^^T channel-per-thread and accumulate
+// P.V^ - both contractions are thread-local, so no reconstructed value is ever written anywhere.
+// Per (head, tile) the CTA emits flash-style partials (max, sum, unnormalised output); k_merge joins them
+// with the sinks.  Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-9 = epilogue.
+#include "s4r_internal.h"
+#include "s4r_sm100.cuh"
+
+namespace s4r {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kTok = 128;          // selected rows per tile
+constexpr int kDh = 128;           // head dimension of the fast path
+constexpr int kRing = 3;           // basis blocks in flight
+constexpr int kBlkBytes = 128 * 128;  // one [128 x 64] bf16 block
+constexpr int kEpiThreads = 256;
+constexpr int kThreads = 64 + kEpiThreads;
+
+struct AttFastParams {
+  const __nv_bfloat16 *q, *coef_k, *coef_v;
+  const int32_t *coef_len, *sel_idx, *sel_count;
+  float *part_o;
+  float2 *part_ms;
+  int Hq, Hkv, G, D, rk, rv, s, n_tiles, sel_stride, nkv;
+  int64_t cap, max_len;
+  float theta;
+  int32_t *dev_status;
+};
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_constant__ CUtensorMap tmap_bk,
+                                                              const __grid_constant__ CUtensorMap tmap_bv,
+                                                              AttFastParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int kbk = p.rk >> 6, kbv = p.rv >> 6;
+  uint8_t *ck = smem;                                   // [kbk][128 tokens][128 B]
+  uint8_t *cv = ck + (size_t)kbk * kBlkBytes;           // [kbv][128 tokens][128 B]
+  uint8_t *ring = cv + (size_t)kbv * kBlkBytes;         // [kRing][128 d][128 B]
+  float2 *sc = reinterpret_cast<float2 *>(ring + (size_t)kRing * kBlkBytes);   // [64 pairs][128 tokens] (sin, cos)
+  float *qs = reinterpret_cast<float *>(sc + 64 * kTok);                       // [128 cols][8]
+  float *ps = qs + kDh * kMaxGroup;                                            // [128 tokens][8] probabilities
+  float *xch = ps + kTok * kMaxGroup;                                          // [2 halves][8][128] exchange
+  uint64_t *bars = reinterpret_cast<uint64_t *>(xch + 2 * kMaxGroup * 128);
+  uint64_t *full = bars, *empty = bars + kRing;
+  uint64_t *k_full = bars + 2 * kRing, *k_empty = k_full + 2, *v_full = k_empty + 2, *v_empty = v_full + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(v_empty + 2);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  int *rows = reinterpret_cast<int *>(tmem_slot + 2);                          // [128]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile = blockIdx.x, kv0 = blockIdx.y * p.nkv, b = blockIdx.z;
+  const int count = min(p.sel_count[b], p.sel_stride);
+  const int t0 = tile * kTok;
+  if (t0 >= count) return;  // uniform over the CTA
+  const int nt = min(kTok, count - t0);
+  int L = p.coef_len[b];
+  L = L < 0 ? 0 : (L > p.max_len ? (int)p.max_len : L);
+
+  if (tid == 0) {
+    for (int i = 0; i < kRing; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1);
+      mbar_init(&v_full[i], 1);
+      mbar_init(&k_empty[i], kEpiThreads);
+      mbar_init(&v_empty[i], kEpiThreads);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&tmap_bk);
+    prefetch_tmap(&tmap_bv);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, 512);
+  if (tid < kTok) {
+    int rix = (tid < nt) ? p.sel_idx[(size_t)b * p.sel_stride + t0 + tid] : -1;
+    rows[tid] = rix < 0 ? -1 : min(rix, max(L - 1, 0));
+  }
+  __syncthreads();
+
+  // ---- gather the selected coefficient rows into swizzled K-major tiles (zero rows past the tile's end)
+  {
+    const int cpr_k = p.rk >> 3, cpr_v = p.rv >> 3;  // 16-byte chunks per row
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    const __nv_bfloat16 *ckb = p.coef_k + (size_t)b * p.cap * p.rk;
+    const __nv_bfloat16 *cvb = p.coef_v + (size_t)b * p.cap * p.rv;
+    for (int i = tid; i < kTok * cpr_k; i += kThreads) {
+      const int t = i / cpr_k, c = i - t * cpr_k, rix = rows[t];
+      const uint4 v = rix >= 0 ? __ldg(reinterpret_cast<const uint4 *>(ckb + (size_t)rix * p.rk) + c) : zero;
+      *reinterpret_cast<uint4 *>(ck + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8)) = v;
+    }
+    for (int i = tid; i < kTok * cpr_v; i += kThreads) {
+      const int t = i / cpr_v, c = i - t * cpr_v, rix = rows[t];
+      const uint4 v = rix >= 0 ? __ldg(reinterpret_cast<const uint4 *>(cvb + (size_t)rix * p.rv) + c) : zero;
+      *reinterpret_cast<uint4 *>(cv + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8)) = v;
+    }
+    // sin / cos of every (pair, token) of the tile at the token's original position s + row
+    if (p.theta > 0.f) {
+      for (int i = tid; i < 64 * kTok; i += kThreads) {
+        const int pair = i >> 7, t = i & (kTok - 1);
+        float sn = 0.f, cs = 1.f;
+        if (rows[t] >= 0) rope_sincos(p.s + rows[t], rope_inv_freq(pair, kDh, p.theta), sn, cs);
+        sc[i] = make_float2(sn, cs);
+      }
+    }
+  }
+  fence_proxy_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int blocks_per_kv = kbk + kbv;
+
+  if (warp == 0) {
+    // ---------------- TMA producer: basis slices, 64-column blocks, K blocks then V blocks per head ----------------
+    if (lane == 0) {
+      int it = 0, issued = 0;
+      bool ok = true;
+      for (int h = 0; h < p.nkv && ok; ++h) {
+        const int y = b * p.D + (kv0 + h) * kDh;
+        for (int blk = 0; blk < blocks_per_kv; ++blk, ++it) {
+          const int slot = it % kRing;
+          const uint32_t ph = (uint32_t)(it / kRing) & 1u;
+          if (!mbar_wait(&empty[slot], ph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(&full[slot], kBlkBytes);
+          if (blk < kbk)
+            tma_load_2d(ring + (size_t)slot * kBlkBytes, &tmap_bk, blk * 64, y, &full[slot]);
+          else
+            tma_load_2d(ring + (size_t)slot * kBlkBytes, &tmap_bv, (blk - kbk) * 64, y, &full[slot]);
+          issued = it + 1;
+        }
+      }
+      if (*abort_flag) {
+        for (int i = max(0, issued - kRing); i < issued; ++i) {
+          const unsigned long long t_0 = global_ns();
+          while (!mbar_try_wait(&full[i % kRing], (uint32_t)(i / kRing) & 1u))
+            if (global_ns() - t_0 > kWaitLimitNs) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(128, 128);
+      const uint64_t ck_desc = umma_desc_sw128(smem_u32(ck)), cv_desc = umma_desc_sw128(smem_u32(cv));
+      int it = 0;
+      bool ok = true;
+      for (int h = 0; h < p.nkv && ok; ++h) {
+        const int buf = h & 1;
+        const uint32_t aph = (uint32_t)(h >> 1) & 1u;
+        // K^ -> columns [buf*128, +128)
+        if (!mbar_wait(&k_empty[buf], aph ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        for (int blk = 0; blk < kbk && ok; ++blk, ++it) {
+          const int slot = it % kRing;
+          if (!mbar_wait(&full[slot], (uint32_t)(it / kRing) & 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t bs_desc = umma_desc_sw128(smem_u32(ring + (size_t)slot * kBlkBytes));
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            umma_bf16(tmem_base + (uint32_t)buf * 128, ck_desc + (uint64_t)((blk * kBlkBytes + k4 * 32) >> 4),
+                      bs_desc + (uint64_t)((k4 * 32) >> 4), idesc, (blk | k4) != 0);
+          umma_commit(&empty[slot]);
+        }
+        if (!ok) break;
+        umma_commit(&k_full[buf]);
+        // V^^T -> columns [256 + buf*128, +128)
+        if (!mbar_wait(&v_empty[buf], aph ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        for (int blk = 0; blk < kbv && ok; ++blk, ++it) {
+          const int slot = it % kRing;
+          if (!mbar_wait(&full[slot], (uint32_t)(it / kRing) & 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t bs_desc = umma_desc_sw128(smem_u32(ring + (size_t)slot * kBlkBytes));
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            umma_bf16(tmem_base + 256u + (uint32_t)buf * 128, bs_desc + (uint64_t)((k4 * 32) >> 4),
+                      cv_desc + (uint64_t)((blk * kBlkBytes + k4 * 32) >> 4), idesc, (blk | k4) != 0);
+          umma_commit(&empty[slot]);
+        }
+        if (!ok) break;
+        umma_commit(&v_full[buf]);
+      }
+    }
+  } else {
+    // ---------------- epilogue: 8 warps; warps e and e+4 share a TMEM lane quadrant and split the columns ----------------
+    const int e = warp - 2, et = tid - 64;   // epilogue warp / thread index
+    const int quad = warp & 3, half = e >> 2;
+    const int lane_row = quad * 32 + lane;  // token (K^) or channel (V^^T) owned by this thread
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const int G = p.G;
+    // RoPE of the query: this thread prepares column qc of q' for the heads g = qg0, qg0+2, ...
+    const int qc = et & 127, qg0 = et >> 7;
+    float q_sn = 0.f, q_cs = 1.f;
+    if (p.theta > 0.f) rope_sincos(p.s + L - 1, rope_inv_freq(qc & 63, kDh, p.theta), q_sn, q_cs);
+    const float q_scale = rsqrtf((float)kDh);
+    // `ok` stays warp-uniform; after a failed wait the loop keeps its shape (every epi_sync is still reached)
+    // but touches tensor memory no more
+    bool ok = true;
+    for (int h = 0; h < p.nkv; ++h) {
+      const int kv = kv0 + h, buf = h & 1;
+      const uint32_t aph = (uint32_t)(h >> 1) & 1u;
+      // q' = RoPE(q) / sqrt(d_h) for the G heads of this KV head, laid out [col][g]
+      for (int g = qg0; g < G; g += 2) {
+        const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)kv * G + g) * kDh;
+        float v = __bfloat162float(qp[qc]);
+        if (p.theta > 0.f) {
+          const float o = __bfloat162float(qp[qc ^ 64]);
+          v = (qc < 64) ? v * q_cs - o * q_sn : v * q_cs + o * q_sn;
+        }
+        qs[qc * kMaxGroup + g] = v * q_scale;
+      }
+      epi_sync();
+      // ---- K^ row of this thread's token: columns [32*half, +32) and their RoPE partners 64 further
+      if (ok) ok = mbar_wait(&k_full[buf], aph, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      float lg[kMaxGroup];
+#pragma unroll
+      for (int g = 0; g < kMaxGroup; ++g) lg[g] = 0.f;
+      if (ok) {
+        uint32_t ka[32], kb[32];
+        const uint32_t base = tmem_base + (uint32_t)buf * 128 + lane_addr + (uint32_t)half * 32;
+        tmem_ld32(base, ka);
+        tmem_ld32(base + 64, kb);
+        tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive(&k_empty[buf]);
+#pragma unroll
+        for (int ii = 0; ii < 32; ++ii) {
+          const int i = half * 32 + ii;
+          float k1 = __uint_as_float(ka[ii]), k2 = __uint_as_float(kb[ii]);
+          if (p.theta > 0.f) {
+            const float2 t = sc[i * kTok + lane_row];
+            const float r1 = k1 * t.y - k2 * t.x, r2 = k2 * t.y + k1 * t.x;
+            k1 = r1;
+            k2 = r2;
+          }
+          const float4 qa = *reinterpret_cast<const float4 *>(qs + i * kMaxGroup);
+          const float4 qb = *reinterpret_cast<const float4 *>(qs + (i + 64) * kMaxGroup);
+          lg[0] = fmaf(qa.x, k1, fmaf(qb.x, k2, lg[0]));
+          lg[1] = fmaf(qa.y, k1, fmaf(qb.y, k2, lg[1]));
+          lg[2] = fmaf(qa.z, k1, fmaf(qb.z, k2, lg[2]));
+          lg[3] = fmaf(qa.w, k1, fmaf(qb.w, k2, lg[3]));
+          if (G > 4) {
+            const float4 qc4 = *reinterpret_cast<const float4 *>(qs + i * kMaxGroup + 4);
+            const float4 qd4 = *reinterpret_cast<const float4 *>(qs + (i + 64) * kMaxGroup + 4);
+            lg[4] = fmaf(qc4.x, k1, fmaf(qd4.x, k2, lg[4]));
+            lg[5] = fmaf(qc4.y, k1, fmaf(qd4.y, k2, lg[5]));
+            lg[6] = fmaf(qc4.z, k1, fmaf(qd4.z, k2, lg[6]));
+            lg[7] = fmaf(qc4.w, k1, fmaf(qd4.w, k2, lg[7]));
+          }
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < kMaxGroup; ++g)
+        if (g < G) xch[(half * kMaxGroup + g) * 128 + lane_row] = lg[g];
+      epi_sync();
+      // ---- tile softmax: epilogue warp e handles head g = e over the 128 tokens
+      if (e < G) {
+        float l4[4], m = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int t = u * 32 + lane;
+          l4[u] = (t < nt) ? xch[e * 128 + t] + xch[(kMaxGroup + e) * 128 + t] : -INFINITY;
+          m = fmaxf(m, l4[u]);
+        }
+        m = warp_max(m);
+        float ssum = 0.f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float pe = (l4[u] == -INFINITY) ? 0.f : __expf(l4[u] - m);
+          ps[(u * 32 + lane) * kMaxGroup + e] = pe;
+          ssum += pe;
+        }
+        ssum = warp_sum(ssum);
+        if (lane == 0) p.part_ms[((size_t)b * p.Hq + (size_t)kv * G + e) * p.n_tiles + tile] = make_float2(m, ssum);
+      }
+      epi_sync();
+      // ---- V^^T row of this thread's channel: tokens [64*half, +64)
+      if (ok) ok = mbar_wait(&v_full[buf], aph, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      float o[kMaxGroup];
+#pragma unroll
+      for (int g = 0; g < kMaxGroup; ++g) o[g] = 0.f;
+      if (ok) {
+        uint32_t va[32], vb[32];
+        const uint32_t base = tmem_base + 256u + (uint32_t)buf * 128 + lane_addr + (uint32_t)half * 64;
+        tmem_ld32(base, va);
+        tmem_ld32(base + 32, vb);
+        tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive(&v_empty[buf]);
+#pragma unroll
+        for (int ii = 0; ii < 64; ++ii) {
+          const float v = __uint_as_float(ii < 32 ? va[ii & 31] : vb[ii & 31]);
+          const float *pp = ps + (half * 64 + ii) * kMaxGroup;
+          const float4 pa = *reinterpret_cast<const float4 *>(pp);
+          o[0] = fmaf(pa.x, v, o[0]);
+          o[1] = fmaf(pa.y, v, o[1]);
+          o[2] = fmaf(pa.z, v, o[2]);
+          o[3] = fmaf(pa.w, v, o[3]);
+          if (G > 4) {
+            const float4 pb = *reinterpret_cast<const float4 *>(pp + 4);
+            o[4] = fmaf(pb.x, v, o[4]);
+            o[5] = fmaf(pb.y, v, o[5]);
+            o[6] = fmaf(pb.z, v, o[6]);
+            o[7] = fmaf(pb.w, v, o[7]);
+          }
+        }
+      }
+      if (half == 1) {
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g)
+          if (g < G) xch[g * 128 + lane_row] = o[g];
+      }
+      epi_sync();
+      if (half == 0) {
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g)
+          if (g < G)
+            p.part_o[(((size_t)b * p.Hq + (size_t)kv * G + g) * p.n_tiles + tile) * kDh + lane_row] =
+                o[g] + xch[g * 128 + lane_row];
+      }
+      epi_sync();  // xch / ps / qs are rewritten by the next head
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *abort_flag && p.dev_status) atomicOr(p.dev_status, S4R_DEV_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+int att_fast_kvsplit(const Layer &ly, int n_tiles) {
+  // split the KV heads over CTAs until the grid roughly fills the GPU
+  int split = 1;
+  while (split < ly.Hkv && (long)ly.B * n_tiles * split < 120 && ly.Hkv % (split * 2) == 0) split *= 2;
+  return split;
+}
+
+cudaError_t launch_attend_sm100(const StepArgs &a) {
+  const Layer &ly = a.ly;
+  if (a.plan.n_att_tiles == 0) return cudaSuccess;
+  CUtensorMap tm_k, tm_v;
+  if (!make_tmap_bf16_2d(&tm_k, a.basis_k, (uint64_t)ly.B * ly.D, (uint64_t)ly.rk, 128) ||
+      !make_tmap_bf16_2d(&tm_v, a.basis_v, (uint64_t)ly.B * ly.D, (uint64_t)ly.rv, 128))
+    return cudaErrorInvalidValue;
+  AttFastParams p;
+  p.q = (const __nv_bfloat16 *)a.q;
+  p.coef_k = (const __nv_bfloat16 *)a.coef_k;
+  p.coef_v = (const __nv_bfloat16 *)a.coef_v;
+  p.coef_len = a.coef_len;
+  p.sel_idx = a.sel_idx;
+  p.sel_count = a.sel_count;
+  p.part_o = (float *)(a.ws + a.plan.off_att);
+  p.part_ms = (float2 *)(a.ws + a.plan.off_att_ms);
+  p.Hq = ly.Hq; p.Hkv = ly.Hkv; p.G = ly.G; p.D = ly.D; p.rk = ly.rk; p.rv = ly.rv; p.s = ly.s;
+  p.n_tiles = a.plan.n_att_tiles;
+  p.sel_stride = a.window + a.top_k;
+  const int split = att_fast_kvsplit(ly, p.n_tiles);
+  p.nkv = ly.Hkv / split;
+  p.cap = ly.cap;
+  p.max_len = a.plan.max_len;
+  p.theta = a.theta;
+  p.dev_status = a.dev_status;
+  const size_t smem = 1024 + (size_t)(ly.rk / 64 + ly.rv / 64 + kRing) * kBlkBytes + sizeof(float2) * 64 * kTok +
+                      sizeof(float) * (kDh * kMaxGroup + kTok * kMaxGroup + 2 * kMaxGroup * 128) + 1024;
+  static size_t smem_set = 0;
+  if (smem > smem_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_attend_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    smem_set = smem;
+  }
+  dim3 grid(p.n_tiles, split, ly.B);
+  k_attend_sm100<<<grid, kThreads, smem, a.stream>>>(tm_k, tm_v, p);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace s4r

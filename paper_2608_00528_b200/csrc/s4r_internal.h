@@ -37,6 +37,11 @@ cudaError_t launch_select(const StepArgs &a);
 bool scan_fast_supported(const Layer &ly);
 int scan_fast_parts(const Layer &ly);  // CTAs (= softmax partials) per sequence; 0 on error
 cudaError_t launch_scan_sm100(const StepArgs &a);
+inline bool att_fast_supported(const Layer &ly) {
+  return ly.dtype == S4R_BF16 && ly.dh == 128 && ly.rk % 64 == 0 && ly.rv % 64 == 0 && ly.rk >= 64 && ly.rv >= 64 &&
+         (ly.rk + ly.rv) / 64 <= 6 && (int64_t)ly.B * ly.D < 0x7fffffffLL;
+}
+cudaError_t launch_attend_sm100(const StepArgs &a);
 
 cudaError_t launch_attend_generic(const StepArgs &a);
 cudaError_t launch_merge(const StepArgs &a);
