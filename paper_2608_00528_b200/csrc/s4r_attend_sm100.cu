@@ -91,6 +91,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
     int rix = (tid < nt) ? p.sel_idx[(size_t)b * p.sel_stride + t0 + tid] : -1;
     rows[tid] = rix < 0 ? -1 : min(rix, max(L - 1, 0));
   }
+  double *inv_freq = reinterpret_cast<double *>(xch);  // [64], only needed while the sin/cos table is built
+  if (tid >= 128 && tid < 192 && p.theta > 0.f) inv_freq[tid - 128] = rope_inv_freq(tid - 128, kDh, p.theta);
   __syncthreads();
 
   // ---- gather the selected coefficient rows into swizzled K-major tiles (zero rows past the tile's end)
@@ -114,7 +116,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
       for (int i = tid; i < 64 * kTok; i += kThreads) {
         const int pair = i >> 7, t = i & (kTok - 1);
         float sn = 0.f, cs = 1.f;
-        if (rows[t] >= 0) rope_sincos(p.s + rows[t], rope_inv_freq(pair, kDh, p.theta), sn, cs);
+        if (rows[t] >= 0) rope_sincos(p.s + rows[t], inv_freq[pair], sn, cs);
         sc[i] = make_float2(sn, cs);
       }
     }

@@ -14,7 +14,7 @@ constexpr int kMaxPoolHalf = 15;   // kappa <= 31
 constexpr int kScanRows = 1024;    // rows of C^K per scan CTA (also the granularity of the softmax partials)
 constexpr int kAttTok = 32;        // selected rows per CTA in the generic reconstruct+attend kernel
 constexpr int kSelThreads = 1024;  // threads per CTA of the selection kernel (one position each per tile)
-constexpr int kMaxCluster = 8;     // portable cluster size
+constexpr int kMaxCluster = 16;    // CTAs per sequence in the selection kernel (8 is the portable cluster size)
 constexpr int kQSlices = 8;        // D' is split into this many slices by the query projection (partials summed by readers)
 constexpr int kMaxParts = 256;     // upper bound of softmax partials per sequence written by a scan kernel
 
@@ -90,7 +90,7 @@ __device__ inline void rope_sincos(int pos, double inv_freq, float &sn, float &c
   double k = rint(a * kInv2Pi);
   double red = fma(-k, k2PiHi, a);
   red = fma(-k, k2PiLo, red);
-  sincosf((float)red, &sn, &cs);
+  __sincosf((float)red, &sn, &cs);  // |red| <= pi: the fast approximations are accurate to ~2^-21 there
 }
 
 // ---- host-side plan of one decode step -------------------------------------------------------------

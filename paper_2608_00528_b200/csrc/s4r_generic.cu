@@ -1,11 +1,7 @@
 // Generic kernels of the S4R decode step and prefill projection: any supported geometry, fp32 or bf16
 // storage, fp32 arithmetic on the CUDA cores.  They are the whole path for fp32 storage and the reference
 // implementation that the specialised sm_100a kernels (TMA / tcgen05) replace for bf16 storage.
-#include <cooperative_groups.h>
-
 #include "s4r_internal.h"
-
-namespace cg = cooperative_groups;
 
 namespace s4r {
 
@@ -195,272 +191,6 @@ cudaError_t launch_scan_generic(const StepArgs &a) {
     k_scan<float><<<grid, 256, 0, a.stream>>>((const float *)a.coef_k, a.coef_len, cq, Z, part, ly.rk, ly.G, ly.cap,
                                               a.plan.max_len, a.plan.z_stride, a.plan.n_scan_chunks, isr,
                                               a.dev_status);
-  S4R_LAUNCH_CHECK();
-  return cudaSuccess;
-}
-
-// ======================================================================================================
-// Relevance + selection (Eq. 9-15).  One thread-block cluster per sequence; each CTA owns a contiguous
-// slice of the cache.  Scores are softmax probabilities (>= 0), so their fp32 bit patterns order like the
-// values; the k-th largest candidate is found by a 3-pass radix select (11 + 11 + 10 bits) whose
-// histograms are summed across the cluster through distributed shared memory, and the winners are written
-// in ascending index order (equal scores: lower index first).
-// ======================================================================================================
-struct SelParams {
-  const float *Z;
-  const float2 *part;
-  const int32_t *coef_len;
-  float *score;
-  int32_t *sel_idx, *sel_count;
-  int G, n_chunks, window, top_k, kappa, pool_mode, group_mode;
-  int64_t max_len, z_stride;
-  int32_t *dev_status;
-};
-
-// exclusive prefix sum over the block (kSelThreads threads); returns the exclusive value, total in *total
-__device__ inline unsigned block_excl_scan(unsigned v, unsigned *s_warp, unsigned *total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  unsigned inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    unsigned t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  if (lane == 31) s_warp[warp] = inc;
-  __syncthreads();
-  if (warp == 0) {
-    unsigned w = s_warp[lane];
-    unsigned winc = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      unsigned t = __shfl_up_sync(0xffffffffu, winc, o);
-      if (lane >= o) winc += t;
-    }
-    s_warp[lane] = winc - w;       // exclusive offset of each warp
-    if (lane == 31) s_warp[32] = winc;  // grand total
-  }
-  __syncthreads();
-  unsigned res = s_warp[warp] + inc - v;
-  *total = s_warp[32];
-  __syncthreads();
-  return res;
-}
-
-// Sum the per-CTA histograms of the cluster and locate the bin that holds the k_rem-th largest element
-// (bins are scanned from the top).  Returns the bin; *above = number of elements in higher bins.
-__device__ inline unsigned find_bin(cg::cluster_group &cluster, unsigned *s_hist, unsigned *s_warp, unsigned *s_bc,
-                                    int nbins, unsigned k_rem, unsigned *above) {
-  const int CL = cluster.num_blocks();
-  cluster.sync();  // every CTA's histogram is complete
-  const int t = threadIdx.x;
-  const int b0 = nbins - 1 - 2 * t, b1 = nbins - 2 - 2 * t;
-  unsigned c0 = 0, c1 = 0;
-  for (int rk = 0; rk < CL; ++rk) {
-    const unsigned *h = cluster.map_shared_rank(s_hist, rk);
-    if (b0 >= 0) c0 += h[b0];
-    if (b1 >= 0) c1 += h[b1];
-  }
-  unsigned total;
-  unsigned excl = block_excl_scan(c0 + c1, s_warp, &total);
-  if (b0 >= 0 && excl < k_rem && k_rem <= excl + c0) {
-    s_bc[0] = (unsigned)b0;
-    s_bc[1] = excl;
-  } else if (b1 >= 0 && excl + c0 < k_rem && k_rem <= excl + c0 + c1) {
-    s_bc[0] = (unsigned)b1;
-    s_bc[1] = excl + c0;
-  }
-  cluster.sync();  // remote reads done before anyone clears its histogram; also a block barrier for s_bc
-  *above = s_bc[1];
-  return s_bc[0];
-}
-
-__global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
-  cg::cluster_group cluster = cg::this_cluster();
-  const int CL = cluster.num_blocks();
-  const int rank = cluster.block_rank();
-  const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  constexpr int HALO = 16;
-  __shared__ float s_p[kMaxGroup][kSelThreads + 2 * HALO];
-  __shared__ unsigned s_hist[2048];
-  __shared__ float s_M[kMaxGroup], s_iS[kMaxGroup];
-  __shared__ unsigned s_warp[33];
-  __shared__ unsigned s_bc[2];
-  __shared__ unsigned s_cnt[2];
-
-  const int L = clamp_len(p.coef_len, b, p.max_len, p.dev_status);
-  const int W_eff = min(p.window, L);
-  const int n_cand = L - W_eff;
-  const int k_eff = min(p.top_k, n_cand);
-  int32_t *out_idx = p.sel_idx + (size_t)b * (p.window + p.top_k);
-
-  if (rank == 0) {  // local window (Eq. 13), padding and count
-    for (int j = tid; j < W_eff; j += kSelThreads) out_idx[k_eff + j] = n_cand + j;
-    for (int j = k_eff + W_eff + tid; j < p.window + p.top_k; j += kSelThreads) out_idx[j] = -1;
-    if (tid == 0) p.sel_count[b] = k_eff + W_eff;
-  }
-  if (k_eff == 0) return;  // uniform over the cluster: nothing to rank
-
-  // ---- softmax normalisers of Eq. 9 from the scan's per-chunk partials
-  const int used_chunks = p.n_chunks;  // every partial is defined; empty ones are (-inf, 0)
-  if (warp < p.G) {
-    const float2 *pp = p.part + (size_t)b * p.n_chunks * kMaxGroup + warp;
-    float m = -INFINITY;
-    for (int c = lane; c < used_chunks; c += 32) m = fmaxf(m, pp[(size_t)c * kMaxGroup].x);
-    m = warp_max(m);
-    float s = 0.f;
-    for (int c = lane; c < used_chunks; c += 32) {
-      float2 v = pp[(size_t)c * kMaxGroup];
-      if (v.y > 0.f) s += v.y * expf(v.x - m);
-    }
-    s = warp_sum(s);
-    if (lane == 0) {
-      s_M[warp] = m;
-      s_iS[warp] = 1.f / s;
-    }
-  }
-  for (int i = tid; i < 2048; i += kSelThreads) s_hist[i] = 0;
-  __syncthreads();
-
-  // ---- scores of this CTA's slice (Eq. 9-12) + first histogram
-  int per = (L + CL - 1) / CL;
-  per = (per + 3) & ~3;
-  const int begin = min(L, rank * per), end = min(L, begin + per);
-  const int half = p.kappa >> 1;
-  const float *zb = p.Z + (size_t)b * p.G * p.z_stride;
-  float *score = p.score + (size_t)b * p.z_stride;
-  const float inv_kappa = 1.f / (float)p.kappa, inv_G = 1.f / (float)p.G;
-  for (int l0 = begin; l0 < end; l0 += kSelThreads) {
-    for (int g = 0; g < p.G; ++g) {
-      const float M = s_M[g], iS = s_iS[g];
-      for (int i = tid; i < kSelThreads + 2 * HALO; i += kSelThreads) {
-        int l = l0 - HALO + i;
-        s_p[g][i] = (l >= 0 && l < L) ? expf(zb[(size_t)g * p.z_stride + l] - M) * iS : 0.f;
-      }
-    }
-    __syncthreads();
-    const int l = l0 + tid;
-    if (l < end) {
-      float agg = 0.f;
-      for (int g = 0; g < p.G; ++g) {
-        const float *row = &s_p[g][HALO + tid];
-        float v;
-        if (p.pool_mode == S4R_POOL_MAX) {
-          v = row[0];
-          for (int j = 1; j <= half; ++j) v = fmaxf(v, fmaxf(row[-j], row[j]));
-        } else {
-          v = row[-half];
-          for (int j = -half + 1; j <= half; ++j) v += row[j];
-          v *= inv_kappa;
-        }
-        agg = (p.group_mode == S4R_GROUP_MEAN) ? agg + v : fmaxf(agg, v);
-      }
-      if (p.group_mode == S4R_GROUP_MEAN) agg *= inv_G;
-      score[l] = agg;
-      if (l < n_cand) atomicAdd(&s_hist[__float_as_uint(agg) >> 21], 1u);
-    }
-    __syncthreads();
-  }
-
-  // ---- radix select of the k_eff-th largest candidate score
-  const int c_end = min(end, n_cand);
-  unsigned k_rem = (unsigned)k_eff, above;
-  const unsigned bin1 = find_bin(cluster, s_hist, s_warp, s_bc, 2048, k_rem, &above);
-  k_rem -= above;
-  for (int i = tid; i < 2048; i += kSelThreads) s_hist[i] = 0;
-  __syncthreads();
-  for (int l = begin + tid; l < c_end; l += kSelThreads) {
-    unsigned v = __float_as_uint(score[l]);
-    if ((v >> 21) == bin1) atomicAdd(&s_hist[(v >> 10) & 0x7ffu], 1u);
-  }
-  const unsigned bin2 = find_bin(cluster, s_hist, s_warp, s_bc, 2048, k_rem, &above);
-  k_rem -= above;
-  const unsigned pre2 = (bin1 << 11) | bin2;
-  for (int i = tid; i < 2048; i += kSelThreads) s_hist[i] = 0;
-  __syncthreads();
-  for (int l = begin + tid; l < c_end; l += kSelThreads) {
-    unsigned v = __float_as_uint(score[l]);
-    if ((v >> 10) == pre2) atomicAdd(&s_hist[v & 0x3ffu], 1u);
-  }
-  const unsigned bin3 = find_bin(cluster, s_hist, s_warp, s_bc, 1024, k_rem, &above);
-  k_rem -= above;  // how many candidates equal to the threshold are taken (lowest indices first)
-  const unsigned tau = (pre2 << 10) | bin3;
-
-  // ---- per-CTA counts, exchanged through distributed shared memory
-  if (tid < 2) s_cnt[tid] = 0;
-  __syncthreads();
-  {
-    unsigned ngt = 0, neq = 0;
-    for (int l = begin + tid; l < c_end; l += kSelThreads) {
-      unsigned v = __float_as_uint(score[l]);
-      ngt += v > tau;
-      neq += v == tau;
-    }
-    ngt = __reduce_add_sync(0xffffffffu, ngt);
-    neq = __reduce_add_sync(0xffffffffu, neq);
-    if (lane == 0) {
-      atomicAdd(&s_cnt[0], ngt);
-      atomicAdd(&s_cnt[1], neq);
-    }
-  }
-  cluster.sync();
-  unsigned gt_before = 0, eq_before = 0;
-  for (int rk = 0; rk < rank; ++rk) {
-    const unsigned *c = cluster.map_shared_rank(s_cnt, rk);
-    gt_before += c[0];
-    eq_before += c[1];
-  }
-  unsigned out_pos = gt_before + min(eq_before, k_rem);
-  unsigned eq_seen = eq_before;
-
-  // ---- ordered compaction of the winners
-  for (int l0 = begin; l0 < c_end; l0 += kSelThreads) {
-    const int l = l0 + tid;
-    unsigned v = (l < c_end) ? __float_as_uint(score[l]) : 0u;
-    const bool in = l < c_end;
-    const unsigned is_eq = in && v == tau;
-    unsigned tot_eq, tot_take;
-    unsigned eq_rank = eq_seen + block_excl_scan(is_eq, s_warp, &tot_eq);
-    const unsigned take = in && (v > tau || (is_eq && eq_rank < k_rem));
-    unsigned pos = out_pos + block_excl_scan(take, s_warp, &tot_take);
-    if (take) out_idx[pos] = l;
-    out_pos += tot_take;
-    eq_seen += tot_eq;
-  }
-  cluster.sync();  // no CTA leaves while a peer may still read its shared memory
-}
-
-cudaError_t launch_select(const StepArgs &a) {
-  SelParams p;
-  p.Z = (const float *)(a.ws + a.plan.off_z);
-  p.part = (const float2 *)(a.ws + a.plan.off_part);
-  p.coef_len = a.coef_len;
-  p.score = (float *)(a.ws + a.plan.off_score);
-  p.sel_idx = a.sel_idx;
-  p.sel_count = a.sel_count;
-  p.G = a.ly.G;
-  p.n_chunks = a.plan.n_parts;
-  p.window = a.window;
-  p.top_k = a.top_k;
-  p.kappa = a.kappa;
-  p.pool_mode = a.pool_mode;
-  p.group_mode = a.group_mode;
-  p.max_len = a.plan.max_len;
-  p.z_stride = a.plan.z_stride;
-  p.dev_status = a.dev_status;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(a.plan.cluster, a.ly.B);
-  cfg.blockDim = dim3(kSelThreads);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = a.stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = a.plan.cluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, k_select, p);
-  if (e != cudaSuccess) return e;
   S4R_LAUNCH_CHECK();
   return cudaSuccess;
 }
