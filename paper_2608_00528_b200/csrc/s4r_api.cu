@@ -48,6 +48,7 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   p->off_z = off;       off = align_up(off + sizeof(float) * ly.B * ly.G * p->z_stride, 256);
   p->off_part = off;    off = align_up(off + sizeof(float2) * ly.B * p->parts_cap * kMaxGroup, 256);
   p->off_score = off;   off = align_up(off + sizeof(float) * ly.B * p->z_stride, 256);
+  p->off_hist = off;    off = align_up(off + sizeof(unsigned) * ly.B * 2048, 256);
   p->off_att = off;     off = align_up(off + sizeof(float) * ly.B * ly.Hq * (size_t)p->n_att_tiles * ly.dh, 256);
   p->off_att_ms = off;  off = align_up(off + sizeof(float2) * ly.B * ly.Hq * (size_t)p->n_att_tiles, 256);
   p->off_basis_t = off;
@@ -188,6 +189,7 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
     if (launch_scan_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
   }
   stage_mark(2, a.stream);
+  if (launch_relevance(a) != cudaSuccess) return S4R_ERR_CUDA;
   if (launch_select(a) != cudaSuccess) return S4R_ERR_CUDA;
   stage_mark(3, a.stream);
   if (att_fast_supported(ly)) {

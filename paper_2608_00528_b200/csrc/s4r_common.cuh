@@ -14,7 +14,7 @@ constexpr int kMaxPoolHalf = 15;   // kappa <= 31
 constexpr int kScanRows = 1024;    // rows of C^K per scan CTA (also the granularity of the softmax partials)
 constexpr int kAttTok = 32;        // selected rows per CTA in the generic reconstruct+attend kernel
 constexpr int kSelThreads = 1024;  // threads per CTA of the selection kernel (one position each per tile)
-constexpr int kMaxCluster = 16;    // CTAs per sequence in the selection kernel (8 is the portable cluster size)
+constexpr int kMaxCluster = 8;     // CTAs per sequence in the selection kernel (8 is the portable cluster size)
 constexpr int kQSlices = 8;        // D' is split into this many slices by the query projection (partials summed by readers)
 constexpr int kMaxParts = 256;     // upper bound of softmax partials per sequence written by a scan kernel
 
@@ -104,7 +104,7 @@ struct DecodePlan {
   int n_att_tiles;      // row tiles per sequence in the attention kernel
   int cluster;          // CTAs per sequence in the selection kernel
   int att_tok;          // selected rows per attention tile
-  size_t off_cq, off_z, off_part, off_score, off_att, off_att_ms, off_basis_t, total;
+  size_t off_cq, off_z, off_part, off_score, off_hist, off_att, off_att_ms, off_basis_t, total;
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -34,11 +34,14 @@ __device__ inline int clamp_len(const int32_t *coef_len, int b, int64_t max_len,
 // ======================================================================================================
 template <typename T>
 __global__ void __launch_bounds__(256) k_qproj(const T *__restrict__ q, const T *__restrict__ basis,
-                                               float *__restrict__ cq_part, int D, int r, int G, int dh, int Hq) {
+                                               float *__restrict__ cq_part, unsigned *__restrict__ hist, int D,
+                                               int r, int G, int dh, int Hq) {
   extern __shared__ float xs[];  // [G][D / kQSlices]
   __shared__ float red[8][kMaxGroup][32];
   const int b = blockIdx.y, slice = blockIdx.z;
   const int Ds = D / kQSlices, d0 = slice * Ds;
+  if (blockIdx.x == 0 && slice == 0)  // first kernel of the step: clear the score histogram of this sequence
+    for (int i = threadIdx.x; i < 2048; i += 256) hist[(size_t)b * 2048 + i] = 0;
   const int col = blockIdx.x * 32 + (threadIdx.x & 31);
   const int rg = threadIdx.x >> 5;
   for (int i = threadIdx.x; i < G * Ds; i += 256) {
@@ -77,7 +80,7 @@ static cudaError_t qproj_t(const StepArgs &a) {
   size_t smem = (size_t)ly.G * (ly.D / kQSlices) * sizeof(float);
   dim3 grid((ly.rk + 31) / 32, ly.B, kQSlices);
   k_qproj<T><<<grid, 256, smem, a.stream>>>((const T *)a.q, (const T *)a.basis_k, (float *)(a.ws + a.plan.off_cq),
-                                            ly.D, ly.rk, ly.G, ly.dh, ly.Hq);
+                                            (unsigned *)(a.ws + a.plan.off_hist), ly.D, ly.rk, ly.G, ly.dh, ly.Hq);
   S4R_LAUNCH_CHECK();
   return cudaSuccess;
 }

@@ -31,6 +31,7 @@ int &launch_counter();
 // generic (any supported geometry, fp32 or bf16 storage, CUDA-core arithmetic in fp32)
 cudaError_t launch_qproj(const StepArgs &a);
 cudaError_t launch_scan_generic(const StepArgs &a);
+cudaError_t launch_relevance(const StepArgs &a);
 cudaError_t launch_select(const StepArgs &a);
 
 // sm_100a specialisations for bf16 storage (TMA + tcgen05)

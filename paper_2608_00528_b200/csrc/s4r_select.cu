@@ -1,13 +1,15 @@
-// Relevance + selection (Eq. 9-15).  One thread-block cluster per sequence; each CTA owns a contiguous
-// slice of the cache and keeps its scores in shared memory.
+// Relevance (Eq. 9-12) and selection (Eq. 13-15).
 //
-//   1. softmax normalisers of Eq. 9 from the scan kernel's (max, sum exp) partials;
-//   2. score[l] = F_G over g of pool_kappa(softmax_g)[l]  (Eq. 11-12), 4096 positions per pass;
-//   3. scores are probabilities (>= 0), so their fp32 bit patterns order like the values: the k-th largest
-//      candidate is found exactly by a 3-pass radix select (11 + 11 + 10 bits) whose histograms are summed
-//      across the cluster through distributed shared memory;
-//   4. winners are written in ascending index order (equal scores: lower index first) by warp-level
-//      ballots; the local window of Eq. 13 is appended behind them.
+// k_relevance (whole GPU): score[l] = F_G over g of pool_kappa(softmax_g)[l].  A warp owns 128 consecutive
+//   positions in registers (4 per lane); pooling neighbours come from the adjacent lanes by shuffle, so the
+//   warp emits the middle 120 positions and nothing is staged in shared memory.  Each CTA also builds a
+//   histogram of the top 11 bits of its candidate scores and adds it to the sequence's global histogram.
+// k_select (one thread-block cluster per sequence): scores are probabilities (>= 0), so their fp32 bit
+//   patterns order like the values and the k-th largest candidate is found exactly by a radix select
+//   (11 + 11 + 10 bits): pass 1 reads the global histogram, passes 2 and 3 are summed across the cluster
+//   through distributed shared memory (pushed with remote atomics, never read remotely).  Winners are
+//   written in ascending index order (equal scores: lower index first) by warp ballots; the local window of
+//   Eq. 13 is appended behind them.
 #include <cooperative_groups.h>
 
 #include "s4r_internal.h"
@@ -18,20 +20,181 @@ namespace s4r {
 
 namespace {
 
-constexpr int kHalo = 16;
-constexpr int kSelTile = 4 * kSelThreads;   // positions per scoring pass
+constexpr int kRelThreads = 256;
+constexpr int kRelOut = 120;                // positions a warp emits (128 held, 4 halo on each side)
 constexpr int kSliceCap = 16384;            // scores of a slice kept in shared memory up to this many
 
-struct SelParams {
+struct RelParams {
   const float *Z;
   const float2 *part;
   const int32_t *coef_len;
   float *score;
+  unsigned *hist;  // [B][2048]
+  int G, n_parts, window, kappa, pool_mode, group_mode;
+  int64_t max_len, z_stride;
+};
+
+struct SelParams {
+  const int32_t *coef_len;
+  const float *score;
+  const unsigned *hist;
   int32_t *sel_idx, *sel_count;
-  int G, n_parts, window, top_k, kappa, pool_mode, group_mode;
+  int window, top_k;
   int64_t max_len, z_stride;
   int32_t *dev_status;
 };
+
+__device__ __forceinline__ int clamp_len_q(const int32_t *coef_len, int b, int64_t max_len) {
+  int L = coef_len[b];
+  return L < 0 ? 0 : ((int64_t)L > max_len ? (int)max_len : L);
+}
+
+// pooled value at f[4 + j] over a window of half-width HALF inside the 12 values f[0..11]
+template <int HALF, bool MAXP>
+__device__ __forceinline__ float pool12(const float (&f)[12], int j, float inv_kappa) {
+  if (MAXP) {
+    float v = f[4 + j];
+#pragma unroll
+    for (int d = 1; d <= HALF; ++d) v = fmaxf(v, fmaxf(f[4 + j - d], f[4 + j + d]));
+    return v;
+  }
+  float v = f[4 + j - HALF];
+#pragma unroll
+  for (int d = -HALF + 1; d <= HALF; ++d) v += f[4 + j + d];
+  return v * inv_kappa;
+}
+
+template <int HALF, bool MAXP>
+__device__ __forceinline__ void pool_group(const float (&f)[12], float (&acc)[4], bool group_mean, float inv_kappa) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float v = pool12<HALF, MAXP>(f, j, inv_kappa);
+    acc[j] = group_mean ? acc[j] + v : fmaxf(acc[j], v);
+  }
+}
+
+__global__ void __launch_bounds__(kRelThreads) k_relevance(RelParams p) {
+  __shared__ float s_c[kMaxGroup];  // p = exp2(z * log2e + c), c = -M log2e - log2 S
+  __shared__ float s_M[kMaxGroup], s_iS[kMaxGroup];
+  __shared__ unsigned s_hist[2048];
+  const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int L = clamp_len_q(p.coef_len, b, p.max_len);
+  const int out0 = (blockIdx.x * (kRelThreads / 32) + warp) * kRelOut;  // first position this warp emits
+  if (blockIdx.x * (kRelThreads / 32) * kRelOut >= L) return;          // uniform over the CTA
+  const int W_eff = min(p.window, L), n_cand = L - W_eff;
+  // ---- softmax normalisers of Eq. 9 from the scan's partials (empty partials are (-inf, 0))
+  if (warp < p.G) {
+    const float2 *pp = p.part + (size_t)b * p.n_parts * kMaxGroup + warp;
+    float m = -INFINITY;
+    for (int c = lane; c < p.n_parts; c += 32) m = fmaxf(m, pp[(size_t)c * kMaxGroup].x);
+    m = warp_max(m);
+    float s = 0.f;
+    for (int c = lane; c < p.n_parts; c += 32) {
+      const float2 v = pp[(size_t)c * kMaxGroup];
+      if (v.y > 0.f) s += v.y * expf(v.x - m);
+    }
+    s = warp_sum(s);
+    if (lane == 0) {
+      s_M[warp] = m;
+      s_iS[warp] = 1.f / s;
+      s_c[warp] = -m * 1.4426950408889634f - log2f(s);
+    }
+  }
+  for (int i = tid; i < 2048; i += kRelThreads) s_hist[i] = 0;
+  __syncthreads();
+
+  const float *zb = p.Z + (size_t)b * p.G * p.z_stride;
+  const int half = p.kappa >> 1;
+  const bool group_mean = p.group_mode == S4R_GROUP_MEAN, maxp = p.pool_mode == S4R_POOL_MAX;
+  const float inv_kappa = 1.f / (float)p.kappa, inv_G = 1.f / (float)p.G;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  const int pos = out0 - 4 + 4 * lane;  // first of this lane's 4 positions (lanes 0 and 31 are halo only)
+  if (out0 < L) {
+    if (half <= 4) {
+      for (int g = 0; g < p.G; ++g) {
+        const float *zr = zb + (size_t)g * p.z_stride;
+        const float c = s_c[g];
+        float4 z = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (pos >= 0 && pos + 3 < L) {
+          z = __ldcg(reinterpret_cast<const float4 *>(zr + pos));
+        } else if (pos >= 0) {
+          if (pos < L) z.x = __ldcg(zr + pos);
+          if (pos + 1 < L) z.y = __ldcg(zr + pos + 1);
+          if (pos + 2 < L) z.z = __ldcg(zr + pos + 2);
+        }
+        float f[12];
+        f[4] = exp2f(fmaf(z.x, 1.4426950408889634f, c));  // exp2(-inf) = 0 outside the cache
+        f[5] = exp2f(fmaf(z.y, 1.4426950408889634f, c));
+        f[6] = exp2f(fmaf(z.z, 1.4426950408889634f, c));
+        f[7] = exp2f(fmaf(z.w, 1.4426950408889634f, c));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          f[j] = __shfl_up_sync(0xffffffffu, f[4 + j], 1);
+          f[8 + j] = __shfl_down_sync(0xffffffffu, f[4 + j], 1);
+        }
+        switch (half * 2 + (maxp ? 1 : 0)) {
+          case 0: case 1: pool_group<0, true>(f, acc, group_mean, inv_kappa); break;
+          case 2: pool_group<1, false>(f, acc, group_mean, inv_kappa); break;
+          case 3: pool_group<1, true>(f, acc, group_mean, inv_kappa); break;
+          case 4: pool_group<2, false>(f, acc, group_mean, inv_kappa); break;
+          case 5: pool_group<2, true>(f, acc, group_mean, inv_kappa); break;
+          case 6: pool_group<3, false>(f, acc, group_mean, inv_kappa); break;
+          case 7: pool_group<3, true>(f, acc, group_mean, inv_kappa); break;
+          case 8: pool_group<4, false>(f, acc, group_mean, inv_kappa); break;
+          default: pool_group<4, true>(f, acc, group_mean, inv_kappa); break;
+        }
+      }
+    } else {
+      // wide pooling kernels (kappa > 9): every output recomputes its own window; rare, kept simple
+      for (int g = 0; g < p.G; ++g) {
+        const float *zr = zb + (size_t)g * p.z_stride;
+        const float M = s_M[g], iS = s_iS[g];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int l = pos + j;
+          float v = 0.f;
+          if (l >= 0 && l < L) {
+            for (int d = -half; d <= half; ++d) {
+              const int q = l + d;
+              const float pv = (q >= 0 && q < L) ? __expf(__ldcg(zr + q) - M) * iS : 0.f;
+              v = maxp ? fmaxf(v, pv) : v + pv;
+            }
+            if (!maxp) v *= inv_kappa;
+          }
+          acc[j] = group_mean ? acc[j] + v : fmaxf(acc[j], v);
+        }
+      }
+    }
+  }
+  // ---- store + histogram of the top 11 bits (lanes that hit the same bin send one atomic)
+  const bool emit = lane >= 1 && lane <= 30 && out0 < L;
+  float sc[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) sc[j] = group_mean ? acc[j] * inv_G : acc[j];
+  float *srow = p.score + (size_t)b * p.z_stride;
+  if (emit) {
+    if (pos + 3 < L) {
+      *reinterpret_cast<float4 *>(srow + pos) = make_float4(sc[0], sc[1], sc[2], sc[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (pos + j < L) srow[pos + j] = sc[j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const bool valid = emit && pos + j < n_cand;
+    const unsigned bin = valid ? (__float_as_uint(sc[j]) >> 21) : 0xffffffffu;
+    const unsigned peers = __match_any_sync(0xffffffffu, bin);
+    if (valid && lane == __ffs(peers) - 1) atomicAdd(&s_hist[bin], (unsigned)__popc(peers));
+  }
+  __syncthreads();
+  unsigned *gh = p.hist + (size_t)b * 2048;
+  for (int i = tid; i < 2048; i += kRelThreads) {
+    const unsigned c = s_hist[i];
+    if (c) atomicAdd(&gh[i], c);
+  }
+}
 
 // exclusive prefix sum over the block; total in *total
 __device__ inline unsigned block_excl_scan(unsigned v, unsigned *s_warp, unsigned *total) {
@@ -62,11 +225,26 @@ __device__ inline unsigned block_excl_scan(unsigned v, unsigned *s_warp, unsigne
   return res;
 }
 
-// Sum the per-CTA histograms of the cluster and locate the bin that holds the k_rem-th largest element
-// (bins are scanned from the top).  Every CTA pushes its non-empty bins into rank 0's `s_tot` with remote
-// atomics (no remote reads, so nobody waits on distributed-shared-memory latency); rank 0 scans the totals,
-// writes (bin, elements above it) into every CTA's `s_bc` and clears `s_tot` for the next round.
-// Returns the bin; *above = number of elements in higher bins.
+// Locate, in a histogram held in this CTA's shared memory, the bin with the k_rem-th largest element (bins
+// scanned from the top).  Result in s_bc[0] (bin) and s_bc[1] (elements in higher bins); block-synchronous.
+__device__ inline void locate_bin(const unsigned *tot, unsigned *s_warp, unsigned *s_bc, int nbins, unsigned k_rem) {
+  const int t = threadIdx.x;
+  const int b0 = nbins - 1 - 2 * t, b1 = nbins - 2 - 2 * t;
+  const unsigned c0 = b0 >= 0 ? tot[b0] : 0u, c1 = b1 >= 0 ? tot[b1] : 0u;
+  unsigned total;
+  const unsigned excl = block_excl_scan(c0 + c1, s_warp, &total);
+  if (b0 >= 0 && excl < k_rem && k_rem <= excl + c0) {
+    s_bc[0] = (unsigned)b0;
+    s_bc[1] = excl;
+  } else if (b1 >= 0 && excl + c0 < k_rem && k_rem <= excl + c0 + c1) {
+    s_bc[0] = (unsigned)b1;
+    s_bc[1] = excl + c0;
+  }
+  __syncthreads();
+}
+
+// Cluster-wide version: every CTA pushes its non-empty bins into rank 0's `s_tot` with remote atomics,
+// rank 0 locates the bin, writes the result into every CTA's `s_bc` and clears `s_tot` for the next round.
 __device__ inline unsigned find_bin(cg::cluster_group &cluster, unsigned *s_hist, unsigned *s_tot, unsigned *s_warp,
                                     unsigned *s_bc, int nbins, unsigned k_rem, unsigned *above) {
   const int CL = cluster.num_blocks();
@@ -81,27 +259,13 @@ __device__ inline unsigned find_bin(cg::cluster_group &cluster, unsigned *s_hist
   }
   cluster.sync();  // all pushes have landed
   if (cluster.block_rank() == 0) {
-    const int b0 = nbins - 1 - 2 * t, b1 = nbins - 2 - 2 * t;
-    const unsigned c0 = b0 >= 0 ? s_tot[b0] : 0u, c1 = b1 >= 0 ? s_tot[b1] : 0u;
-    unsigned total;
-    const unsigned excl = block_excl_scan(c0 + c1, s_warp, &total);
-    unsigned found = 0xffffffffu, abv = 0;
-    if (b0 >= 0 && excl < k_rem && k_rem <= excl + c0) {
-      found = (unsigned)b0;
-      abv = excl;
-    } else if (b1 >= 0 && excl + c0 < k_rem && k_rem <= excl + c0 + c1) {
-      found = (unsigned)b1;
-      abv = excl + c0;
+    locate_bin(s_tot, s_warp, s_bc, nbins, k_rem);
+    if (t < CL && t > 0) {
+      unsigned *bc = cluster.map_shared_rank(s_bc, t);
+      bc[0] = s_bc[0];
+      bc[1] = s_bc[1];
     }
-    if (found != 0xffffffffu) {
-      for (int rk = 0; rk < CL; ++rk) {
-        unsigned *bc = cluster.map_shared_rank(s_bc, rk);
-        bc[0] = found;
-        bc[1] = abv;
-      }
-    }
-    if (b0 >= 0) s_tot[b0] = 0;
-    if (b1 >= 0) s_tot[b1] = 0;
+    for (int i = t; i < nbins; i += kSelThreads) s_tot[i] = 0;
   }
   cluster.sync();  // result delivered, totals cleared
   *above = s_bc[1];
@@ -113,14 +277,10 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
   const int CL = cluster.num_blocks();
   const int rank = cluster.block_rank();
   const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  extern __shared__ __align__(16) float dsm[];
-  float *s_score = dsm;                 // [kSliceCap]
-  float *s_p = dsm + kSliceCap;         // [G][kSelTile + 2 * kHalo]
-  constexpr int kRow = kSelTile + 2 * kHalo;
+  extern __shared__ __align__(16) float s_score[];  // [kSliceCap]
   __shared__ unsigned s_hist[2048];
-  __shared__ unsigned s_tot[2048];      // cluster-wide histogram, used in rank 0 only
-  __shared__ unsigned s_cnts[kMaxCluster][2];  // (greater, equal) counts of the lower-ranked CTAs
-  __shared__ float s_M[kMaxGroup], s_iS[kMaxGroup];
+  __shared__ unsigned s_tot[2048];              // cluster-wide histogram, used in rank 0 only
+  __shared__ unsigned s_cnts[kMaxCluster][2];   // (greater, equal) counts of the lower-ranked CTAs
   __shared__ unsigned s_warp[33];
   __shared__ unsigned s_bc[2];
   __shared__ unsigned s_wcnt[32][2];
@@ -142,149 +302,44 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
   }
   if (k_eff == 0) return;  // uniform over the cluster: nothing to rank
 
-  // ---- softmax normalisers of Eq. 9 from the scan's partials (empty partials are (-inf, 0))
-  if (warp < p.G) {
-    const float2 *pp = p.part + (size_t)b * p.n_parts * kMaxGroup + warp;
-    float m = -INFINITY;
-    for (int c = lane; c < p.n_parts; c += 32) m = fmaxf(m, pp[(size_t)c * kMaxGroup].x);
-    m = warp_max(m);
-    float s = 0.f;
-    for (int c = lane; c < p.n_parts; c += 32) {
-      float2 v = pp[(size_t)c * kMaxGroup];
-      if (v.y > 0.f) s += v.y * expf(v.x - m);
-    }
-    s = warp_sum(s);
-    if (lane == 0) {
-      s_M[warp] = m;
-      s_iS[warp] = 1.f / s;
-    }
-  }
+  // ---- pass 1 of the radix select from the global histogram of the top 11 bits
   for (int i = tid; i < 2048; i += kSelThreads) {
-    s_hist[i] = 0;
+    s_hist[i] = __ldcg(p.hist + (size_t)b * 2048 + i);
     s_tot[i] = 0;
   }
-  cluster.sync();  // rank 0's totals are clear before anybody pushes into them
-
-  // ---- scores of this CTA's slice (Eq. 9-12) + first histogram
-  int per = (L + CL - 1) / CL;
-  per = (per + 3) & ~3;
-  const int begin = min(L, rank * per), end = min(L, begin + per);
-  const int half = p.kappa >> 1;
-  const float *zb = p.Z + (size_t)b * p.G * p.z_stride;
-  float *score = (per <= kSliceCap) ? s_score : p.score + (size_t)b * p.z_stride + begin;  // indexed by l - begin
-  const float inv_kappa = 1.f / (float)p.kappa, inv_G = 1.f / (float)p.G;
-  for (int l0 = begin; l0 < end; l0 += kSelTile) {
-    {
-      // all loads of the pass are issued before anything is stored, so they overlap
-      const int l = l0 + 4 * tid;
-      const bool vec = l + 3 < L;
-      const int side = (tid >> 4) & 1, hj = tid & 15;
-      const int lh = side ? l0 + kSelTile + hj : l0 - kHalo + hj;
-      const bool halo_ok = tid < 2 * kHalo && lh >= 0 && lh < L;
-      float4 z[kMaxGroup];
-      float zh[kMaxGroup];
-#pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g) {
-        z[g] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-        zh[g] = -INFINITY;
-        if (g < p.G) {
-          const float *zr = zb + (size_t)g * p.z_stride;
-          if (vec) {
-            z[g] = __ldcg(reinterpret_cast<const float4 *>(zr + l));
-          } else {
-            if (l < L) z[g].x = __ldcg(zr + l);
-            if (l + 1 < L) z[g].y = __ldcg(zr + l + 1);
-            if (l + 2 < L) z[g].z = __ldcg(zr + l + 2);
-          }
-          if (halo_ok) zh[g] = __ldcg(zr + lh);
-        }
-      }
-#pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g) {
-        if (g < p.G) {
-          const float M = s_M[g], iS = s_iS[g];
-          float *row = s_p + g * kRow;
-          // exp(-inf) = 0 for the positions past the end
-          *reinterpret_cast<float4 *>(row + kHalo + 4 * tid) =
-              make_float4(__expf(z[g].x - M) * iS, __expf(z[g].y - M) * iS, __expf(z[g].z - M) * iS,
-                          __expf(z[g].w - M) * iS);
-          if (tid < 2 * kHalo) row[side ? kHalo + kSelTile + hj : hj] = __expf(zh[g] - M) * iS;
-        }
-      }
-    }
-    __syncthreads();
-    float sc4[4];
-    if (half <= 4) {
-      // this thread's 4 positions and up to 4 neighbours on each side, from three aligned vector reads
-#pragma unroll
-      for (int j = 0; j < 4; ++j) sc4[j] = 0.f;
-      for (int g = 0; g < p.G; ++g) {
-        const float4 *c4 = reinterpret_cast<const float4 *>(s_p + g * kRow + kHalo + 4 * tid - 4);
-        const float4 a = c4[0], bq = c4[1], cq = c4[2];
-        const float f[12] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y, cq.z, cq.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          float v;
-          if (p.pool_mode == S4R_POOL_MAX) {
-            v = f[4 + j];
-#pragma unroll
-            for (int d = 1; d <= 4; ++d)
-              if (d <= half) v = fmaxf(v, fmaxf(f[4 + j - d], f[4 + j + d]));
-          } else {
-            v = 0.f;
-#pragma unroll
-            for (int d = -4; d <= 4; ++d)
-              if (d >= -half && d <= half) v += f[4 + j + d];
-            v *= inv_kappa;
-          }
-          sc4[j] = (p.group_mode == S4R_GROUP_MEAN) ? sc4[j] + v : fmaxf(sc4[j], v);
-        }
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float agg = 0.f;
-        for (int g = 0; g < p.G; ++g) {
-          const float *c = s_p + g * kRow + kHalo + 4 * tid + j;
-          float v;
-          if (p.pool_mode == S4R_POOL_MAX) {
-            v = c[0];
-            for (int d = 1; d <= half; ++d) v = fmaxf(v, fmaxf(c[-d], c[d]));
-          } else {
-            v = c[-half];
-            for (int d = -half + 1; d <= half; ++d) v += c[d];
-            v *= inv_kappa;
-          }
-          agg = (p.group_mode == S4R_GROUP_MEAN) ? agg + v : fmaxf(agg, v);
-        }
-        sc4[j] = agg;
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int l = l0 + 4 * tid + j;
-      const float agg = (p.group_mode == S4R_GROUP_MEAN) ? sc4[j] * inv_G : sc4[j];
-      if (l < end) score[l - begin] = agg;
-      // histogram of the top 11 bits; lanes that hit the same bin send one atomic (scores cluster in few bins)
-      const bool valid = l < end && l < n_cand;
-      const unsigned bin = valid ? (__float_as_uint(agg) >> 21) : 0xffffffffu;
-      const unsigned peers = __match_any_sync(0xffffffffu, bin);
-      if (valid && lane == __ffs(peers) - 1) atomicAdd(&s_hist[bin], (unsigned)__popc(peers));
-    }
-    __syncthreads();
-  }
-
-  // ---- radix select of the k_eff-th largest candidate score
-  const int c_end = min(end, n_cand);
+  cluster.sync();  // rank 0's totals are clear before anybody pushes into them (also a block barrier)
   unsigned k_rem = (unsigned)k_eff, above;
-  const unsigned bin1 = find_bin(cluster, s_hist, s_tot, s_warp, s_bc, 2048, k_rem, &above);
-  k_rem -= above;
+  locate_bin(s_hist, s_warp, s_bc, 2048, k_rem);
+  const unsigned bin1 = s_bc[0];
+  k_rem -= s_bc[1];
+  __syncthreads();
   for (int i = tid; i < 2048; i += kSelThreads) s_hist[i] = 0;
   __syncthreads();
-  for (int l = begin + tid; l < c_end; l += kSelThreads) {
-    unsigned v = __float_as_uint(score[l - begin]);
-    if ((v >> 21) == bin1) atomicAdd(&s_hist[(v >> 10) & 0x7ffu], 1u);
+
+  // ---- this CTA's slice of the candidates: copy the scores into shared memory, histogram of the next 11 bits
+  int per = (n_cand + CL - 1) / CL;
+  per = (per + 3) & ~3;
+  const int begin = min(n_cand, rank * per), c_end = min(n_cand, begin + per);
+  const float *gscore = p.score + (size_t)b * p.z_stride;
+  const bool in_smem = per <= kSliceCap;
+  for (int l0 = begin + 4 * tid; l0 < c_end; l0 += 4 * kSelThreads) {
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (l0 + 3 < c_end) {
+      const float4 t = __ldcg(reinterpret_cast<const float4 *>(gscore + l0));
+      v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (l0 + j < c_end) v[j] = __ldcg(gscore + l0 + j);
+    }
+    if (in_smem) *reinterpret_cast<float4 *>(s_score + (l0 - begin)) = make_float4(v[0], v[1], v[2], v[3]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const unsigned u = __float_as_uint(v[j]);
+      if (l0 + j < c_end && (u >> 21) == bin1) atomicAdd(&s_hist[(u >> 10) & 0x7ffu], 1u);
+    }
   }
+  const float *score = in_smem ? s_score : gscore + begin;  // indexed by l - begin
   const unsigned bin2 = find_bin(cluster, s_hist, s_tot, s_warp, s_bc, 2048, k_rem, &above);
   k_rem -= above;
   const unsigned pre2 = (bin1 << 11) | bin2;
@@ -371,63 +426,56 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
 
 }  // namespace
 
-cudaError_t launch_select(const StepArgs &a) {
-  SelParams p;
+cudaError_t launch_relevance(const StepArgs &a) {
+  if (a.plan.max_len <= 0) return cudaSuccess;
+  RelParams p;
   p.Z = (const float *)(a.ws + a.plan.off_z);
   p.part = (const float2 *)(a.ws + a.plan.off_part);
   p.coef_len = a.coef_len;
   p.score = (float *)(a.ws + a.plan.off_score);
-  p.sel_idx = a.sel_idx;
-  p.sel_count = a.sel_count;
+  p.hist = (unsigned *)(a.ws + a.plan.off_hist);
   p.G = a.ly.G;
   p.n_parts = a.plan.n_parts;
   p.window = a.window;
-  p.top_k = a.top_k;
   p.kappa = a.kappa;
   p.pool_mode = a.pool_mode;
   p.group_mode = a.group_mode;
   p.max_len = a.plan.max_len;
   p.z_stride = a.plan.z_stride;
+  const int per_cta = (kRelThreads / 32) * kRelOut;
+  dim3 grid((unsigned)((a.plan.max_len + per_cta - 1) / per_cta), a.ly.B);
+  k_relevance<<<grid, kRelThreads, 0, a.stream>>>(p);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select(const StepArgs &a) {
+  SelParams p;
+  p.coef_len = a.coef_len;
+  p.score = (const float *)(a.ws + a.plan.off_score);
+  p.hist = (const unsigned *)(a.ws + a.plan.off_hist);
+  p.sel_idx = a.sel_idx;
+  p.sel_count = a.sel_count;
+  p.window = a.window;
+  p.top_k = a.top_k;
+  p.max_len = a.plan.max_len;
+  p.z_stride = a.plan.z_stride;
   p.dev_status = a.dev_status;
-  const size_t smem = sizeof(float) * ((size_t)kSliceCap + (size_t)a.ly.G * (kSelTile + 2 * kHalo));
+  const size_t smem = sizeof(float) * (size_t)kSliceCap;
   static size_t smem_set = 0;
   if (smem > smem_set) {
     cudaError_t e = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     smem_set = smem;
   }
-  int cluster = a.plan.cluster;
-  if (cluster > 8) {  // 16 CTAs per cluster is beyond the portable size: opt in once and check that it can be placed
-    static int ok16 = -1;
-    if (ok16 < 0) {
-      ok16 = 0;
-      if (cudaFuncSetAttribute(k_select, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
-        cudaLaunchConfig_t probe = {};
-        probe.gridDim = dim3(16, 1);
-        probe.blockDim = dim3(kSelThreads);
-        probe.dynamicSmemBytes = smem;
-        cudaLaunchAttribute pa[1];
-        pa[0].id = cudaLaunchAttributeClusterDimension;
-        pa[0].val.clusterDim.x = 16;
-        pa[0].val.clusterDim.y = 1;
-        pa[0].val.clusterDim.z = 1;
-        probe.attrs = pa;
-        probe.numAttrs = 1;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, k_select, &probe) == cudaSuccess && n >= 1) ok16 = 1;
-      }
-      (void)cudaGetLastError();
-    }
-    if (!ok16) cluster = 8;
-  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(cluster, a.ly.B);
+  cfg.gridDim = dim3(a.plan.cluster, a.ly.B);
   cfg.blockDim = dim3(kSelThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = a.stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = cluster;
+  attr[0].val.clusterDim.x = a.plan.cluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
