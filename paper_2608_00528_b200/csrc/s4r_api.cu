@@ -53,6 +53,7 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   p->off_att_ms = off;  off = align_up(off + sizeof(float2) * ly.B * ly.Hq * (size_t)p->n_att_tiles, 256);
   p->off_basis_t = off;
   p->total = off > 256 ? off : 256;
+  if (ly.dtype == S4R_BF16 && compress_fast_workspace(ly) > p->total) p->total = compress_fast_workspace(ly);
   return true;
 }
 
@@ -103,7 +104,6 @@ int s4r_compress(const s4r_layer_t *layer, const void *K, const void *V, int64_t
                  const void *value_basis, const void *norm_stats, void *sink_k, void *sink_v, void *coef_k,
                  void *coef_v, int32_t *coef_len, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                  void *stream) {
-  (void)workspace; (void)workspace_bytes; (void)dev_status;
   launch_counter() = 0;
   Layer ly;
   if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
@@ -117,8 +117,19 @@ int s4r_compress(const s4r_layer_t *layer, const void *K, const void *V, int64_t
     return S4R_ERR_INVALID_ARG;
   if (int rc = check_arch()) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  if (launch_compress_generic(ly, K, key_basis, ly.rk, sink_k, coef_k, T, st) != cudaSuccess) return S4R_ERR_CUDA;
-  if (launch_compress_generic(ly, V, value_basis, ly.rv, sink_v, coef_v, T, st) != cudaSuccess) return S4R_ERR_CUDA;
+  const bool fast_k = compress_fast_supported(ly, ly.rk, T), fast_v = compress_fast_supported(ly, ly.rv, T);
+  char *bt_k = (char *)workspace;
+  char *bt_v = bt_k + align_up(sizeof(__nv_bfloat16) * (size_t)ly.B * ly.rk * ly.D, 256);
+  if (fast_k || fast_v) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < compress_fast_workspace(ly))
+      return S4R_ERR_WORKSPACE;
+  }
+  if (launch_compress_generic(ly, K, key_basis, ly.rk, sink_k, coef_k, T, !fast_k, st) != cudaSuccess) return S4R_ERR_CUDA;
+  if (fast_k && launch_compress_sm100(ly, K, key_basis, ly.rk, bt_k, coef_k, T, dev_status, st) != cudaSuccess)
+    return S4R_ERR_CUDA;
+  if (launch_compress_generic(ly, V, value_basis, ly.rv, sink_v, coef_v, T, !fast_v, st) != cudaSuccess) return S4R_ERR_CUDA;
+  if (fast_v && launch_compress_sm100(ly, V, value_basis, ly.rv, bt_v, coef_v, T, dev_status, st) != cudaSuccess)
+    return S4R_ERR_CUDA;
   if (launch_set_len(ly, coef_len, T, st) != cudaSuccess) return S4R_ERR_CUDA;
   return S4R_OK;
 }

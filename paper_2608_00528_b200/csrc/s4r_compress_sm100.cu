@@ -1,0 +1,234 @@
+// Prefill projection (Eq. 3) for bf16 on sm_100a: C[T - s, r] = S[s:T, D'] B[D', r] per sequence, as a
+// persistent tcgen05 GEMM.
+//
+// A work item is 256 consecutive token rows of one sequence.  For each 64-wide block of D' a pipeline stage
+// holds two [128 x 64] row blocks of S and one [r x 64] block of B^T (all TMA, 128-byte swizzle); one thread
+// issues 2 x 4 tcgen05.mma (M = 128, N = r, K = 16) per stage into two fp32 accumulators in tensor memory, so
+// every block of B^T that crosses L2 -> SM is used for 256 rows.  Four epilogue warps read the accumulators
+// back, round once to bf16 and store whole 16-byte pieces of the coefficient rows.  B^T ([r, D'], K-major for
+// the tensor core) is produced once per call by a small transpose kernel into the workspace.
+// Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-5 = epilogue.  grid = number of SMs.
+#include "s4r_internal.h"
+#include "s4r_sm100.cuh"
+
+namespace s4r {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kMTile = 256;
+constexpr int kStages = 3;
+constexpr int kCmpThreads = 192;
+
+struct CompressParams {
+  __nv_bfloat16 *coef;
+  int B, r, D, s, n_mtiles;
+  int64_t T, cap;
+  int32_t *dev_status;
+};
+
+// Bt[b][n][k] = basis[b][k][n]
+__global__ void __launch_bounds__(256) k_transpose_basis(const __nv_bfloat16 *__restrict__ basis,
+                                                         __nv_bfloat16 *__restrict__ bt, int D, int r) {
+  __shared__ __nv_bfloat16 tile[32][33];
+  const int b = blockIdx.z, k0 = blockIdx.x * 32, n0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8) {
+    const int k = k0 + i, n = n0 + tx;
+    tile[i][tx] = (k < D && n < r) ? basis[((size_t)b * D + k) * r + n] : __float2bfloat16_rn(0.f);
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int n = n0 + i, k = k0 + tx;
+    if (n < r && k < D) bt[((size_t)b * r + n) * D + k] = tile[tx][i];
+  }
+}
+
+__global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_constant__ CUtensorMap tmap_x,
+                                                                   const __grid_constant__ CUtensorMap tmap_bt,
+                                                                   CompressParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.r * 128;
+  const uint32_t stage_bytes = 2 * a_bytes + ((b_bytes + 1023u) & ~1023u);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kStages * stage_bytes);
+  uint64_t *full = bars, *empty = bars + kStages, *acc_full = bars + 2 * kStages, *acc_empty = acc_full + 1;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 1);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kblocks = p.D >> 6;
+  const int n_items = p.B * p.n_mtiles;
+  const int64_t n_rows = p.T - p.s;
+
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 128);
+    *abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&tmap_x);
+    prefetch_tmap(&tmap_bt);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol = policy_evict_first();
+      int it = 0, issued = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int b = item / p.n_mtiles, mt = item - b * p.n_mtiles;
+        const int y0 = (int)((int64_t)b * p.T + p.s + (int64_t)mt * kMTile);
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % kStages;
+          if (!mbar_wait(&empty[s], ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          uint8_t *st = smem + (size_t)s * stage_bytes;
+          mbar_expect_tx(&full[s], 2 * a_bytes + b_bytes);
+          tma_load_2d_hint(st, &tmap_x, kb * 64, y0, &full[s], pol);
+          tma_load_2d_hint(st + a_bytes, &tmap_x, kb * 64, y0 + 128, &full[s], pol);
+          tma_load_2d(st + 2 * a_bytes, &tmap_bt, kb * 64, b * p.r, &full[s]);
+          issued = it + 1;
+        }
+      }
+      if (*abort_flag) {
+        for (int i = max(0, issued - kStages); i < issued; ++i) {
+          const unsigned long long t_0 = global_ns();
+          while (!mbar_try_wait(&full[i % kStages], (uint32_t)(i / kStages) & 1u))
+            if (global_ns() - t_0 > kWaitLimitNs) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(128, p.r);
+      int it = 0, n_done = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
+        if (!mbar_wait(acc_empty, ((uint32_t)n_done & 1u) ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % kStages;
+          if (!mbar_wait(&full[s], (uint32_t)(it / kStages) & 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+          const uint64_t a0 = umma_desc_sw128(st), a1 = umma_desc_sw128(st + a_bytes), bd = umma_desc_sw128(st + 2 * a_bytes);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4) {
+            umma_bf16(tmem_base, a0 + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc, (kb | k4) != 0);
+            umma_bf16(tmem_base + 256u, a1 + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc, (kb | k4) != 0);
+          }
+          umma_commit(&empty[s]);
+        }
+        if (ok) umma_commit(acc_full);
+      }
+    }
+  } else {
+    const int quad = warp & 3;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    int n_done = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n_done) {
+      const int b = item / p.n_mtiles, mt = item - b * p.n_mtiles;
+      if (ok) ok = mbar_wait(acc_full, (uint32_t)n_done & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+        const int64_t row = (int64_t)mt * kMTile + half * 128 + quad * 32 + lane;
+        __nv_bfloat16 *dst = p.coef + ((size_t)b * p.cap + (size_t)row) * p.r;
+        for (int c0 = 0; c0 < p.r; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + (uint32_t)half * 256u + lane_addr + (uint32_t)c0, v);
+          tmem_ld_wait();
+          if (row < n_rows) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              if (c0 + j < p.r) {
+                uint4 o;
+                __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+                __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+                __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+                o.x = *reinterpret_cast<uint32_t *>(&t0);
+                o.y = *reinterpret_cast<uint32_t *>(&t1);
+                o.z = *reinterpret_cast<uint32_t *>(&t2);
+                o.w = *reinterpret_cast<uint32_t *>(&t3);
+                *reinterpret_cast<uint4 *>(dst + c0 + j) = o;
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *abort_flag && p.dev_status) atomicOr(p.dev_status, S4R_DEV_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+bool compress_fast_supported(const Layer &ly, int r, int64_t T) {
+  return ly.dtype == S4R_BF16 && r % 16 == 0 && r >= 16 && r <= 256 && ly.D % 64 == 0 && T - ly.s > 0 &&
+         (int64_t)ly.B * T < 0x7fffffffLL - 512 && (int64_t)ly.B * r < 0x7fffffffLL;
+}
+
+size_t compress_fast_workspace(const Layer &ly) {
+  return align_up(sizeof(__nv_bfloat16) * (size_t)ly.B * ly.rk * ly.D, 256) +
+         align_up(sizeof(__nv_bfloat16) * (size_t)ly.B * ly.rv * ly.D, 256);
+}
+
+// X: [B, T, D'] rows; basis [B, D', r]; bt: workspace [B, r, D']; coef [B, cap, r]
+cudaError_t launch_compress_sm100(const Layer &ly, const void *X, const void *basis, int r, void *bt, void *coef,
+                                  int64_t T, int32_t *dev_status, cudaStream_t st) {
+  dim3 tg((ly.D + 31) / 32, (r + 31) / 32, ly.B);
+  k_transpose_basis<<<tg, 256, 0, st>>>((const __nv_bfloat16 *)basis, (__nv_bfloat16 *)bt, ly.D, r);
+  ++launch_counter();
+  CUtensorMap tm_x, tm_bt;
+  if (!make_tmap_bf16_2d(&tm_x, X, (uint64_t)ly.B * (uint64_t)T, (uint64_t)ly.D, 128) ||
+      !make_tmap_bf16_2d(&tm_bt, bt, (uint64_t)ly.B * (uint64_t)r, (uint64_t)ly.D, (uint32_t)r))
+    return cudaErrorInvalidValue;
+  CompressParams p;
+  p.coef = (__nv_bfloat16 *)coef;
+  p.B = ly.B; p.r = r; p.D = ly.D; p.s = ly.s;
+  p.T = T; p.cap = ly.cap;
+  p.n_mtiles = (int)((T - ly.s + kMTile - 1) / kMTile);
+  p.dev_status = dev_status;
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return cudaErrorInvalidValue;
+  }
+  const uint32_t stage_bytes = 2 * 128 * 128 + (((uint32_t)r * 128 + 1023u) & ~1023u);
+  const size_t smem = 1024 + (size_t)kStages * stage_bytes + 256;
+  static size_t smem_set = 0;
+  if (smem > smem_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_compress_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    smem_set = smem;
+  }
+  const int n_items = ly.B * p.n_mtiles;
+  const int grid = n_items < sms ? n_items : sms;
+  k_compress_sm100<<<grid, kCmpThreads, smem, st>>>(tm_x, tm_bt, p);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace s4r

@@ -537,13 +537,13 @@ __global__ void k_set_len(int32_t *coef_len, int B, int32_t v) {
 
 template <typename T>
 static cudaError_t compress_t(const Layer &ly, const void *X, const void *basis, int r, void *sink, void *coef,
-                              int64_t n_tok, cudaStream_t st) {
+                              int64_t n_tok, bool do_gemm, cudaStream_t st) {
   if (ly.s > 0) {
     k_copy_sinks<T><<<ly.B, 256, 0, st>>>((const T *)X, (T *)sink, n_tok, ly.s, ly.D);
     S4R_LAUNCH_CHECK();
   }
   const int64_t n = n_tok - ly.s;
-  if (n > 0) {
+  if (n > 0 && do_gemm) {
     dim3 grid((r + 63) / 64, (unsigned)((n + 63) / 64), ly.B);
     k_compress<T><<<grid, 256, 0, st>>>((const T *)X, (const T *)basis, (T *)coef, n_tok, ly.s, ly.D, r, ly.cap);
     S4R_LAUNCH_CHECK();
@@ -551,9 +551,9 @@ static cudaError_t compress_t(const Layer &ly, const void *X, const void *basis,
   return cudaSuccess;
 }
 cudaError_t launch_compress_generic(const Layer &ly, const void *X, const void *basis, int r, void *sink,
-                                    void *coef, int64_t T, cudaStream_t st) {
-  return ly.dtype == S4R_BF16 ? compress_t<__nv_bfloat16>(ly, X, basis, r, sink, coef, T, st)
-                              : compress_t<float>(ly, X, basis, r, sink, coef, T, st);
+                                    void *coef, int64_t T, bool do_gemm, cudaStream_t st) {
+  return ly.dtype == S4R_BF16 ? compress_t<__nv_bfloat16>(ly, X, basis, r, sink, coef, T, do_gemm, st)
+                              : compress_t<float>(ly, X, basis, r, sink, coef, T, do_gemm, st);
 }
 cudaError_t launch_set_len(const Layer &ly, int32_t *coef_len, int64_t T, cudaStream_t st) {
   k_set_len<<<(ly.B + 127) / 128, 128, 0, st>>>(coef_len, ly.B, (int32_t)(T - ly.s));

@@ -46,8 +46,13 @@ cudaError_t launch_attend_sm100(const StepArgs &a);
 
 cudaError_t launch_attend_generic(const StepArgs &a);
 cudaError_t launch_merge(const StepArgs &a);
+// copies the sink rows; runs the CUDA-core GEMM too unless do_gemm is false
 cudaError_t launch_compress_generic(const Layer &ly, const void *X, const void *basis, int r, void *sink,
-                                    void *coef, int64_t T, cudaStream_t st);
+                                    void *coef, int64_t T, bool do_gemm, cudaStream_t st);
+bool compress_fast_supported(const Layer &ly, int r, int64_t T);
+size_t compress_fast_workspace(const Layer &ly);
+cudaError_t launch_compress_sm100(const Layer &ly, const void *X, const void *basis, int r, void *bt, void *coef,
+                                  int64_t T, int32_t *dev_status, cudaStream_t st);
 cudaError_t launch_set_len(const Layer &ly, int32_t *coef_len, int64_t T, cudaStream_t st);
 cudaError_t launch_append(const Layer &ly, const void *k_t, const void *v_t, const void *basis_k,
                           const void *basis_v, void *coef_k, void *coef_v, int32_t *coef_len,

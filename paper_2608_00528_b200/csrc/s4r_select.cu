@@ -111,17 +111,27 @@ __global__ void __launch_bounds__(kRelThreads) k_relevance(RelParams p) {
   const int pos = out0 - 4 + 4 * lane;  // first of this lane's 4 positions (lanes 0 and 31 are halo only)
   if (out0 < L) {
     if (half <= 4) {
-      for (int g = 0; g < p.G; ++g) {
-        const float *zr = zb + (size_t)g * p.z_stride;
-        const float c = s_c[g];
-        float4 z = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-        if (pos >= 0 && pos + 3 < L) {
-          z = __ldcg(reinterpret_cast<const float4 *>(zr + pos));
-        } else if (pos >= 0) {
-          if (pos < L) z.x = __ldcg(zr + pos);
-          if (pos + 1 < L) z.y = __ldcg(zr + pos + 1);
-          if (pos + 2 < L) z.z = __ldcg(zr + pos + 2);
+      // all loads first, so their latencies overlap
+      float4 zz[kMaxGroup];
+#pragma unroll
+      for (int g = 0; g < kMaxGroup; ++g) {
+        zz[g] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (g < p.G) {
+          const float *zr = zb + (size_t)g * p.z_stride;
+          if (pos >= 0 && pos + 3 < L) {
+            zz[g] = __ldcg(reinterpret_cast<const float4 *>(zr + pos));
+          } else if (pos >= 0) {
+            if (pos < L) zz[g].x = __ldcg(zr + pos);
+            if (pos + 1 < L) zz[g].y = __ldcg(zr + pos + 1);
+            if (pos + 2 < L) zz[g].z = __ldcg(zr + pos + 2);
+          }
         }
+      }
+#pragma unroll
+      for (int g = 0; g < kMaxGroup; ++g) {
+        if (g >= p.G) break;
+        const float c = s_c[g];
+        const float4 z = zz[g];
         float f[12];
         f[4] = exp2f(fmaf(z.x, 1.4426950408889634f, c));  // exp2(-inf) = 0 outside the cache
         f[5] = exp2f(fmaf(z.y, 1.4426950408889634f, c));

@@ -174,7 +174,8 @@ def _absdot(x: torch.Tensor, basis: np.ndarray) -> np.ndarray:
     return np.abs(to_np(x)) @ np.abs(basis)
 
 
-@pytest.mark.parametrize("ci,ctx,B", [(0, 1500, 2), (1, 2000 + 13, 2), (3, 1100, 1)])
+@pytest.mark.parametrize("ci,ctx,B", [(0, 1500, 2), (1, 2000 + 13, 2), (3, 1100, 1), (1, 5 * 256 + 4 + 77, 3),
+                                      (3, 300, 2), (1, 4 + 200, 1)])
 def test_compress_matches_oracle(ci, ctx, B):
     s4r = _s4r()
     cfg = _cfg(ci, context=ctx, batch=B)
