@@ -1,0 +1,125 @@
+"""Parity at the benchmark's full sizes (128K context), in the launch configuration bench.py times.
+
+The whole batch is generated on the GPU and compressed by the library.  For a subset of the sequences the
+oracle builds the bases, compresses its own copy of the same input bits and runs its decode step; the
+library's coefficients are compared with the oracle's, then the oracle's coefficients are put into the
+library's cache for those sequences so that the decode comparison is on identical inputs.  The remaining
+sequences are checked through properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import s4r_oracle as O
+from tests.helpers import Problem, run_gpu_step, check_step, to_np, from_np
+
+pytestmark = pytest.mark.gpu
+
+
+class FullSizeProblem(Problem):
+    def __init__(self, cfg, checked):
+        import paper_2608_00528_b200 as s4r
+        self.cfg, self.layer, self.st = cfg, 0, W.storage_dtype(cfg)
+        self.device = torch.device("cuda")
+        dev, st = self.device, self.st
+        B, s, D, T = cfg.batch, cfg.sink_count, cfg.d_kv, cfg.context
+        self.L = cfg.cache_len
+        self.cap = self.L
+        self.checked = list(checked)
+        self.d_K = torch.empty(B, T, D, dtype=st, device=dev)
+        self.d_V = torch.empty_like(self.d_K)
+        self.d_BK = torch.empty(B, D, cfg.rank_k, dtype=st, device=dev)
+        self.d_BV = torch.empty(B, D, cfg.rank_v, dtype=st, device=dev)
+        self.d_q = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=st, device=dev)
+        self.K, self.V = [None] * B, [None] * B            # sink rows only (the oracle needs nothing else of them)
+        self.q, self.BK, self.BV, self.CK, self.CV = ([None] * B for _ in range(5))
+        for b in range(B):
+            self.d_K[b] = W.make_kv(cfg, 0, b, "k", device=dev)
+            self.d_V[b] = W.make_kv(cfg, 0, b, "v", device=dev)
+            q = W.make_query(cfg, self.d_K[b], 0, b)
+            self.d_q[b] = q
+            rows_k = self.d_K[b][W.sample_rows(cfg, 0, b, "k").to(dev)]
+            rows_v = self.d_V[b][W.sample_rows(cfg, 0, b, "v").to(dev)]
+            if b in self.checked:
+                bk = O.round_to_storage(O.build_basis(to_np(rows_k), cfg.rank_k)[0], cfg.dtype)
+                bv = O.round_to_storage(O.build_basis(to_np(rows_v), cfg.rank_v)[0], cfg.dtype)
+                self.BK[b], self.BV[b], self.q[b] = bk, bv, to_np(q)
+                self.d_BK[b], self.d_BV[b] = from_np(bk, st, dev), from_np(bv, st, dev)
+                self.K[b], self.V[b] = self.d_K[b, :s].cpu(), self.d_V[b, :s].cpu()
+            else:
+                self.d_BK[b] = W.make_bench_basis(rows_k, cfg.rank_k, st)
+                self.d_BV[b] = W.make_bench_basis(rows_v, cfg.rank_v, st)
+        self.d_sink_k = torch.zeros(B, s, D, dtype=st, device=dev)
+        self.d_sink_v = torch.zeros_like(self.d_sink_k)
+        self.d_CK = torch.zeros(B, self.cap, cfg.rank_k, dtype=st, device=dev)
+        self.d_CV = torch.zeros(B, self.cap, cfg.rank_v, dtype=st, device=dev)
+        self.d_len = torch.zeros(B, dtype=torch.int32, device=dev)
+        ly = self.layer_desc()
+        ws = s4r.alloc_workspace(ly, self.cap, cfg.window, cfg.top_k)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        s4r.compress(ly, self.d_K, self.d_V, self.d_BK, self.d_BV, self.d_sink_k, self.d_sink_v, self.d_CK, self.d_CV,
+                     self.d_len, workspace=ws, dev_status=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        assert self.d_len.tolist() == [self.L] * B
+        assert torch.equal(self.d_sink_k, self.d_K[:, :s]) and torch.equal(self.d_sink_v, self.d_V[:, :s])
+
+    def layer_desc(self):
+        import paper_2608_00528_b200 as s4r
+        cfg = self.cfg
+        return s4r.Layer(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rank_k, cfg.rank_v,
+                         cfg.sink_count, s4r.S4R_BF16, self.cap)
+
+    def check_compress_and_adopt_oracle_coefficients(self, n_rows_abs=4096):
+        """Oracle compress of the checked sequences; library coefficients must agree to one bf16 ulp plus the
+        fp32 accumulation error; afterwards those sequences' cache rows hold the oracle's coefficients."""
+        cfg, s = self.cfg, self.cfg.sink_count
+        rng = np.random.default_rng(1234)
+        for b in self.checked:
+            for name, d_x, basis, d_c, store in (("k", self.d_K, self.BK, self.d_CK, self.CK),
+                                                 ("v", self.d_V, self.BV, self.d_CV, self.CV)):
+                x = to_np(d_x[b, s:])
+                want = O.round_to_storage(x @ basis[b], cfg.dtype)
+                got = to_np(d_c[b, :self.L])
+                rows = np.sort(rng.choice(self.L, n_rows_abs, replace=False))
+                absdot = np.abs(x[rows]) @ np.abs(basis[b])
+                tol_rows = O.storage_ulp(want[rows], "bf16") * 1.0001 + 2.0 ** -18 * absdot
+                assert (np.abs(got[rows] - want[rows]) <= tol_rows).all(), f"seq {b} {name}: compress mismatch"
+                # every row: equal, or off by one grid step of the larger neighbour
+                assert (np.abs(got - want) <= 2 * O.storage_ulp(np.maximum(np.abs(want), np.abs(got)), "bf16")
+                        + 1e-4 * np.abs(want).max()).all()
+                assert (got != want).mean() < 0.02
+                store[b] = want
+                d_c[b, :self.L] = from_np(want, self.st, self.device)
+                del x, got
+
+
+def _properties(p, out, sel, cnt, b, W_, k):
+    """Checks that need no oracle: count, range, uniqueness, order, local window, finite output."""
+    L = p.L
+    n = int(cnt[b])
+    W_eff, k_eff = min(W_, L), min(k, L - min(W_, L))
+    assert n == W_eff + k_eff
+    idx = sel[b, :n].cpu().numpy()
+    assert (sel[b, n:] == -1).all()
+    assert idx.min() >= 0 and idx.max() < L and np.unique(idx).size == n
+    assert np.all(np.diff(idx[:k_eff]) > 0) and idx[:k_eff].max() < L - W_eff
+    assert np.array_equal(idx[k_eff:], np.arange(L - W_eff, L))
+    assert torch.isfinite(out[b]).all()
+
+
+@pytest.mark.parametrize("ci,checked", [(2, (0, 7)), (3, (1, 3))])
+def test_full_size_config(ci, checked):
+    cfg = W.get_config(ci)
+    p = FullSizeProblem(cfg, checked)
+    p.check_compress_and_adopt_oracle_coefficients()
+    del p.d_K, p.d_V
+    torch.cuda.empty_cache()
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status == 0
+    worst = check_step(p, out, sel, cnt, seqs=list(checked))
+    print(f"{cfg.name}: sequences {checked} selection ok, max rel output error {worst:.3e}")
+    for b in range(cfg.batch):
+        _properties(p, out, sel, cnt, b, cfg.window, cfg.top_k)
+    out2, sel2, cnt2, _ = run_gpu_step(p)
+    assert torch.equal(sel, sel2) and torch.equal(out, out2)          # run-to-run bitwise determinism

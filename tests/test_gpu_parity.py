@@ -228,3 +228,38 @@ def test_append_matches_oracle_and_respects_capacity():
                 _check_coefficients(p.d_CV[b, p.L + step][None], want[None], "bf16", _absdot(vt[b][None], p.BV[b]))
         else:
             assert status.item() & s4r.DEV_BOUNDS and p.d_len.tolist() == [p.L + 2] * 2
+
+
+def test_multi_layer_multi_step_generation_with_append():
+    """Config 4's flow at reduced size: per layer compress once, then per step append the new token and decode.
+    The oracle keeps its own caches; after each append the library's new row is checked against the oracle's
+    and replaced by it, so every decode comparison runs on identical inputs."""
+    s4r = _s4r()
+    cfg = _cfg(4, context=3000 + 17, batch=2, n_layers=2, decode_steps=5, top_k=256)
+    steps = cfg.decode_steps
+    for layer in range(cfg.n_layers):
+        p = Problem(cfg, layer=layer, device="cuda", capacity=cfg.cache_len + steps).upload()
+        ly = p.layer_desc()
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for step in range(1, steps + 1):
+            kt = torch.stack([W.make_token(cfg, layer, b, "k", step, "cuda") for b in range(cfg.batch)])
+            vt = torch.stack([W.make_token(cfg, layer, b, "v", step, "cuda") for b in range(cfg.batch)])
+            s4r.append(ly, kt, vt, p.d_BK, p.d_BV, p.d_CK, p.d_CV, p.d_len, dev_status=status)
+            torch.cuda.synchronize()
+            L = p.L + step
+            assert status.item() == 0 and p.d_len.tolist() == [L] * cfg.batch
+            for b in range(cfg.batch):
+                ck = O.project_token(to_np(kt[b]), p.BK[b], "bf16")
+                cv = O.project_token(to_np(vt[b]), p.BV[b], "bf16")
+                _check_coefficients(p.d_CK[b, L - 1][None], ck[None], "bf16", _absdot(kt[b][None], p.BK[b]))
+                _check_coefficients(p.d_CV[b, L - 1][None], cv[None], "bf16", _absdot(vt[b][None], p.BV[b]))
+                p.CK[b] = np.concatenate([p.CK[b], ck[None]])
+                p.CV[b] = np.concatenate([p.CV[b], cv[None]])
+                p.d_CK[b, L - 1] = from_np(ck, p.st, "cuda")
+                p.d_CV[b, L - 1] = from_np(cv, p.st, "cuda")
+                q = W.make_query(cfg, p.K[b], layer, b, step=step)
+                p.q[b] = to_np(q)
+                p.d_q[b] = q.cuda()
+            out, sel, cnt, st = run_gpu_step(p)
+            assert st == 0
+            check_step(p, out, sel, cnt, L=L)
