@@ -2,9 +2,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
 
-One "step" = one pass of the decode path for one layer over the whole batch: the cache update (s4r_append)
-followed by s4r_decode_step (query projection, latent scoring, relevance, selection, sparse reconstruction,
-attention).  The prefill projection (s4r_compress) builds the cache during set-up and is timed separately
+One "step" = one pass of the decode path for one layer over the whole batch through
+s4r_append_decode_step: the cache update (new key/value rows projected and appended), query projection,
+latent scoring, relevance, selection, sparse reconstruction and attention.  The prefill projection (s4r_compress) builds the cache during set-up and is timed separately
 (`compress` in the JSON line).  Workload: the 128K-context Llama-3.1-8B-shaped layer with batch 8 on which the
 headline metric is quoted (coefficients 0.8 GB, far larger than L2, so nothing is carried between steps).
 With N > 1 every rank runs its own batch of sequences (weak scaling, no collective on the data path).
@@ -238,10 +238,8 @@ def main():
 
     def step(i):
         j = i % pool
-        s4r.append(ly, kt[j], vt[j], c["BK"], c["BV"], c["CK"], c["CV"], c["len"], dev_status=status)
-        launches[0] += s4r.last_launch_count()
-        s4r.decode_step(ly, qs[j], c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"], capacity,
-                        cfg.window, cfg.top_k, out, sel, cnt, c["ws"], **kw)
+        s4r.append_decode_step(ly, kt[j], vt[j], qs[j], c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"],
+                               c["BV"], capacity, cfg.window, cfg.top_k, out, sel, cnt, c["ws"], **kw)
         launches[0] += s4r.last_launch_count()
 
     def barrier():
@@ -340,7 +338,7 @@ def main():
         "config": {"workload": cfg.name, "batch_per_gpu": B, "global_batch": B * world, "context": cfg.context,
                    "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
                    "rank": cfg.rank_k, "window": cfg.window, "top_k": cfg.top_k, "sinks": cfg.sink_count,
-                   "rope_theta": cfg.rope_theta, "step": "s4r_append + s4r_decode_step",
+                   "rope_theta": cfg.rope_theta, "step": "s4r_append_decode_step (cache update + decode step)",
                    "l2": "inputs larger than L2 (key coefficients %.0f MB per step)" % (scan_bytes / 1e6),
                    "parallelism": f"dp{world} (independent sequences, no collective)"},
         "roofline": {"bound": "hbm", "kernel": "latent_scoring", "achieved": achieved, "peak": peak, "unit": "GB/s",

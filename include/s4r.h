@@ -148,6 +148,17 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
                     int32_t *sel_idx, int32_t *sel_count, void *workspace, size_t workspace_bytes,
                     int32_t *dev_status, void *stream);
 
+/* s4r_append followed by s4r_decode_step as one call (Sec. 3.2.1 then 3.2.2-3.2.3): the new token's key and
+ * value rows are projected in the same pass over the bases that projects the query (Eq. 5), appended
+ * (Eq. 6), and the step then runs on the grown cache.  Results are bit-identical to the two separate calls.
+ * k_t, v_t [B, D'] pre-RoPE; coef_k, coef_v, coef_len are updated; max_len must bound coef_len[b] + 1. */
+int s4r_append_decode_step(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,
+                           const void *sink_k, const void *sink_v, void *coef_k, void *coef_v, int32_t *coef_len,
+                           const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                           int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out,
+                           int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
+                           size_t workspace_bytes, int32_t *dev_status, void *stream);
+
 /* Same step for callers whose per-step data lives in HOST memory: q_host, out_host, sel_idx_host and
  * sel_count_host are host buffers (pinned memory makes the copies asynchronous); q_dev, out_dev,
  * sel_idx_dev, sel_count_dev are device staging buffers of the same shapes.  The call copies q to the

@@ -20,7 +20,7 @@ GROUP_MEAN, GROUP_MAX = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_compress", "s4r_append", "s4r_decode_step", "s4r_decode_step_host",
-           "s4r_decode_step_static",
+           "s4r_decode_step_static", "s4r_append_decode_step",
            "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
            "s4r_stage_times", "s4r_strerror", "s4r_version")
 STAGES = ("query_projection", "latent_scoring", "selection", "reconstruct_attend", "merge")
@@ -291,3 +291,25 @@ def _static_fn():
         fn.argtypes = [ctypes.POINTER(_Layer), vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, ctypes.POINTER(_Score),
                        ctypes.POINTER(_Rope), vp, i32, vp, vp, vp, vp]
     return fn
+
+
+def append_decode_step(layer: Layer, k_t, v_t, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,
+                       max_len: int, window: int, top_k: int, out, sel_idx, sel_count, workspace, *,
+                       pool_kernel: int = 7, pool_mode: int = POOL_MAX, group_mode: int = GROUP_MEAN,
+                       score_window: int = 1, rope_theta: float = 0.0, dev_status=None, stream=None):
+    """s4r_append_decode_step: append the new token's coefficient rows and run the decode step in one call."""
+    _need_cuda(k_t, v_t, q, coef_k, coef_v, coef_len, key_basis, value_basis, out, sel_idx, sel_count, workspace)
+    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, score_window, rope_theta)
+    out_dtype = S4R_BF16 if out.dtype == torch.bfloat16 else S4R_F32
+    fn = load().s4r_append_decode_step
+    if not fn.argtypes:
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        fn.restype = ctypes.c_int
+        fn.argtypes = [ctypes.POINTER(_Layer), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32,
+                       ctypes.POINTER(_Score), ctypes.POINTER(_Rope), vp, i32, vp, vp, vp, ctypes.c_size_t, vp, vp]
+    rc = fn(ctypes.byref(layer.c()), _ptr(k_t), _ptr(v_t), _ptr(q), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k),
+            _ptr(coef_v), _ptr(coef_len), _ptr(key_basis), _ptr(value_basis), int(max_len), int(window), int(top_k),
+            ctypes.byref(sc), ctypes.byref(rp), _ptr(out), out_dtype, _ptr(sel_idx), _ptr(sel_count), _ptr(workspace),
+            workspace.numel(), _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_append_decode_step")

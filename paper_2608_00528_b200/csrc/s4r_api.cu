@@ -44,7 +44,7 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   size_t off = 0;
   p->n_parts = p->n_scan_chunks;
   p->parts_cap = p->n_scan_chunks > kMaxParts ? p->n_scan_chunks : kMaxParts;
-  p->off_cq = off;      off = align_up(off + sizeof(float) * ly.B * kQSlices * ly.G * ly.rk, 256);
+  p->off_cq = off;      off = align_up(off + sizeof(float) * ly.B * ly.G * ly.rk, 256);
   p->off_z = off;       off = align_up(off + sizeof(float) * ly.B * ly.G * p->z_stride, 256);
   p->off_part = off;    off = align_up(off + sizeof(float2) * ly.B * p->parts_cap * kMaxGroup, 256);
   p->off_score = off;   off = align_up(off + sizeof(float) * ly.B * p->z_stride, 256);
@@ -151,12 +151,12 @@ int s4r_append(const s4r_layer_t *layer, const void *k_t, const void *v_t, const
   return S4R_OK;
 }
 
-int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
-                    const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,
-                    const void *value_basis, int64_t max_len, int32_t window, int32_t top_k,
-                    const s4r_score_t *score, const s4r_rope_t *rope, void *out, int32_t out_dtype,
-                    int32_t *sel_idx, int32_t *sel_count, void *workspace, size_t workspace_bytes,
-                    int32_t *dev_status, void *stream) {
+static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,
+                       const void *sink_k, const void *sink_v, const void *coef_k, const void *coef_v,
+                       const int32_t *coef_len, const void *key_basis, const void *value_basis, int64_t max_len,
+                       int32_t window, int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out,
+                       int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
+                       size_t workspace_bytes, int32_t *dev_status, void *stream) {
   launch_counter() = 0;
   StepArgs a;
   if (!layer_ok(layer, &a.ly)) return S4R_ERR_INVALID_ARG;
@@ -186,6 +186,11 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
   a.pool_mode = sc.pool_mode; a.group_mode = sc.group_mode; a.theta = rope ? rope->theta : 0.f; a.out = out;
   a.out_dtype = out_dtype; a.sel_idx = sel_idx; a.sel_count = sel_count; a.ws = (char *)workspace;
   a.dev_status = dev_status; a.stream = (cudaStream_t)stream;
+  if (k_t) {
+    a.k_t = k_t; a.v_t = v_t;
+    a.coef_k_w = const_cast<void *>(coef_k); a.coef_v_w = const_cast<void *>(coef_v);
+    a.coef_len_w = const_cast<int32_t *>(coef_len);
+  }
   bool fast_scan = scan_fast_supported(ly);
   if (fast_scan) {
     const int parts = scan_fast_parts(ly);
@@ -212,6 +217,29 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
   if (launch_merge(a) != cudaSuccess) return S4R_ERR_CUDA;
   stage_mark(5, a.stream);
   return S4R_OK;
+}
+
+int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
+                    const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,
+                    const void *value_basis, int64_t max_len, int32_t window, int32_t top_k,
+                    const s4r_score_t *score, const s4r_rope_t *rope, void *out, int32_t out_dtype,
+                    int32_t *sel_idx, int32_t *sel_count, void *workspace, size_t workspace_bytes,
+                    int32_t *dev_status, void *stream) {
+  return decode_impl(layer, nullptr, nullptr, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,
+                     max_len, window, top_k, score, rope, out, out_dtype, sel_idx, sel_count, workspace,
+                     workspace_bytes, dev_status, stream);
+}
+
+int s4r_append_decode_step(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,
+                           const void *sink_k, const void *sink_v, void *coef_k, void *coef_v, int32_t *coef_len,
+                           const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                           int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out,
+                           int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
+                           size_t workspace_bytes, int32_t *dev_status, void *stream) {
+  if (!k_t || !v_t) return S4R_ERR_INVALID_ARG;
+  return decode_impl(layer, k_t, v_t, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis, max_len,
+                     window, top_k, score, rope, out, out_dtype, sel_idx, sel_count, workspace, workspace_bytes,
+                     dev_status, stream);
 }
 
 int s4r_decode_step_host(const s4r_layer_t *layer, const void *q_host, void *q_dev, const void *sink_k,

@@ -7,11 +7,12 @@
 //   V^^T[d_h x tokens] = (B^V slice) C^V[rows]^T      (tcgen05.mma, A = basis slice, B = gathered rows)
 // with the basis slices streamed through a TMA ring in 64-column blocks and the fp32 results held in tensor
 // memory (2 x 2 accumulators of 128 columns, so the tensor pipe runs one head ahead of the epilogue).
-// The epilogue warps read K^ row-per-thread, apply RoPE from a per-tile sin/cos table, form the logits of
-// the G query heads in fp32, take the tile softmax, then read V^^T channel-per-thread and accumulate
-// P.V^ - both contractions are thread-local, so no reconstructed value is ever written anywhere.
-// Per (head, tile) the CTA emits flash-style partials (max, sum, unnormalised output); k_merge joins them
-// with the sinks.  Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-9 = epilogue.
+// Sixteen epilogue warps read K^ row-per-thread (four warps share a row quadrant and split its columns),
+// apply RoPE from a per-tile sin/cos table, form the logits of the G query heads in fp32 (packed fp32x2
+// FMAs), take the tile softmax, then read V^^T channel-per-thread and accumulate P.V^ - both contractions are
+// thread-local up to a small exchange through shared memory, so no reconstructed value is ever written
+// anywhere.  Per (head, tile) the CTA emits flash-style partials (max, sum, unnormalised output); k_merge
+// joins them with the sinks.  Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-17 = epilogue.
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
 
@@ -19,13 +20,16 @@ namespace s4r {
 
 using namespace sm100;
 
+void fill_inv_freq(double *dst, int head_dim, float theta);
+
 namespace {
 
 constexpr int kTok = 128;          // selected rows per tile
 constexpr int kDh = 128;           // head dimension of the fast path
 constexpr int kRing = 3;           // basis blocks in flight
 constexpr int kBlkBytes = 128 * 128;  // one [128 x 64] bf16 block
-constexpr int kEpiThreads = 256;
+constexpr int kEpiWarps = 16;
+constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kThreads = 64 + kEpiThreads;
 
 struct AttFastParams {
@@ -37,24 +41,33 @@ struct AttFastParams {
   int64_t cap, max_len;
   float theta;
   int32_t *dev_status;
+  double inv_freq[64];
 };
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
+__device__ __forceinline__ float2 bcast2(float v) { return make_float2(v, v); }
+
+// 16-byte asynchronous copy global -> shared; copies zeros instead when `valid` is false
+__device__ __forceinline__ void cp_async16_zfill(void *dst, const void *src, bool valid) {
+  const int n = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(n) : "memory");
+}
+
 __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_constant__ CUtensorMap tmap_bk,
                                                               const __grid_constant__ CUtensorMap tmap_bv,
-                                                              AttFastParams p) {
+                                                              const __grid_constant__ AttFastParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const int kbk = p.rk >> 6, kbv = p.rv >> 6;
+  const int kbk = p.rk >> 6, kbv = p.rv >> 6, G = p.G;
   uint8_t *ck = smem;                                   // [kbk][128 tokens][128 B]
   uint8_t *cv = ck + (size_t)kbk * kBlkBytes;           // [kbv][128 tokens][128 B]
   uint8_t *ring = cv + (size_t)kbv * kBlkBytes;         // [kRing][128 d][128 B]
   float2 *sc = reinterpret_cast<float2 *>(ring + (size_t)kRing * kBlkBytes);   // [64 pairs][128 tokens] (sin, cos)
   float *qs = reinterpret_cast<float *>(sc + 64 * kTok);                       // [128 cols][8]
   float *ps = qs + kDh * kMaxGroup;                                            // [128 tokens][8] probabilities
-  float *xch = ps + kTok * kMaxGroup;                                          // [2 halves][8][128] exchange
-  uint64_t *bars = reinterpret_cast<uint64_t *>(xch + 2 * kMaxGroup * 128);
+  float *xch = ps + kTok * kMaxGroup;                                          // [4 quarters][G][128] exchange
+  uint64_t *bars = reinterpret_cast<uint64_t *>(xch + 4 * G * 128);
   uint64_t *full = bars, *empty = bars + kRing;
   uint64_t *k_full = bars + 2 * kRing, *k_empty = k_full + 2, *v_full = k_empty + 2, *v_empty = v_full + 2;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(v_empty + 2);
@@ -78,8 +91,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
     for (int i = 0; i < 2; ++i) {
       mbar_init(&k_full[i], 1);
       mbar_init(&v_full[i], 1);
-      mbar_init(&k_empty[i], kEpiThreads);
-      mbar_init(&v_empty[i], kEpiThreads);
+      mbar_init(&k_empty[i], kEpiWarps);  // one arrival per epilogue warp
+      mbar_init(&v_empty[i], kEpiWarps);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -91,42 +104,46 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
     int rix = (tid < nt) ? p.sel_idx[(size_t)b * p.sel_stride + t0 + tid] : -1;
     rows[tid] = rix < 0 ? -1 : min(rix, max(L - 1, 0));
   }
-  double *inv_freq = reinterpret_cast<double *>(xch);  // [64], only needed while the sin/cos table is built
-  if (tid >= 128 && tid < 192 && p.theta > 0.f) inv_freq[tid - 128] = rope_inv_freq(tid - 128, kDh, p.theta);
-  __syncthreads();
-
-  // ---- gather the selected coefficient rows into swizzled K-major tiles (zero rows past the tile's end)
-  {
-    const int cpr_k = p.rk >> 3, cpr_v = p.rv >> 3;  // 16-byte chunks per row
-    const uint4 zero = make_uint4(0, 0, 0, 0);
-    const __nv_bfloat16 *ckb = p.coef_k + (size_t)b * p.cap * p.rk;
-    const __nv_bfloat16 *cvb = p.coef_v + (size_t)b * p.cap * p.rv;
-    for (int i = tid; i < kTok * cpr_k; i += kThreads) {
-      const int t = i / cpr_k, c = i - t * cpr_k, rix = rows[t];
-      const uint4 v = rix >= 0 ? __ldg(reinterpret_cast<const uint4 *>(ckb + (size_t)rix * p.rk) + c) : zero;
-      *reinterpret_cast<uint4 *>(ck + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8)) = v;
-    }
-    for (int i = tid; i < kTok * cpr_v; i += kThreads) {
-      const int t = i / cpr_v, c = i - t * cpr_v, rix = rows[t];
-      const uint4 v = rix >= 0 ? __ldg(reinterpret_cast<const uint4 *>(cvb + (size_t)rix * p.rv) + c) : zero;
-      *reinterpret_cast<uint4 *>(cv + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8)) = v;
-    }
-    // sin / cos of every (pair, token) of the tile at the token's original position s + row
-    if (p.theta > 0.f) {
-      for (int i = tid; i < 64 * kTok; i += kThreads) {
-        const int pair = i >> 7, t = i & (kTok - 1);
-        float sn = 0.f, cs = 1.f;
-        if (rows[t] >= 0) rope_sincos(p.s + rows[t], inv_freq[pair], sn, cs);
-        sc[i] = make_float2(sn, cs);
-      }
-    }
-  }
-  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int blocks_per_kv = kbk + kbv;
+
+  if (warp != 0) {
+    // ---- all warps but the producer gather the selected coefficient rows into swizzled K-major tiles while
+    //      the producer already fills the ring with basis blocks
+    // asynchronous 16-byte copies: every row piece is in flight at once (the rows are scattered over the
+    // cache, so each piece is a DRAM round trip); pieces of rows past the tile's end are zero-filled
+    constexpr int kWorkers = kThreads - 32;
+    const int wt = tid - 32;
+    const int cpr_k = p.rk >> 3, cpr_v = p.rv >> 3;  // 16-byte chunks per row
+    const __nv_bfloat16 *ckb = p.coef_k + (size_t)b * p.cap * p.rk;
+    const __nv_bfloat16 *cvb = p.coef_v + (size_t)b * p.cap * p.rv;
+    for (int i = wt; i < kTok * cpr_k; i += kWorkers) {
+      const int t = i / cpr_k, c = i - t * cpr_k, rix = rows[t];
+      cp_async16_zfill(ck + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8),
+                       reinterpret_cast<const uint4 *>(ckb + (size_t)max(rix, 0) * p.rk) + c, rix >= 0);
+    }
+    for (int i = wt; i < kTok * cpr_v; i += kWorkers) {
+      const int t = i / cpr_v, c = i - t * cpr_v, rix = rows[t];
+      cp_async16_zfill(cv + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8),
+                       reinterpret_cast<const uint4 *>(cvb + (size_t)max(rix, 0) * p.rv) + c, rix >= 0);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    // sin / cos of every (pair, token) of the tile at the token's original position s + row
+    if (p.theta > 0.f) {
+      for (int i = wt; i < 64 * kTok; i += kWorkers) {
+        const int pair = i >> 7, t = i & (kTok - 1);
+        float sn = 0.f, cs = 1.f;
+        if (rows[t] >= 0) rope_sincos(p.s + rows[t], p.inv_freq[pair], sn, cs);
+        sc[i] = make_float2(sn, cs);
+      }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    fence_proxy_async_smem();
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads - 32) : "memory");  // tiles and table complete (producer not involved)
+  }
 
   if (warp == 0) {
     // ---------------- TMA producer: basis slices, 64-column blocks, K blocks then V blocks per head ----------------
@@ -200,16 +217,17 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
       }
     }
   } else {
-    // ---------------- epilogue: 8 warps; warps e and e+4 share a TMEM lane quadrant and split the columns ----------------
+    // ---------------- epilogue: 16 warps; warps e, e+4, e+8, e+12 share a TMEM lane quadrant and split the columns --------
     const int e = warp - 2, et = tid - 64;   // epilogue warp / thread index
-    const int quad = warp & 3, half = e >> 2;
-    const int lane_row = quad * 32 + lane;  // token (K^) or channel (V^^T) owned by this thread
+    const int quad = warp & 3, qt = e >> 2;  // lane quadrant, column quarter
+    const int lane_row = quad * 32 + lane;   // token (K^) or channel (V^^T) owned by this thread
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const int G = p.G;
-    // RoPE of the query: this thread prepares column qc of q' for the heads g = qg0, qg0+2, ...
+    const int npair = (G + 1) >> 1;          // heads are processed in pairs (packed fp32x2 arithmetic)
+    const bool rope = p.theta > 0.f;
+    // RoPE of the query: this thread prepares column qc of q' for the heads g = qg0, qg0 + 4
     const int qc = et & 127, qg0 = et >> 7;
     float q_sn = 0.f, q_cs = 1.f;
-    if (p.theta > 0.f) rope_sincos(p.s + L - 1, rope_inv_freq(qc & 63, kDh, p.theta), q_sn, q_cs);
+    if (rope) rope_sincos(p.s + L - 1, p.inv_freq[qc & 63], q_sn, q_cs);
     const float q_scale = rsqrtf((float)kDh);
     // `ok` stays warp-uniform; after a failed wait the loop keeps its shape (every epi_sync is still reached)
     // but touches tensor memory no more
@@ -217,61 +235,63 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
     for (int h = 0; h < p.nkv; ++h) {
       const int kv = kv0 + h, buf = h & 1;
       const uint32_t aph = (uint32_t)(h >> 1) & 1u;
-      // q' = RoPE(q) / sqrt(d_h) for the G heads of this KV head, laid out [col][g]
-      for (int g = qg0; g < G; g += 2) {
-        const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)kv * G + g) * kDh;
-        float v = __bfloat162float(qp[qc]);
-        if (p.theta > 0.f) {
-          const float o = __bfloat162float(qp[qc ^ 64]);
-          v = (qc < 64) ? v * q_cs - o * q_sn : v * q_cs + o * q_sn;
+      // q' = RoPE(q) / sqrt(d_h) for the G heads of this KV head, laid out [col][g] (unused heads are zero)
+      for (int g = qg0; g < kMaxGroup; g += 4) {
+        float v = 0.f;
+        if (g < G) {
+          const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)kv * G + g) * kDh;
+          v = __bfloat162float(qp[qc]);
+          if (rope) {
+            const float o = __bfloat162float(qp[qc ^ 64]);
+            v = (qc < 64) ? v * q_cs - o * q_sn : v * q_cs + o * q_sn;
+          }
         }
         qs[qc * kMaxGroup + g] = v * q_scale;
       }
       epi_sync();
-      // ---- K^ row of this thread's token: columns [32*half, +32) and their RoPE partners 64 further
+      // ---- K^ row of this thread's token: pairs [16*qt, +16), i.e. columns 16*qt.. and their partners 64 further
       if (ok) ok = mbar_wait(&k_full[buf], aph, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
-      float lg[kMaxGroup];
+      float2 lg[4];
 #pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g) lg[g] = 0.f;
+      for (int gp = 0; gp < 4; ++gp) lg[gp] = make_float2(0.f, 0.f);
       if (ok) {
-        uint32_t ka[32], kb[32];
-        const uint32_t base = tmem_base + (uint32_t)buf * 128 + lane_addr + (uint32_t)half * 32;
-        tmem_ld32(base, ka);
-        tmem_ld32(base + 64, kb);
+        uint32_t ka[16], kb[16];
+        const uint32_t base = tmem_base + (uint32_t)buf * 128 + lane_addr + (uint32_t)qt * 16;
+        tmem_ld16(base, ka);
+        tmem_ld16(base + 64, kb);
         tmem_ld_wait();
         tc_fence_before();
-        mbar_arrive(&k_empty[buf]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&k_empty[buf]);
 #pragma unroll
-        for (int ii = 0; ii < 32; ++ii) {
-          const int i = half * 32 + ii;
-          float k1 = __uint_as_float(ka[ii]), k2 = __uint_as_float(kb[ii]);
-          if (p.theta > 0.f) {
-            const float2 t = sc[i * kTok + lane_row];
-            const float r1 = k1 * t.y - k2 * t.x, r2 = k2 * t.y + k1 * t.x;
-            k1 = r1;
-            k2 = r2;
+        for (int ii = 0; ii < 16; ++ii) {
+          const int i = qt * 16 + ii;
+          float2 k12 = make_float2(__uint_as_float(ka[ii]), __uint_as_float(kb[ii]));
+          if (rope) {
+            const float2 t = sc[i * kTok + lane_row];  // (sin, cos)
+            // (k1 c - k2 s, k2 c + k1 s)
+            k12 = __ffma2_rn(make_float2(-k12.y, k12.x), bcast2(t.x), __fmul2_rn(k12, bcast2(t.y)));
           }
+          const float2 k1 = bcast2(k12.x), k2 = bcast2(k12.y);
           const float4 qa = *reinterpret_cast<const float4 *>(qs + i * kMaxGroup);
           const float4 qb = *reinterpret_cast<const float4 *>(qs + (i + 64) * kMaxGroup);
-          lg[0] = fmaf(qa.x, k1, fmaf(qb.x, k2, lg[0]));
-          lg[1] = fmaf(qa.y, k1, fmaf(qb.y, k2, lg[1]));
-          lg[2] = fmaf(qa.z, k1, fmaf(qb.z, k2, lg[2]));
-          lg[3] = fmaf(qa.w, k1, fmaf(qb.w, k2, lg[3]));
-          if (G > 4) {
+          lg[0] = __ffma2_rn(make_float2(qa.x, qa.y), k1, __ffma2_rn(make_float2(qb.x, qb.y), k2, lg[0]));
+          lg[1] = __ffma2_rn(make_float2(qa.z, qa.w), k1, __ffma2_rn(make_float2(qb.z, qb.w), k2, lg[1]));
+          if (npair > 2) {
             const float4 qc4 = *reinterpret_cast<const float4 *>(qs + i * kMaxGroup + 4);
             const float4 qd4 = *reinterpret_cast<const float4 *>(qs + (i + 64) * kMaxGroup + 4);
-            lg[4] = fmaf(qc4.x, k1, fmaf(qd4.x, k2, lg[4]));
-            lg[5] = fmaf(qc4.y, k1, fmaf(qd4.y, k2, lg[5]));
-            lg[6] = fmaf(qc4.z, k1, fmaf(qd4.z, k2, lg[6]));
-            lg[7] = fmaf(qc4.w, k1, fmaf(qd4.w, k2, lg[7]));
+            lg[2] = __ffma2_rn(make_float2(qc4.x, qc4.y), k1, __ffma2_rn(make_float2(qd4.x, qd4.y), k2, lg[2]));
+            lg[3] = __ffma2_rn(make_float2(qc4.z, qc4.w), k1, __ffma2_rn(make_float2(qd4.z, qd4.w), k2, lg[3]));
           }
         }
       }
 #pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g)
-        if (g < G) xch[(half * kMaxGroup + g) * 128 + lane_row] = lg[g];
+      for (int gp = 0; gp < 4; ++gp) {
+        if (2 * gp < G) xch[(qt * G + 2 * gp) * 128 + lane_row] = lg[gp].x;
+        if (2 * gp + 1 < G) xch[(qt * G + 2 * gp + 1) * 128 + lane_row] = lg[gp].y;
+      }
       epi_sync();
       // ---- tile softmax: epilogue warp e handles head g = e over the 128 tokens
       if (e < G) {
@@ -279,7 +299,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int t = u * 32 + lane;
-          l4[u] = (t < nt) ? xch[e * 128 + t] + xch[(kMaxGroup + e) * 128 + t] : -INFINITY;
+          l4[u] = (t < nt) ? (xch[e * 128 + t] + xch[(G + e) * 128 + t]) + (xch[(2 * G + e) * 128 + t] + xch[(3 * G + e) * 128 + t])
+                           : -INFINITY;
           m = fmaxf(m, l4[u]);
         }
         m = warp_max(m);
@@ -292,53 +313,60 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
         }
         ssum = warp_sum(ssum);
         if (lane == 0) p.part_ms[((size_t)b * p.Hq + (size_t)kv * G + e) * p.n_tiles + tile] = make_float2(m, ssum);
+      } else if (e < kMaxGroup) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) ps[(u * 32 + lane) * kMaxGroup + e] = 0.f;  // unused heads: keep the packed math finite
       }
       epi_sync();
-      // ---- V^^T row of this thread's channel: tokens [64*half, +64)
+      // ---- V^^T row of this thread's channel: tokens [32*qt, +32)
       if (ok) ok = mbar_wait(&v_full[buf], aph, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
-      float o[kMaxGroup];
+      float2 o[4];
 #pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g) o[g] = 0.f;
+      for (int gp = 0; gp < 4; ++gp) o[gp] = make_float2(0.f, 0.f);
       if (ok) {
-        uint32_t va[32], vb[32];
-        const uint32_t base = tmem_base + 256u + (uint32_t)buf * 128 + lane_addr + (uint32_t)half * 64;
-        tmem_ld32(base, va);
-        tmem_ld32(base + 32, vb);
+        uint32_t va[32];
+        tmem_ld32(tmem_base + 256u + (uint32_t)buf * 128 + lane_addr + (uint32_t)qt * 32, va);
         tmem_ld_wait();
         tc_fence_before();
-        mbar_arrive(&v_empty[buf]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&v_empty[buf]);
 #pragma unroll
-        for (int ii = 0; ii < 64; ++ii) {
-          const float v = __uint_as_float(ii < 32 ? va[ii & 31] : vb[ii & 31]);
-          const float *pp = ps + (half * 64 + ii) * kMaxGroup;
+        for (int ii = 0; ii < 32; ++ii) {
+          const float2 v = bcast2(__uint_as_float(va[ii]));
+          const float *pp = ps + (qt * 32 + ii) * kMaxGroup;
           const float4 pa = *reinterpret_cast<const float4 *>(pp);
-          o[0] = fmaf(pa.x, v, o[0]);
-          o[1] = fmaf(pa.y, v, o[1]);
-          o[2] = fmaf(pa.z, v, o[2]);
-          o[3] = fmaf(pa.w, v, o[3]);
-          if (G > 4) {
+          o[0] = __ffma2_rn(make_float2(pa.x, pa.y), v, o[0]);
+          o[1] = __ffma2_rn(make_float2(pa.z, pa.w), v, o[1]);
+          if (npair > 2) {
             const float4 pb = *reinterpret_cast<const float4 *>(pp + 4);
-            o[4] = fmaf(pb.x, v, o[4]);
-            o[5] = fmaf(pb.y, v, o[5]);
-            o[6] = fmaf(pb.z, v, o[6]);
-            o[7] = fmaf(pb.w, v, o[7]);
+            o[2] = __ffma2_rn(make_float2(pb.x, pb.y), v, o[2]);
+            o[3] = __ffma2_rn(make_float2(pb.z, pb.w), v, o[3]);
           }
         }
       }
-      if (half == 1) {
+      if (qt > 0) {
 #pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g)
-          if (g < G) xch[g * 128 + lane_row] = o[g];
+        for (int gp = 0; gp < 4; ++gp) {
+          if (2 * gp < G) xch[((qt - 1) * G + 2 * gp) * 128 + lane_row] = o[gp].x;
+          if (2 * gp + 1 < G) xch[((qt - 1) * G + 2 * gp + 1) * 128 + lane_row] = o[gp].y;
+        }
       }
       epi_sync();
-      if (half == 0) {
+      if (qt == 0) {
 #pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g)
-          if (g < G)
-            p.part_o[(((size_t)b * p.Hq + (size_t)kv * G + g) * p.n_tiles + tile) * kDh + lane_row] =
-                o[g] + xch[g * 128 + lane_row];
+        for (int gp = 0; gp < 4; ++gp) {
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const int g = 2 * gp + hh;
+            if (g < G) {
+              const float mine = hh ? o[gp].y : o[gp].x;
+              p.part_o[(((size_t)b * p.Hq + (size_t)kv * G + g) * p.n_tiles + tile) * kDh + lane_row] =
+                  (mine + xch[g * 128 + lane_row]) + (xch[(G + g) * 128 + lane_row] + xch[(2 * G + g) * 128 + lane_row]);
+            }
+          }
+        }
       }
       epi_sync();  // xch / ps / qs are rewritten by the next head
     }
@@ -386,8 +414,9 @@ cudaError_t launch_attend_sm100(const StepArgs &a) {
   p.max_len = a.plan.max_len;
   p.theta = a.theta;
   p.dev_status = a.dev_status;
+  fill_inv_freq(p.inv_freq, kDh, a.theta);
   const size_t smem = 1024 + (size_t)(ly.rk / 64 + ly.rv / 64 + kRing) * kBlkBytes + sizeof(float2) * 64 * kTok +
-                      sizeof(float) * (kDh * kMaxGroup + kTok * kMaxGroup + 2 * kMaxGroup * 128) + 1024;
+                      sizeof(float) * (kDh * kMaxGroup + kTok * kMaxGroup + 4 * ly.G * 128) + 1024;
   static size_t smem_set = 0;
   if (smem > smem_set) {
     cudaError_t e = cudaFuncSetAttribute(k_attend_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

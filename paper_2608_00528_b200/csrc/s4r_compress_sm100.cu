@@ -24,6 +24,7 @@ constexpr int kCmpThreads = 192;
 struct CompressParams {
   __nv_bfloat16 *coef;
   int B, r, D, s, n_mtiles;
+  int mn_major;  // 1: B operand straight from the basis [D', r] (N contiguous); 0: from the transposed copy [r, D']
   int64_t T, cap;
   int32_t *dev_status;
 };
@@ -68,7 +69,7 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
       mbar_init(&empty[i], 1);
     }
     mbar_init(acc_full, 1);
-    mbar_init(acc_empty, 128);
+    mbar_init(acc_empty, 4);  // one arrival per epilogue warp
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tmap_x);
@@ -95,7 +96,12 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
           mbar_expect_tx(&full[s], 2 * a_bytes + b_bytes);
           tma_load_2d_hint(st, &tmap_x, kb * 64, y0, &full[s], pol);
           tma_load_2d_hint(st + a_bytes, &tmap_x, kb * 64, y0 + 128, &full[s], pol);
-          tma_load_2d(st + 2 * a_bytes, &tmap_bt, kb * 64, b * p.r, &full[s]);
+          if (p.mn_major) {
+            for (int g = 0; g < (p.r >> 6); ++g)  // [64 rows of D' x 64 columns] boxes, one per 64 columns of r
+              tma_load_2d(st + 2 * a_bytes + g * 8192, &tmap_bt, g * 64, b * p.D + kb * 64, &full[s]);
+          } else {
+            tma_load_2d(st + 2 * a_bytes, &tmap_bt, kb * 64, b * p.r, &full[s]);
+          }
           issued = it + 1;
         }
       }
@@ -109,7 +115,8 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(128, p.r);
+      const uint32_t idesc = umma_idesc_bf16(128, p.r) | (p.mn_major ? (1u << 16) : 0u);
+      const uint64_t b_kstep = p.mn_major ? (uint64_t)(2048 >> 4) : (uint64_t)2;  // 16 values of K further
       int it = 0, n_done = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
@@ -120,11 +127,12 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
           if (!mbar_wait(&full[s], (uint32_t)(it / kStages) & 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
-          const uint64_t a0 = umma_desc_sw128(st), a1 = umma_desc_sw128(st + a_bytes), bd = umma_desc_sw128(st + 2 * a_bytes);
+          const uint64_t a0 = umma_desc_sw128(st), a1 = umma_desc_sw128(st + a_bytes);
+          const uint64_t bd = p.mn_major ? umma_desc_mn_sw128(st + 2 * a_bytes, 8192) : umma_desc_sw128(st + 2 * a_bytes);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4) {
-            umma_bf16(tmem_base, a0 + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc, (kb | k4) != 0);
-            umma_bf16(tmem_base + 256u, a1 + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc, (kb | k4) != 0);
+            umma_bf16(tmem_base, a0 + (uint64_t)(k4 * 2), bd + b_kstep * k4, idesc, (kb | k4) != 0);
+            umma_bf16(tmem_base + 256u, a1 + (uint64_t)(k4 * 2), bd + b_kstep * k4, idesc, (kb | k4) != 0);
           }
           umma_commit(&empty[s]);
         }
@@ -170,7 +178,8 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
         }
       }
       tc_fence_before();
-      mbar_arrive(acc_empty);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty);
     }
   }
   tc_fence_before();
@@ -197,16 +206,21 @@ size_t compress_fast_workspace(const Layer &ly) {
 // X: [B, T, D'] rows; basis [B, D', r]; bt: workspace [B, r, D']; coef [B, cap, r]
 cudaError_t launch_compress_sm100(const Layer &ly, const void *X, const void *basis, int r, void *bt, void *coef,
                                   int64_t T, int32_t *dev_status, cudaStream_t st) {
-  dim3 tg((ly.D + 31) / 32, (r + 31) / 32, ly.B);
-  k_transpose_basis<<<tg, 256, 0, st>>>((const __nv_bfloat16 *)basis, (__nv_bfloat16 *)bt, ly.D, r);
-  ++launch_counter();
+  const bool mn_major = (r % 64 == 0);
   CUtensorMap tm_x, tm_bt;
-  if (!make_tmap_bf16_2d(&tm_x, X, (uint64_t)ly.B * (uint64_t)T, (uint64_t)ly.D, 128) ||
-      !make_tmap_bf16_2d(&tm_bt, bt, (uint64_t)ly.B * (uint64_t)r, (uint64_t)ly.D, (uint32_t)r))
-    return cudaErrorInvalidValue;
+  if (!make_tmap_bf16_2d(&tm_x, X, (uint64_t)ly.B * (uint64_t)T, (uint64_t)ly.D, 128)) return cudaErrorInvalidValue;
+  if (mn_major) {
+    if (!make_tmap_bf16_2d(&tm_bt, basis, (uint64_t)ly.B * (uint64_t)ly.D, (uint64_t)r, 64)) return cudaErrorInvalidValue;
+  } else {
+    dim3 tg((ly.D + 31) / 32, (r + 31) / 32, ly.B);
+    k_transpose_basis<<<tg, 256, 0, st>>>((const __nv_bfloat16 *)basis, (__nv_bfloat16 *)bt, ly.D, r);
+    ++launch_counter();
+    if (!make_tmap_bf16_2d(&tm_bt, bt, (uint64_t)ly.B * (uint64_t)r, (uint64_t)ly.D, (uint32_t)r))
+      return cudaErrorInvalidValue;
+  }
   CompressParams p;
   p.coef = (__nv_bfloat16 *)coef;
-  p.B = ly.B; p.r = r; p.D = ly.D; p.s = ly.s;
+  p.B = ly.B; p.r = r; p.D = ly.D; p.s = ly.s; p.mn_major = mn_major ? 1 : 0;
   p.T = T; p.cap = ly.cap;
   p.n_mtiles = (int)((T - ly.s + kMTile - 1) / kMTile);
   p.dev_status = dev_status;

@@ -27,68 +27,6 @@ __device__ inline int clamp_len(const int32_t *coef_len, int b, int64_t max_len,
 }
 
 // ======================================================================================================
-// Query projection (Eq. 5):  cq[b][g][c] = sum_d Qt[g][d] * B^K[b][d][c],  Qt[g][d] = q[b][(d/dh)*G+g][d%dh]
-// grid (ceil(r/32), B, kQSlices): each CTA covers D'/kQSlices rows of the basis and writes a partial
-// cq_part[b][slice][g][c]; readers add the kQSlices partials in slice order (deterministic).
-// block 256 = 32 columns x 8 row groups; row groups are summed in a fixed order.
-// ======================================================================================================
-template <typename T>
-__global__ void __launch_bounds__(256) k_qproj(const T *__restrict__ q, const T *__restrict__ basis,
-                                               float *__restrict__ cq_part, unsigned *__restrict__ hist, int D,
-                                               int r, int G, int dh, int Hq) {
-  extern __shared__ float xs[];  // [G][D / kQSlices]
-  __shared__ float red[8][kMaxGroup][32];
-  const int b = blockIdx.y, slice = blockIdx.z;
-  const int Ds = D / kQSlices, d0 = slice * Ds;
-  if (blockIdx.x == 0 && slice == 0)  // first kernel of the step: clear the score histogram of this sequence
-    for (int i = threadIdx.x; i < 2048; i += 256) hist[(size_t)b * 2048 + i] = 0;
-  const int col = blockIdx.x * 32 + (threadIdx.x & 31);
-  const int rg = threadIdx.x >> 5;
-  for (int i = threadIdx.x; i < G * Ds; i += 256) {
-    int g = i / Ds, d = d0 + (i - g * Ds);
-    xs[i] = Store<T>::ld(q + ((size_t)b * Hq + (size_t)(d / dh) * G + g) * dh + (d % dh));
-  }
-  __syncthreads();
-  float acc[kMaxGroup];
-#pragma unroll
-  for (int g = 0; g < kMaxGroup; ++g) acc[g] = 0.f;
-  if (col < r) {
-    const T *bp = basis + ((size_t)b * D + d0) * r + col;
-    for (int d = rg; d < Ds; d += 8) {
-      float bv = Store<T>::ld(bp + (size_t)d * r);
-#pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g)
-        if (g < G) acc[g] = fmaf(xs[g * Ds + d], bv, acc[g]);
-    }
-  }
-#pragma unroll
-  for (int g = 0; g < kMaxGroup; ++g) red[rg][g][threadIdx.x & 31] = acc[g];
-  __syncthreads();
-  if (rg == 0 && col < r) {
-    for (int g = 0; g < G; ++g) {
-      float s = 0.f;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) s += red[k][g][threadIdx.x & 31];
-      cq_part[(((size_t)b * kQSlices + slice) * G + g) * r + col] = s;
-    }
-  }
-}
-
-template <typename T>
-static cudaError_t qproj_t(const StepArgs &a) {
-  const Layer &ly = a.ly;
-  size_t smem = (size_t)ly.G * (ly.D / kQSlices) * sizeof(float);
-  dim3 grid((ly.rk + 31) / 32, ly.B, kQSlices);
-  k_qproj<T><<<grid, 256, smem, a.stream>>>((const T *)a.q, (const T *)a.basis_k, (float *)(a.ws + a.plan.off_cq),
-                                            (unsigned *)(a.ws + a.plan.off_hist), ly.D, ly.rk, ly.G, ly.dh, ly.Hq);
-  S4R_LAUNCH_CHECK();
-  return cudaSuccess;
-}
-cudaError_t launch_qproj(const StepArgs &a) {
-  return a.ly.dtype == S4R_BF16 ? qproj_t<__nv_bfloat16>(a) : qproj_t<float>(a);
-}
-
-// ======================================================================================================
 // Latent scoring (Eq. 8): Z[b][g][l] = <cq[b][g], C^K[b][l]> / sqrt(r), plus per-chunk softmax partials
 // (max, sum exp) of Eq. 9.  grid (n_chunks, B), block 256; 8 lanes share a row, 4 rows per warp pass.
 // ======================================================================================================
@@ -109,12 +47,7 @@ __global__ void __launch_bounds__(256) k_scan(const T *__restrict__ coef_k, cons
     if (threadIdx.x < G) part[((size_t)b * n_chunks + chunk) * kMaxGroup + threadIdx.x] = make_float2(-INFINITY, 0.f);
     return;
   }
-  for (int i = threadIdx.x; i < G * r; i += 256) {
-    float t = 0.f;
-#pragma unroll
-    for (int sl = 0; sl < kQSlices; ++sl) t += cq[((size_t)b * kQSlices + sl) * G * r + i];
-    cqs[i] = t;
-  }
+  for (int i = threadIdx.x; i < G * r; i += 256) cqs[i] = cq[(size_t)b * G * r + i];
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane & 7, slot = lane >> 3;
   const int nvec = r / V;
@@ -393,77 +326,6 @@ cudaError_t launch_attend_generic(const StepArgs &a) {
   return a.ly.dtype == S4R_BF16 ? attend_t<__nv_bfloat16>(a) : attend_t<float>(a);
 }
 
-// ------------------------------------------------------------------------------------------------------
-// Merge of the tile partials with the sink tokens (Eq. 17-18).  grid (H_q, B), block d_h threads.
-// Sinks are kept in storage precision and handled in fp32 here.
-// ------------------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(256) k_merge(AttParams p) {
-  __shared__ float s_red[8];
-  __shared__ float s_log[64];
-  const int h = blockIdx.x, b = blockIdx.y, i = threadIdx.x, dh = p.dh;
-  const int kv = h / p.G, half = dh >> 1, lane = i & 31, warp = i >> 5, nwarp = dh >> 5;
-  const int L = clamp_len(p.coef_len, b, p.max_len, nullptr);
-  const int count = min(p.sel_count[b], p.sel_stride);
-  const int tiles = (count + p.att_tok - 1) / p.att_tok;
-  const double inv_freq = p.theta > 0.f ? rope_inv_freq(i % half, dh, p.theta) : 0.0;
-  const float qi = rotated_query((const T *)p.q, b, h, i, p.Hq, dh, p.theta, p.s + L - 1, inv_freq);
-  // sink logits
-  for (int j = 0; j < p.s; ++j) {
-    const T *kp = (const T *)p.sink_k + ((size_t)b * p.s + j) * p.D + (size_t)kv * dh;
-    float v = Store<T>::ld(kp + i);
-    if (p.theta > 0.f) {
-      float o = Store<T>::ld(kp + (i < half ? i + half : i - half));
-      float sn, cs;
-      rope_sincos(j, inv_freq, sn, cs);
-      v = (i < half) ? v * cs - o * sn : v * cs + o * sn;
-    }
-    float d = warp_sum(qi * v);
-    if (lane == 0) s_red[warp] = d;
-    __syncthreads();
-    if (i == 0) {
-      float t = 0.f;
-      for (int k = 0; k < nwarp; ++k) t += s_red[k];
-      s_log[j] = t;
-    }
-    __syncthreads();
-  }
-  const float2 *ms = p.part_ms + ((size_t)b * p.Hq + h) * p.n_tiles;
-  const float *po = p.part_o + ((size_t)b * p.Hq + h) * p.n_tiles * dh;
-  float M = -INFINITY;
-  for (int t = 0; t < tiles; ++t) M = fmaxf(M, ms[t].x);
-  for (int j = 0; j < p.s; ++j) M = fmaxf(M, s_log[j]);
-  float den = 0.f, num = 0.f;
-  for (int t = 0; t < tiles; ++t) {
-    float2 v = ms[t];
-    float w = expf(v.x - M);
-    den = fmaf(v.y, w, den);
-    num = fmaf(po[(size_t)t * dh + i], w, num);
-  }
-  for (int j = 0; j < p.s; ++j) {
-    float w = expf(s_log[j] - M);
-    den += w;
-    num = fmaf(Store<T>::ld((const T *)p.sink_v + ((size_t)b * p.s + j) * p.D + (size_t)kv * dh + i), w, num);
-  }
-  const float o = (tiles + p.s > 0 && den > 0.f) ? num / den : 0.f;
-  const size_t oi = ((size_t)b * p.Hq + h) * dh + i;
-  if (p.out_dtype == S4R_F32)
-    ((float *)p.out)[oi] = o;
-  else
-    ((__nv_bfloat16 *)p.out)[oi] = __float2bfloat16_rn(o);
-}
-
-cudaError_t launch_merge(const StepArgs &a) {
-  AttParams p = make_att_params(a);
-  dim3 grid(a.ly.Hq, a.ly.B);
-  if (a.ly.dtype == S4R_BF16)
-    k_merge<__nv_bfloat16><<<grid, a.ly.dh, 0, a.stream>>>(p);
-  else
-    k_merge<float><<<grid, a.ly.dh, 0, a.stream>>>(p);
-  S4R_LAUNCH_CHECK();
-  return cudaSuccess;
-}
-
 // ======================================================================================================
 // Prefill projection (Eq. 3), generic tiled version: C[t - s][c] = sum_d X[t][d] * Bm[d][c] for rows t >= s;
 // rows t < s are copied to the sink buffer (Sec. 3.1.1).  grid (ceil(r/64), ceil((T-s)/64), B), block 256.
@@ -557,74 +419,6 @@ cudaError_t launch_compress_generic(const Layer &ly, const void *X, const void *
 }
 cudaError_t launch_set_len(const Layer &ly, int32_t *coef_len, int64_t T, cudaStream_t st) {
   k_set_len<<<(ly.B + 127) / 128, 128, 0, st>>>(coef_len, ly.B, (int32_t)(T - ly.s));
-  S4R_LAUNCH_CHECK();
-  return cudaSuccess;
-}
-
-// ======================================================================================================
-// Cache update (Eq. 5-6): one new coefficient row per sequence for K and V, then coef_len += 1.
-// grid (ceil(rmax/32), B, 2), block 256 = 32 columns x 8 row groups.
-// ======================================================================================================
-template <typename T>
-__global__ void __launch_bounds__(256) k_append(const T *__restrict__ k_t, const T *__restrict__ v_t,
-                                                const T *__restrict__ basis_k, const T *__restrict__ basis_v,
-                                                T *__restrict__ coef_k, T *__restrict__ coef_v,
-                                                const int32_t *__restrict__ coef_len, int D, int rk, int rv,
-                                                int64_t cap, int32_t *dev_status) {
-  extern __shared__ float xs[];  // [D]
-  __shared__ float red[8][32];
-  const int b = blockIdx.y, which = blockIdx.z;
-  const int r = which ? rv : rk;
-  const T *x = (which ? v_t : k_t) + (size_t)b * D;
-  const T *basis = (which ? basis_v : basis_k) + (size_t)b * D * r;
-  T *coef = (which ? coef_v : coef_k) + (size_t)b * cap * r;
-  const int len = coef_len[b];
-  if (len < 0 || len >= cap) {
-    if (dev_status && threadIdx.x == 0 && blockIdx.x == 0 && which == 0) atomicOr(dev_status, S4R_DEV_BOUNDS);
-    return;
-  }
-  const int col = blockIdx.x * 32 + (threadIdx.x & 31), rg = threadIdx.x >> 5;
-  if (blockIdx.x * 32 >= r) return;
-  for (int i = threadIdx.x; i < D; i += 256) xs[i] = Store<T>::ld(x + i);
-  __syncthreads();
-  float acc = 0.f;
-  if (col < r)
-    for (int d = rg; d < D; d += 8) acc = fmaf(xs[d], Store<T>::ld(basis + (size_t)d * r + col), acc);
-  red[rg][threadIdx.x & 31] = acc;
-  __syncthreads();
-  if (rg == 0 && col < r) {
-    float s = 0.f;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x & 31];
-    Store<T>::st(coef + (size_t)len * r + col, s);
-  }
-}
-
-__global__ void k_bump_len(int32_t *coef_len, int B, int64_t cap) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < B) {
-    int v = coef_len[i];
-    if (v >= 0 && v < cap) coef_len[i] = v + 1;
-  }
-}
-
-cudaError_t launch_append(const Layer &ly, const void *k_t, const void *v_t, const void *basis_k,
-                          const void *basis_v, void *coef_k, void *coef_v, int32_t *coef_len, int32_t *dev_status,
-                          cudaStream_t st) {
-  const int rmax = ly.rk > ly.rv ? ly.rk : ly.rv;
-  dim3 grid((rmax + 31) / 32, ly.B, 2);
-  size_t smem = (size_t)ly.D * sizeof(float);
-  if (ly.dtype == S4R_BF16)
-    k_append<__nv_bfloat16><<<grid, 256, smem, st>>>(
-        (const __nv_bfloat16 *)k_t, (const __nv_bfloat16 *)v_t, (const __nv_bfloat16 *)basis_k,
-        (const __nv_bfloat16 *)basis_v, (__nv_bfloat16 *)coef_k, (__nv_bfloat16 *)coef_v, coef_len, ly.D, ly.rk, ly.rv,
-        ly.cap, dev_status);
-  else
-    k_append<float><<<grid, 256, smem, st>>>((const float *)k_t, (const float *)v_t, (const float *)basis_k,
-                                             (const float *)basis_v, (float *)coef_k, (float *)coef_v, coef_len, ly.D,
-                                             ly.rk, ly.rv, ly.cap, dev_status);
-  S4R_LAUNCH_CHECK();
-  k_bump_len<<<(ly.B + 127) / 128, 128, 0, st>>>(coef_len, ly.B, ly.cap);
   S4R_LAUNCH_CHECK();
   return cudaSuccess;
 }

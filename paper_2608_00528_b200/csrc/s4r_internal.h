@@ -14,6 +14,10 @@ struct StepArgs {
   Layer ly;
   const void *q, *sink_k, *sink_v, *coef_k, *coef_v, *basis_k, *basis_v;
   const int32_t *coef_len;
+  // fused cache update (Eq. 5-6) in the first kernel of the step; k_t == nullptr: the caller appended already
+  const void *k_t = nullptr, *v_t = nullptr;
+  void *coef_k_w = nullptr, *coef_v_w = nullptr;
+  int32_t *coef_len_w = nullptr;
   int window, top_k, kappa, pool_mode, group_mode;
   float theta;
   void *out;
@@ -40,7 +44,9 @@ int scan_fast_parts(const Layer &ly);  // CTAs (= softmax partials) per sequence
 cudaError_t launch_scan_sm100(const StepArgs &a);
 inline bool att_fast_supported(const Layer &ly) {
   return ly.dtype == S4R_BF16 && ly.dh == 128 && ly.rk % 64 == 0 && ly.rv % 64 == 0 && ly.rk >= 64 && ly.rv >= 64 &&
-         (ly.rk + ly.rv) / 64 <= 6 && (int64_t)ly.B * ly.D < 0x7fffffffLL;
+         (ly.rk + ly.rv) / 64 <= 6 && (int64_t)ly.B * ly.D < 0x7fffffffLL &&
+         // shared memory of k_attend_sm100: coefficient tiles + 3 ring blocks, sin/cos table, q', p, exchange, misc
+         (size_t)((ly.rk + ly.rv) / 64 + 3) * 16384 + 65536 + 8192 + (size_t)4 * ly.G * 128 * 4 + 2048 <= 232448;
 }
 cudaError_t launch_attend_sm100(const StepArgs &a);
 

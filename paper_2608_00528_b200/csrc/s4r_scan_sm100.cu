@@ -78,37 +78,54 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], 4 * 32);
+      mbar_init(&acc_empty[a], 4);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tmap);
   }
   if (warp == 1) tmem_alloc(tmem_slot, 2 * kAccCols);
-  // B operand: row n = t*8 + g holds term t (0 hi, 1 mid, 2 lo, 3 zero) of c^Q[g], K-major, 128-byte swizzle
-  for (int i = tid; i < kMaxGroup * p.r; i += kScanThreads) {
-    const int g = i / p.r, k = i - g * p.r;
-    float c = 0.f;
-    if (g < p.G) {
-#pragma unroll
-      for (int sl = 0; sl < kQSlices; ++sl) c += p.cq_part[(((size_t)b * kQSlices + sl) * p.G + g) * p.r + k];
-    }
-    const __nv_bfloat16 hi = __float2bfloat16_rn(c);
-    const float r1 = c - __bfloat162float(hi);
-    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-    uint8_t *blk = b_op + (size_t)(k >> 6) * (kAccCols * 128);
-    const int kc = k & 63;
-    *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(g, kc)) = hi;
-    *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(8 + g, kc)) = mid;
-    *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(16 + g, kc)) = lo;
-    *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(24 + g, kc)) = __float2bfloat16_rn(0.f);
-  }
-  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+
+  if (warp != 0) {
+    // While the producer (warp 0) already streams tiles, the other warps build the B operand: row n = t*8 + g
+    // holds term t (0 hi, 1 mid, 2 lo, 3 zero) of c^Q[g], K-major, 128-byte swizzle.  Loads go out in batches
+    // of 8 so that their latencies overlap.
+    constexpr int kWorkers = kScanThreads - 32;
+    const int n_el = kMaxGroup * p.r;
+    for (int i0 = tid - 32; i0 < n_el; i0 += 8 * kWorkers) {
+      float cval[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * kWorkers;
+        const int g = i / p.r, k = i - g * p.r;
+        cval[u] = (i < n_el && g < p.G) ? __ldcg(p.cq_part + ((size_t)b * p.G + g) * p.r + k) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * kWorkers;
+        if (i < n_el) {
+          const int g = i / p.r, k = i - g * p.r;
+          const float c = cval[u];
+          const __nv_bfloat16 hi = __float2bfloat16_rn(c);
+          const float r1 = c - __bfloat162float(hi);
+          const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+          uint8_t *blk = b_op + (size_t)(k >> 6) * (kAccCols * 128);
+          const int kc = k & 63;
+          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(g, kc)) = hi;
+          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(8 + g, kc)) = mid;
+          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(16 + g, kc)) = lo;
+          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(24 + g, kc)) = __float2bfloat16_rn(0.f);
+        }
+      }
+    }
+    fence_proxy_async_smem();
+    asm volatile("bar.sync 1, %0;" ::"n"(kScanThreads - 32) : "memory");  // B operand complete (producer not involved)
+  }
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -179,7 +196,8 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
       tmem_ld32(tmem_base + (uint32_t)a * kAccCols + ((uint32_t)(quad * 32) << 16), v);
       tmem_ld_wait();
       tc_fence_before();
-      mbar_arrive(&acc_empty[a]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[a]);
       const int row = (t_begin + it) * kTileRows + row_in_tile;
       if (row < L) {
 #pragma unroll

@@ -21,7 +21,8 @@ namespace s4r {
 namespace {
 
 constexpr int kRelThreads = 256;
-constexpr int kRelOut = 120;                // positions a warp emits (128 held, 4 halo on each side)
+constexpr int kRelOut = 120;                // positions a warp emits per chunk (128 held, 4 halo on each side)
+constexpr int kRelChunks = 2;               // consecutive chunks per warp
 constexpr int kSliceCap = 16384;            // scores of a slice kept in shared memory up to this many
 
 struct RelParams {
@@ -73,27 +74,29 @@ __device__ __forceinline__ void pool_group(const float (&f)[12], float (&acc)[4]
   }
 }
 
-__global__ void __launch_bounds__(kRelThreads) k_relevance(RelParams p) {
+template <int MAXG>
+__global__ void __launch_bounds__(kRelThreads, 4) k_relevance(RelParams p) {
   __shared__ float s_c[kMaxGroup];  // p = exp2(z * log2e + c), c = -M log2e - log2 S
   __shared__ float s_M[kMaxGroup], s_iS[kMaxGroup];
   __shared__ unsigned s_hist[2048];
   const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int L = clamp_len_q(p.coef_len, b, p.max_len);
-  const int out0 = (blockIdx.x * (kRelThreads / 32) + warp) * kRelOut;  // first position this warp emits
-  if (blockIdx.x * (kRelThreads / 32) * kRelOut >= L) return;          // uniform over the CTA
+  if (blockIdx.x * (kRelThreads / 32) * kRelOut * kRelChunks >= L) return;  // uniform over the CTA
   const int W_eff = min(p.window, L), n_cand = L - W_eff;
   // ---- softmax normalisers of Eq. 9 from the scan's partials (empty partials are (-inf, 0))
   if (warp < p.G) {
     const float2 *pp = p.part + (size_t)b * p.n_parts * kMaxGroup + warp;
-    float m = -INFINITY;
-    for (int c = lane; c < p.n_parts; c += 32) m = fmaxf(m, pp[(size_t)c * kMaxGroup].x);
-    m = warp_max(m);
-    float s = 0.f;
+    // one load per lane in the common case (up to 32 partials); merged as (max, scaled sum) pairs
+    float m = -INFINITY, s = 0.f;
     for (int c = lane; c < p.n_parts; c += 32) {
-      const float2 v = pp[(size_t)c * kMaxGroup];
-      if (v.y > 0.f) s += v.y * expf(v.x - m);
+      const float2 v = __ldcg(pp + (size_t)c * kMaxGroup);
+      if (v.y > 0.f) ms_merge(m, s, v.x, v.y);
     }
-    s = warp_sum(s);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+      ms_merge(m, s, m2, s2);
+    }
     if (lane == 0) {
       s_M[warp] = m;
       s_iS[warp] = 1.f / s;
@@ -107,14 +110,18 @@ __global__ void __launch_bounds__(kRelThreads) k_relevance(RelParams p) {
   const int half = p.kappa >> 1;
   const bool group_mean = p.group_mode == S4R_GROUP_MEAN, maxp = p.pool_mode == S4R_POOL_MAX;
   const float inv_kappa = 1.f / (float)p.kappa, inv_G = 1.f / (float)p.G;
+  float *srow = p.score + (size_t)b * p.z_stride;
+#pragma unroll 1
+  for (int ch = 0; ch < kRelChunks; ++ch) {
+  const int out0 = ((blockIdx.x * (kRelThreads / 32) + warp) * kRelChunks + ch) * kRelOut;  // first position emitted
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   const int pos = out0 - 4 + 4 * lane;  // first of this lane's 4 positions (lanes 0 and 31 are halo only)
   if (out0 < L) {
     if (half <= 4) {
       // all loads first, so their latencies overlap
-      float4 zz[kMaxGroup];
+      float4 zz[MAXG];
 #pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g) {
+      for (int g = 0; g < MAXG; ++g) {
         zz[g] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         if (g < p.G) {
           const float *zr = zb + (size_t)g * p.z_stride;
@@ -128,7 +135,7 @@ __global__ void __launch_bounds__(kRelThreads) k_relevance(RelParams p) {
         }
       }
 #pragma unroll
-      for (int g = 0; g < kMaxGroup; ++g) {
+      for (int g = 0; g < MAXG; ++g) {
         if (g >= p.G) break;
         const float c = s_c[g];
         const float4 z = zz[g];
@@ -181,7 +188,6 @@ __global__ void __launch_bounds__(kRelThreads) k_relevance(RelParams p) {
   float sc[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) sc[j] = group_mean ? acc[j] * inv_G : acc[j];
-  float *srow = p.score + (size_t)b * p.z_stride;
   if (emit) {
     if (pos + 3 < L) {
       *reinterpret_cast<float4 *>(srow + pos) = make_float4(sc[0], sc[1], sc[2], sc[3]);
@@ -198,6 +204,7 @@ __global__ void __launch_bounds__(kRelThreads) k_relevance(RelParams p) {
     const unsigned peers = __match_any_sync(0xffffffffu, bin);
     if (valid && lane == __ffs(peers) - 1) atomicAdd(&s_hist[bin], (unsigned)__popc(peers));
   }
+  }  // chunks
   __syncthreads();
   unsigned *gh = p.hist + (size_t)b * 2048;
   for (int i = tid; i < 2048; i += kRelThreads) {
@@ -452,9 +459,12 @@ cudaError_t launch_relevance(const StepArgs &a) {
   p.group_mode = a.group_mode;
   p.max_len = a.plan.max_len;
   p.z_stride = a.plan.z_stride;
-  const int per_cta = (kRelThreads / 32) * kRelOut;
+  const int per_cta = (kRelThreads / 32) * kRelOut * kRelChunks;
   dim3 grid((unsigned)((a.plan.max_len + per_cta - 1) / per_cta), a.ly.B);
-  k_relevance<<<grid, kRelThreads, 0, a.stream>>>(p);
+  if (a.ly.G <= 4)
+    k_relevance<4><<<grid, kRelThreads, 0, a.stream>>>(p);
+  else
+    k_relevance<8><<<grid, kRelThreads, 0, a.stream>>>(p);
   ++launch_counter();
   return cudaGetLastError();
 }

@@ -1,0 +1,475 @@
+// The short kernels of the decode step: per-step projections (Eq. 5-6) and the final merge (Eq. 17-18).
+// Both are latency-bound, so they are written to need as few dependent round trips to memory as possible.
+//
+// k_project: vectors times basis for one sequence by a cluster of kProjCluster CTAs.  Each CTA multiplies a
+//   slice of D' rows of the basis with the matching slice of the vectors: every thread first issues all of
+//   its 16-byte basis loads, then the vectors are staged, then the FMAs run.  Row groups are reduced in
+//   shared memory and rank 0 adds the CTAs' partials in rank order through distributed shared memory, so the
+//   sum has a fixed order and needs no scratch in global memory.
+//   A pass over a basis ("set") carries up to G query vectors Q~[g] (-> c^Q [B][G][r], fp32) and one token
+//   vector (-> one new coefficient row).  Query only: one set.  Append only: k_t over B^K, v_t over B^V.
+//   Fused append + query: {Q~, k_t} over B^K in one pass, then v_t over B^V; coef_len += 1 at the end.
+//   Being the first kernel of a decode step it also clears the score histogram.
+// k_merge: one CTA per (sequence, query head) joins the attention partials of all tiles with the sink
+//   tokens (handled in fp32).  Everything it needs is staged with one wave of cp.async.
+#include <cooperative_groups.h>
+
+#include "s4r_internal.h"
+
+namespace cg = cooperative_groups;
+
+namespace s4r {
+
+namespace {
+
+constexpr int kMaxVec = kMaxGroup + 1;
+constexpr int kRowsInFlight = 16;
+
+struct ProjSet {
+  const void *basis;   // [B, D, r]
+  int r;
+  int nq;              // query vectors in this pass (0 or G)
+  const void *x_tok;   // token vector [B, D] or nullptr
+  void *coef;          // cache that receives the token's coefficient row
+};
+
+struct ProjParams {
+  ProjSet set[2];
+  int n_sets;
+  const void *q;       // [B, Hq, dh]
+  float *cq;           // [B][G][r_k]
+  unsigned *hist;      // cleared when non-null, [B][2048]
+  int32_t *coef_len;   // read when a token vector is present
+  int bump_len;
+  int slot;            // floats per (rank, set) slot of partial sums: max over sets of nv * r
+  int D, G, dh, Hq;
+  int64_t cap;
+  int32_t *dev_status;
+};
+
+template <typename T>
+__device__ __forceinline__ void unpack16(const uint4 &t, float (&v)[Store<T>::kVec]);
+template <>
+__device__ __forceinline__ void unpack16<float>(const uint4 &t, float (&v)[4]) {
+  v[0] = __uint_as_float(t.x); v[1] = __uint_as_float(t.y); v[2] = __uint_as_float(t.z); v[3] = __uint_as_float(t.w);
+}
+template <>
+__device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4 &t, float (&v)[8]) {
+  const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_project(ProjParams p) {
+  constexpr int V = Store<T>::kVec;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = cluster.block_rank(), CL = cluster.num_blocks();
+  const int b = blockIdx.y, tid = threadIdx.x;
+  extern __shared__ __align__(16) float psm[];
+  const int Ds = p.D / CL, d0 = rank * Ds;
+  float *xs = psm;                          // [kMaxVec][Ds]
+  float *partial = xs + kMaxVec * Ds;       // [CL][2][slot]  partial sums of every rank (used in rank 0)
+  float *red = partial + (size_t)CL * 2 * p.slot;  // [row groups][nv][r]  (groups * r <= 256 * V)
+
+  int len = 0;
+  const bool has_tok = p.set[0].x_tok != nullptr || (p.n_sets > 1 && p.set[1].x_tok != nullptr);
+  if (has_tok) {
+    len = p.coef_len[b];
+    if (len < 0 || len >= p.cap) {
+      if (p.dev_status && tid == 0 && rank == 0) atomicOr(p.dev_status, S4R_DEV_BOUNDS);
+      len = -1;  // the token rows are skipped (cache full); query vectors are still projected
+    }
+  }
+  if (p.hist && rank == 0)
+    for (int i = tid; i < 2048; i += 256) p.hist[(size_t)b * 2048 + i] = 0;
+
+  for (int si = 0; si < p.n_sets; ++si) {
+    const ProjSet &st = p.set[si];
+    const int r = st.r, nq = st.nq;
+    const bool tok = st.x_tok != nullptr;
+    const int nv = nq + (tok ? 1 : 0);
+    const T *basis = (const T *)st.basis + ((size_t)b * p.D + d0) * r;
+    const int cpr = r / V;                  // 16-byte chunks per basis row
+    const int groups = min(256 / cpr, Ds);  // row groups working side by side
+    const int c = tid % cpr, rg = tid / cpr;
+    const bool active = rg < groups;
+    float acc[kMaxVec][V];
+#pragma unroll
+    for (int v = 0; v < kMaxVec; ++v)
+#pragma unroll
+      for (int e = 0; e < V; ++e) acc[v][e] = 0.f;
+
+    for (int base = 0; base < Ds; base += groups * kRowsInFlight) {
+      // 1. all basis loads of this batch
+      uint4 raw[kRowsInFlight];
+#pragma unroll
+      for (int i = 0; i < kRowsInFlight; ++i) {
+        const int d = base + rg + i * groups;
+        raw[i] = (active && d < Ds) ? __ldg(reinterpret_cast<const uint4 *>(basis + (size_t)d * r + c * V))
+                                    : make_uint4(0, 0, 0, 0);
+      }
+      // 2. the vectors (first batch only), while those loads are in flight
+      if (base == 0) {
+        for (int i = tid; i < nv * Ds; i += 256) {
+          const int v = i / Ds, d = d0 + (i - v * Ds);
+          float x;
+          if (v < nq)
+            x = Store<T>::ld((const T *)p.q + ((size_t)b * p.Hq + (size_t)(d / p.dh) * p.G + v) * p.dh + (d % p.dh));
+          else
+            x = Store<T>::ld((const T *)st.x_tok + (size_t)b * p.D + d);
+          xs[i] = x;
+        }
+        __syncthreads();
+      }
+      // 3. multiply-accumulate
+#pragma unroll
+      for (int i = 0; i < kRowsInFlight; ++i) {
+        const int d = base + rg + i * groups;
+        if (active && d < Ds) {
+          float bv[V];
+          unpack16<T>(raw[i], bv);
+#pragma unroll
+          for (int v = 0; v < kMaxVec; ++v) {
+            if (v < nv) {
+              const float xv = xs[v * Ds + d];
+#pragma unroll
+              for (int e = 0; e < V; ++e) acc[v][e] = fmaf(xv, bv[e], acc[v][e]);
+            }
+          }
+        }
+      }
+    }
+    if (active) {
+#pragma unroll
+      for (int v = 0; v < kMaxVec; ++v)
+        if (v < nv)
+#pragma unroll
+          for (int e = 0; e < V; ++e) red[((size_t)rg * nv + v) * r + c * V + e] = acc[v][e];
+    }
+    __syncthreads();
+    // this CTA's partial sums, pushed straight into rank 0's slot for this rank (remote stores only: nobody
+    // waits on a read from another SM's shared memory)
+    float *slot0 = cluster.map_shared_rank(partial, 0) + ((size_t)rank * 2 + si) * p.slot;
+    for (int i = tid; i < nv * r; i += 256) {
+      float s = 0.f;
+      for (int g2 = 0; g2 < groups; ++g2) s += red[(size_t)g2 * nv * r + i];
+      slot0[i] = s;
+    }
+    __syncthreads();  // red and xs are reused by the next set
+  }
+  cluster.sync();  // every CTA's partials have landed in rank 0
+  if (rank == 0) {
+    for (int si = 0; si < p.n_sets; ++si) {
+      const ProjSet &st = p.set[si];
+      const int r = st.r, nq = st.nq, nv = nq + (st.x_tok ? 1 : 0);
+      for (int i = tid; i < nv * r; i += 256) {
+        float s = 0.f;
+        for (int rk = 0; rk < CL; ++rk) s += partial[((size_t)rk * 2 + si) * p.slot + i];  // rank order
+        const int v = i / r, col = i - v * r;
+        if (v < nq)
+          p.cq[((size_t)b * p.G + v) * r + col] = s;
+        else if (len >= 0)
+          Store<T>::st((T *)st.coef + ((size_t)b * p.cap + len) * r + col, s);
+      }
+    }
+    if (p.bump_len && has_tok && len >= 0 && tid == 0) p.coef_len[b] = len + 1;
+  }
+}
+
+static int project_slot(const ProjParams &p) {
+  int slot = 0;
+  for (int i = 0; i < p.n_sets; ++i) {
+    const int n = (p.set[i].nq + (p.set[i].x_tok ? 1 : 0)) * p.set[i].r;
+    if (n > slot) slot = n;
+  }
+  return (slot + 3) & ~3;
+}
+
+template <typename T>
+static size_t project_smem(const ProjParams &p) {
+  constexpr int V = Store<T>::kVec;
+  int nv_max = 0;
+  for (int i = 0; i < p.n_sets; ++i) {
+    const int nv = p.set[i].nq + (p.set[i].x_tok ? 1 : 0);
+    if (nv > nv_max) nv_max = nv;
+  }
+  return sizeof(float) * ((size_t)kMaxVec * (p.D / kProjCluster) + (size_t)kProjCluster * 2 * p.slot +
+                          (size_t)nv_max * 256 * V);
+}
+
+template <typename T>
+static cudaError_t project_launch(const ProjParams &p, int B, cudaStream_t st) {
+  constexpr int V = Store<T>::kVec;
+  const int Ds = p.D / kProjCluster;
+  int nv_max = 0;
+  for (int i = 0; i < p.n_sets; ++i) {
+    const int nv = p.set[i].nq + (p.set[i].x_tok ? 1 : 0);
+    if (nv > nv_max) nv_max = nv;
+  }
+  const size_t smem = project_smem<T>(p);
+  static size_t smem_set = 0;
+  if (smem > 48 * 1024 && smem > smem_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_project<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    smem_set = smem;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kProjCluster, B);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kProjCluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, k_project<T>, p);
+  if (e != cudaSuccess) return e;
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------------------
+
+constexpr int kMergeTiles = 32;  // tile partials staged per pass
+
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+struct MergeParams {
+  const void *q, *sink_k, *sink_v;
+  const int32_t *coef_len, *sel_count;
+  const float *part_o;
+  const float2 *part_ms;
+  void *out;
+  int out_dtype, B, Hq, G, dh, D, s, n_tiles, att_tok, sel_stride;
+  int64_t max_len;
+  float theta;
+  double inv_freq[64];
+};
+
+__device__ __forceinline__ void cp_async16(void *dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async8(void *dst, const void *src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+// grid (Hq, B), block dh threads: thread i owns channel i of the head
+template <typename T>
+__global__ void __launch_bounds__(128) k_merge(MergeParams p) {
+  extern __shared__ __align__(16) uint8_t msm[];
+  const int h = blockIdx.x, b = blockIdx.y, i = threadIdx.x, dh = p.dh, nthr = dh;
+  const int kv = h / p.G, half = dh >> 1, lane = i & 31, warp = i >> 5, nwarp = dh >> 5;
+  T *q_s = reinterpret_cast<T *>(msm);                                   // [dh]
+  T *sk_s = q_s + dh;                                                    // [s][dh]
+  T *sv_s = sk_s + (size_t)p.s * dh;                                     // [s][dh]
+  float *po_s = reinterpret_cast<float *>(sv_s + (size_t)p.s * dh);      // [kMergeTiles][dh]
+  float2 *ms_s = reinterpret_cast<float2 *>(po_s + kMergeTiles * dh);    // [kMergeTiles]
+  float *red_s = reinterpret_cast<float *>(ms_s + kMergeTiles);          // [4][64]
+  float *slog_s = red_s + 4 * 64;                                        // [64]
+
+  int L = p.coef_len[b];
+  L = L < 0 ? 0 : ((int64_t)L > p.max_len ? (int)p.max_len : L);
+  const int count = min(p.sel_count[b], p.sel_stride);
+  const int tiles = (count + p.att_tok - 1) / p.att_tok;
+  const float2 *ms = p.part_ms + ((size_t)b * p.Hq + h) * p.n_tiles;
+  const float *po = p.part_o + ((size_t)b * p.Hq + h) * p.n_tiles * dh;
+  constexpr int EPC = 16 / sizeof(T);  // elements per 16-byte chunk
+  const int cpr = dh / EPC;            // chunks per head row
+
+  // ---- one wave of asynchronous copies: q, sinks, the first tile partials
+  {
+    const T *qp = (const T *)p.q + ((size_t)b * p.Hq + h) * dh;
+    if (i < cpr) cp_async16(q_s + i * EPC, qp + i * EPC);
+    for (int cidx = i; cidx < p.s * cpr; cidx += nthr) {
+      const int sj = cidx / cpr, cc = cidx - sj * cpr;
+      const size_t off = ((size_t)b * p.s + sj) * p.D + (size_t)kv * dh + cc * EPC;
+      cp_async16(sk_s + sj * dh + cc * EPC, (const T *)p.sink_k + off);
+      cp_async16(sv_s + sj * dh + cc * EPC, (const T *)p.sink_v + off);
+    }
+    const int nt0 = min(tiles, kMergeTiles);
+    if (i < nt0) cp_async8(ms_s + i, ms + i);
+    for (int cidx = i; cidx < nt0 * (dh / 4); cidx += nthr) cp_async16(po_s + cidx * 4, po + cidx * 4);
+  }
+  // maximum over all tiles when they do not fit one pass
+  float M = -INFINITY;
+  if (tiles > kMergeTiles) {
+    for (int t = i; t < tiles; t += nthr) M = fmaxf(M, ms[t].x);
+    M = warp_max(M);
+    if (lane == 0) red_s[warp] = M;
+  }
+  cp_async_wait_all();
+  __syncthreads();
+  if (tiles > kMergeTiles) {
+    M = red_s[0];
+    for (int w = 1; w < nwarp; ++w) M = fmaxf(M, red_s[w]);
+  } else {
+    for (int t = 0; t < tiles; ++t) M = fmaxf(M, ms_s[t].x);
+  }
+  __syncthreads();  // red_s is reused below
+
+  // ---- rotated, scaled query channel and the sink logits
+  const bool rope = p.theta > 0.f;
+  const int partner = i < half ? i + half : i - half;
+  const double inv_freq = p.inv_freq[i % half];
+  float qi = to_float(q_s[i]);
+  if (rope) {
+    const float o = to_float(q_s[partner]);
+    float sn, cs;
+    rope_sincos(p.s + L - 1, inv_freq, sn, cs);
+    qi = i < half ? qi * cs - o * sn : qi * cs + o * sn;
+  }
+  qi *= rsqrtf((float)dh);
+  for (int sj = 0; sj < p.s; ++sj) {
+    float v = to_float(sk_s[sj * dh + i]);
+    if (rope) {
+      const float o = to_float(sk_s[sj * dh + partner]);
+      float sn, cs;
+      rope_sincos(sj, inv_freq, sn, cs);
+      v = i < half ? v * cs - o * sn : v * cs + o * sn;
+    }
+    const float d = warp_sum(qi * v);
+    if (lane == 0) red_s[warp * 64 + sj] = d;
+  }
+  __syncthreads();
+  if (i < p.s) {
+    float d = 0.f;
+    for (int w = 0; w < nwarp; ++w) d += red_s[w * 64 + i];
+    slog_s[i] = d;
+  }
+  __syncthreads();
+  for (int sj = 0; sj < p.s; ++sj) M = fmaxf(M, slog_s[sj]);
+
+  // ---- weighted sums
+  float den = 0.f, num = 0.f;
+  for (int t0 = 0; t0 < tiles; t0 += kMergeTiles) {
+    const int nt = min(kMergeTiles, tiles - t0);
+    if (t0 > 0) {  // restage the next pass
+      __syncthreads();
+      if (i < nt) cp_async8(ms_s + i, ms + t0 + i);
+      for (int cidx = i; cidx < nt * (dh / 4); cidx += nthr) cp_async16(po_s + cidx * 4, po + (size_t)t0 * dh + cidx * 4);
+      cp_async_wait_all();
+      __syncthreads();
+    }
+    for (int t = 0; t < nt; ++t) {
+      const float2 v = ms_s[t];
+      const float w = v.y > 0.f ? __expf(v.x - M) : 0.f;
+      den = fmaf(v.y, w, den);
+      num = fmaf(po_s[t * dh + i], w, num);
+    }
+  }
+  for (int sj = 0; sj < p.s; ++sj) {
+    const float w = __expf(slog_s[sj] - M);
+    den += w;
+    num = fmaf(to_float(sv_s[sj * dh + i]), w, num);
+  }
+  const float o = (tiles + p.s > 0 && den > 0.f) ? num / den : 0.f;
+  const size_t oi = ((size_t)b * p.Hq + h) * dh + i;
+  if (p.out_dtype == S4R_F32)
+    ((float *)p.out)[oi] = o;
+  else
+    ((__nv_bfloat16 *)p.out)[oi] = __float2bfloat16_rn(o);
+}
+
+}  // namespace
+
+void fill_inv_freq(double *dst, int head_dim, float theta) {
+  for (int i = 0; i < 64; ++i) dst[i] = 0.0;
+  if (theta > 0.f)
+    for (int i = 0; i < head_dim / 2 && i < 64; ++i) dst[i] = pow((double)theta, -2.0 * (double)i / (double)head_dim);
+}
+
+// Query projection; when a.k_t is set, the new token's key and value rows are projected and appended too.
+cudaError_t launch_qproj(const StepArgs &a) {
+  const Layer &ly = a.ly;
+  ProjParams p = {};
+  p.q = a.q;
+  p.cq = (float *)(a.ws + a.plan.off_cq);
+  p.hist = (unsigned *)(a.ws + a.plan.off_hist);
+  p.D = ly.D; p.G = ly.G; p.dh = ly.dh; p.Hq = ly.Hq; p.cap = ly.cap; p.dev_status = a.dev_status;
+  p.set[0].basis = a.basis_k; p.set[0].r = ly.rk; p.set[0].nq = ly.G;
+  p.n_sets = 1;
+  if (a.k_t) {
+    // fused cache update; if its partial sums would not fit in shared memory, append first in a launch of its own
+    ProjParams f = p;
+    f.set[0].x_tok = a.k_t; f.set[1].basis = a.basis_v; f.set[1].r = ly.rv; f.set[1].x_tok = a.v_t; f.n_sets = 2;
+    f.slot = project_slot(f);
+    const size_t need = ly.dtype == S4R_BF16 ? project_smem<__nv_bfloat16>(f) : project_smem<float>(f);
+    if (need > 200 * 1024) {
+      cudaError_t e = launch_append(ly, a.k_t, a.v_t, a.basis_k, a.basis_v, a.coef_k_w, a.coef_v_w, a.coef_len_w,
+                                    a.dev_status, a.stream);
+      if (e != cudaSuccess) return e;
+      p.slot = project_slot(p);
+      return ly.dtype == S4R_BF16 ? project_launch<__nv_bfloat16>(p, ly.B, a.stream)
+                                  : project_launch<float>(p, ly.B, a.stream);
+    }
+    p.set[0].x_tok = a.k_t; p.set[0].coef = a.coef_k_w;
+    p.set[1].basis = a.basis_v; p.set[1].r = ly.rv; p.set[1].nq = 0; p.set[1].x_tok = a.v_t; p.set[1].coef = a.coef_v_w;
+    p.n_sets = 2;
+    p.coef_len = a.coef_len_w;
+    p.bump_len = 1;
+  }
+  p.slot = project_slot(p);
+  return ly.dtype == S4R_BF16 ? project_launch<__nv_bfloat16>(p, ly.B, a.stream) : project_launch<float>(p, ly.B, a.stream);
+}
+
+cudaError_t launch_append(const Layer &ly, const void *k_t, const void *v_t, const void *basis_k,
+                          const void *basis_v, void *coef_k, void *coef_v, int32_t *coef_len, int32_t *dev_status,
+                          cudaStream_t st) {
+  ProjParams p = {};
+  p.D = ly.D; p.G = ly.G; p.dh = ly.dh; p.Hq = ly.Hq; p.cap = ly.cap; p.dev_status = dev_status;
+  p.set[0].basis = basis_k; p.set[0].r = ly.rk; p.set[0].x_tok = k_t; p.set[0].coef = coef_k;
+  p.set[1].basis = basis_v; p.set[1].r = ly.rv; p.set[1].x_tok = v_t; p.set[1].coef = coef_v;
+  p.n_sets = 2;
+  p.coef_len = coef_len;
+  p.bump_len = 1;
+  p.slot = project_slot(p);
+  return ly.dtype == S4R_BF16 ? project_launch<__nv_bfloat16>(p, ly.B, st) : project_launch<float>(p, ly.B, st);
+}
+
+cudaError_t launch_merge(const StepArgs &a) {
+  const Layer &ly = a.ly;
+  MergeParams p;
+  p.q = a.q; p.sink_k = a.sink_k; p.sink_v = a.sink_v; p.coef_len = a.coef_len; p.sel_count = a.sel_count;
+  p.part_o = (const float *)(a.ws + a.plan.off_att);
+  p.part_ms = (const float2 *)(a.ws + a.plan.off_att_ms);
+  p.out = a.out; p.out_dtype = a.out_dtype; p.B = ly.B; p.Hq = ly.Hq; p.G = ly.G; p.dh = ly.dh; p.D = ly.D;
+  p.s = ly.s; p.n_tiles = a.plan.n_att_tiles; p.att_tok = a.plan.att_tok; p.sel_stride = a.window + a.top_k;
+  p.max_len = a.plan.max_len; p.theta = a.theta;
+  fill_inv_freq(p.inv_freq, ly.dh, a.theta);
+  const size_t esz = ly.dtype == S4R_BF16 ? 2 : 4;
+  const size_t smem = esz * (size_t)ly.dh * (1 + 2 * (size_t)ly.s) + sizeof(float) * kMergeTiles * ly.dh +
+                      sizeof(float2) * kMergeTiles + sizeof(float) * (4 * 64 + 64) + 16;
+  dim3 grid(ly.Hq, ly.B);
+  if (ly.dtype == S4R_BF16) {
+    static size_t set_b = 0;
+    if (smem > 48 * 1024 && smem > set_b) {
+      cudaFuncSetAttribute(k_merge<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      set_b = smem;
+    }
+    k_merge<__nv_bfloat16><<<grid, ly.dh, smem, a.stream>>>(p);
+  } else {
+    static size_t set_f = 0;
+    if (smem > 48 * 1024 && smem > set_f) {
+      cudaFuncSetAttribute(k_merge<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      set_f = smem;
+    }
+    k_merge<float><<<grid, ly.dh, smem, a.stream>>>(p);
+  }
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace s4r

@@ -263,3 +263,32 @@ def test_multi_layer_multi_step_generation_with_append():
             out, sel, cnt, st = run_gpu_step(p)
             assert st == 0
             check_step(p, out, sel, cnt, L=L)
+
+
+def test_fused_append_decode_equals_separate_calls():
+    s4r = _s4r()
+    cfg = _cfg(1, context=5000 + 3, batch=2)
+    res = []
+    for fused in (False, True):
+        p = Problem(cfg, device="cuda", capacity=cfg.cache_len + 4).upload()
+        ly = p.layer_desc()
+        ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+        out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, device="cuda")
+        sel = torch.empty(cfg.batch, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+        cnt = torch.empty(cfg.batch, dtype=torch.int32, device="cuda")
+        for step in (1, 2):
+            kt = torch.stack([W.make_token(cfg, 0, b, "k", step, "cuda") for b in range(cfg.batch)])
+            vt = torch.stack([W.make_token(cfg, 0, b, "v", step, "cuda") for b in range(cfg.batch)])
+            if fused:
+                s4r.append_decode_step(ly, kt, vt, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK,
+                                       p.d_BV, p.cap, cfg.window, cfg.top_k, out, sel, cnt, ws,
+                                       rope_theta=cfg.rope_theta)
+            else:
+                s4r.append(ly, kt, vt, p.d_BK, p.d_BV, p.d_CK, p.d_CV, p.d_len)
+                s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                cfg.window, cfg.top_k, out, sel, cnt, ws, rope_theta=cfg.rope_theta)
+        torch.cuda.synchronize()
+        res.append((out.clone(), sel.clone(), cnt.clone(), p.d_CK.clone(), p.d_CV.clone(), p.d_len.clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
+    assert res[0][5].tolist() == [cfg.cache_len + 2] * cfg.batch
