@@ -62,6 +62,8 @@ typedef enum {
 #define S4R_POOL_AVG 1
 #define S4R_GROUP_MEAN 0
 #define S4R_GROUP_MAX 1
+#define S4R_VALUE_AUTO 0
+#define S4R_VALUE_RECONSTRUCT 1
 
 /* Layer geometry, validated on every call.
  * Supported: head_dim 128 (also 64), G <= 8, rank_k and rank_v multiples of 8 in [8, 512],
@@ -85,6 +87,10 @@ typedef struct {
   int32_t pool_kernel;  /* kappa, odd, 1 = no pooling, <= 31                              */
   int32_t pool_mode;    /* S4R_POOL_MAX | S4R_POOL_AVG                                    */
   int32_t group_mode;   /* S4R_GROUP_MEAN | S4R_GROUP_MAX                                 */
+  int32_t value_path;   /* S4R_VALUE_AUTO (0) | S4R_VALUE_RECONSTRUCT: how Eq. 16-18 treat the values.
+                         * RECONSTRUCT forms V^ = C^V[sel] (B^V)^T on chip and then P V^, literally Eq. 16.
+                         * AUTO lets the library evaluate the same product as (P C^V[sel]) (B^V)^T where that is
+                         * faster (bf16, head_dim 128); the two agree up to fp32 rounding order.             */
 } s4r_score_t;
 
 /* RoPE of Eq. 18: rotate-half pairing (i, i + d_h/2), inv_freq_i = theta^(-2i/d_h), no scaling.
@@ -219,6 +225,8 @@ int s4r_stage_timing(int enable);
 int s4r_stage_times(float *ms_out, int n);
 
 const char *s4r_strerror(int status);
+/* Text of the last CUDA runtime error that made a call on this host thread return S4R_ERR_CUDA. */
+const char *s4r_last_cuda_error(void);
 int s4r_version(void);
 
 #ifdef __cplusplus

@@ -17,19 +17,25 @@ from . import _build
 S4R_F32, S4R_BF16 = 0, 1
 POOL_MAX, POOL_AVG = 0, 1
 GROUP_MEAN, GROUP_MAX = 0, 1
+VALUE_AUTO, VALUE_RECONSTRUCT = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_compress", "s4r_append", "s4r_decode_step", "s4r_decode_step_host",
            "s4r_decode_step_static", "s4r_append_decode_step",
            "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
-           "s4r_stage_times", "s4r_strerror", "s4r_version")
+           "s4r_stage_times", "s4r_strerror", "s4r_last_cuda_error", "s4r_version")
 STAGES = ("query_projection", "latent_scoring", "selection", "reconstruct_attend", "merge")
 
 
 class S4RError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {strerror(status)} ({status})")
+        detail = ""
+        if status == -4:
+            fn = load().s4r_last_cuda_error
+            fn.restype = ctypes.c_char_p
+            detail = ": " + fn().decode()
+        super().__init__(f"{where}: {strerror(status)} ({status}){detail}")
 
 
 class _Layer(ctypes.Structure):
@@ -40,7 +46,7 @@ class _Layer(ctypes.Structure):
 
 class _Score(ctypes.Structure):
     _fields_ = [("score_window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("pool_mode", ctypes.c_int32),
-                ("group_mode", ctypes.c_int32)]
+                ("group_mode", ctypes.c_int32), ("value_path", ctypes.c_int32)]
 
 
 class _Rope(ctypes.Structure):
@@ -218,17 +224,17 @@ def append(layer: Layer, k_t, v_t, key_basis, value_basis, coef_k, coef_v, coef_
         raise S4RError(rc, "s4r_append")
 
 
-def _score_rope(pool_kernel, pool_mode, group_mode, score_window, theta):
-    return _Score(score_window, pool_kernel, pool_mode, group_mode), _Rope(float(theta), 0)
+def _score_rope(pool_kernel, pool_mode, group_mode, score_window, theta, value_path=0):
+    return _Score(score_window, pool_kernel, pool_mode, group_mode, value_path), _Rope(float(theta), 0)
 
 
 def decode_step(layer: Layer, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis, max_len: int,
                 window: int, top_k: int, out, sel_idx, sel_count, workspace, *, pool_kernel: int = 7,
                 pool_mode: int = POOL_MAX, group_mode: int = GROUP_MEAN, score_window: int = 1,
-                rope_theta: float = 0.0, dev_status=None, stream=None):
+                rope_theta: float = 0.0, value_path: int = VALUE_AUTO, dev_status=None, stream=None):
     """s4r_decode_step: writes `out` [B, H_q, d_h], `sel_idx` [B, window + top_k] and `sel_count` [B]."""
     _need_cuda(q, coef_k, coef_v, coef_len, key_basis, value_basis, out, sel_idx, sel_count, workspace)
-    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, score_window, rope_theta)
+    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, score_window, rope_theta, value_path)
     out_dtype = S4R_BF16 if out.dtype == torch.bfloat16 else S4R_F32
     rc = load().s4r_decode_step(ctypes.byref(layer.c()), _ptr(q), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k),
                                 _ptr(coef_v), _ptr(coef_len), _ptr(key_basis), _ptr(value_basis), int(max_len),

@@ -49,7 +49,8 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   p->off_part = off;    off = align_up(off + sizeof(float2) * ly.B * p->parts_cap * kMaxGroup, 256);
   p->off_score = off;   off = align_up(off + sizeof(float) * ly.B * p->z_stride, 256);
   p->off_hist = off;    off = align_up(off + sizeof(unsigned) * ly.B * 2048, 256);
-  p->off_att = off;     off = align_up(off + sizeof(float) * ly.B * ly.Hq * (size_t)p->n_att_tiles * ly.dh, 256);
+  p->off_att = off;     off = align_up(off + sizeof(float) * ly.B * ly.Hq * (size_t)p->n_att_tiles *
+                                             (att_fast_supported(ly) && 2 * ly.rv > ly.dh ? 2 * ly.rv : ly.dh), 256);
   p->off_att_ms = off;  off = align_up(off + sizeof(float2) * ly.B * ly.Hq * (size_t)p->n_att_tiles, 256);
   p->off_basis_t = off;
   p->total = off > 256 ? off : 256;
@@ -82,6 +83,16 @@ static inline void stage_mark(int i, cudaStream_t st) {
     cudaEventRecord(t.ev[i], st);
     if (i == S4R_N_STAGES) t.recorded = true;
   }
+}
+
+static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+static inline bool cuda_failed(cudaError_t e) {
+  if (e != cudaSuccess) {
+    g_last_cuda_error = e;
+    (void)cudaGetLastError();
+    return true;
+  }
+  return false;
 }
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -124,13 +135,11 @@ int s4r_compress(const s4r_layer_t *layer, const void *K, const void *V, int64_t
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < compress_fast_workspace(ly))
       return S4R_ERR_WORKSPACE;
   }
-  if (launch_compress_generic(ly, K, key_basis, ly.rk, sink_k, coef_k, T, !fast_k, st) != cudaSuccess) return S4R_ERR_CUDA;
-  if (fast_k && launch_compress_sm100(ly, K, key_basis, ly.rk, bt_k, coef_k, T, dev_status, st) != cudaSuccess)
-    return S4R_ERR_CUDA;
-  if (launch_compress_generic(ly, V, value_basis, ly.rv, sink_v, coef_v, T, !fast_v, st) != cudaSuccess) return S4R_ERR_CUDA;
-  if (fast_v && launch_compress_sm100(ly, V, value_basis, ly.rv, bt_v, coef_v, T, dev_status, st) != cudaSuccess)
-    return S4R_ERR_CUDA;
-  if (launch_set_len(ly, coef_len, T, st) != cudaSuccess) return S4R_ERR_CUDA;
+  if (cuda_failed(launch_compress_generic(ly, K, key_basis, ly.rk, sink_k, coef_k, T, !fast_k, st))) return S4R_ERR_CUDA;
+  if (fast_k && cuda_failed(launch_compress_sm100(ly, K, key_basis, ly.rk, bt_k, coef_k, T, dev_status, st))) return S4R_ERR_CUDA;
+  if (cuda_failed(launch_compress_generic(ly, V, value_basis, ly.rv, sink_v, coef_v, T, !fast_v, st))) return S4R_ERR_CUDA;
+  if (fast_v && cuda_failed(launch_compress_sm100(ly, V, value_basis, ly.rv, bt_v, coef_v, T, dev_status, st))) return S4R_ERR_CUDA;
+  if (cuda_failed(launch_set_len(ly, coef_len, T, st))) return S4R_ERR_CUDA;
   return S4R_OK;
 }
 
@@ -167,11 +176,12 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (ly.s > 0 && (!sink_k || !sink_v)) return S4R_ERR_INVALID_ARG;
   if (out_dtype != S4R_F32 && out_dtype != S4R_BF16) return S4R_ERR_INVALID_ARG;
   if (max_len < 0 || max_len > ly.cap || window < 0 || top_k < 0) return S4R_ERR_INVALID_ARG;
-  s4r_score_t sc = {1, 7, S4R_POOL_MAX, S4R_GROUP_MEAN};
+  s4r_score_t sc = {1, 7, S4R_POOL_MAX, S4R_GROUP_MEAN, S4R_VALUE_AUTO};
   if (score) sc = *score;
   if (sc.score_window < 1 || sc.pool_kernel < 1 || (sc.pool_kernel & 1) == 0) return S4R_ERR_INVALID_ARG;
   if (sc.pool_mode != S4R_POOL_MAX && sc.pool_mode != S4R_POOL_AVG) return S4R_ERR_INVALID_ARG;
   if (sc.group_mode != S4R_GROUP_MEAN && sc.group_mode != S4R_GROUP_MAX) return S4R_ERR_INVALID_ARG;
+  if (sc.value_path != S4R_VALUE_AUTO && sc.value_path != S4R_VALUE_RECONSTRUCT) return S4R_ERR_INVALID_ARG;
   if (sc.score_window != 1) return S4R_ERR_UNSUPPORTED;
   if (sc.pool_kernel > 2 * kMaxPoolHalf + 1) return S4R_ERR_UNSUPPORTED;
   if (rope && rope->reserved != 0) return S4R_ERR_INVALID_ARG;
@@ -183,7 +193,7 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (int rc = check_arch()) return rc;
   a.q = q; a.sink_k = sink_k; a.sink_v = sink_v; a.coef_k = coef_k; a.coef_v = coef_v; a.coef_len = coef_len;
   a.basis_k = key_basis; a.basis_v = value_basis; a.window = window; a.top_k = top_k; a.kappa = sc.pool_kernel;
-  a.pool_mode = sc.pool_mode; a.group_mode = sc.group_mode; a.theta = rope ? rope->theta : 0.f; a.out = out;
+  a.pool_mode = sc.pool_mode; a.group_mode = sc.group_mode; a.value_path = sc.value_path; a.theta = rope ? rope->theta : 0.f; a.out = out;
   a.out_dtype = out_dtype; a.sel_idx = sel_idx; a.sel_count = sel_count; a.ws = (char *)workspace;
   a.dev_status = dev_status; a.stream = (cudaStream_t)stream;
   if (k_t) {
@@ -197,24 +207,31 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
     if (parts < 1 || parts > a.plan.parts_cap) fast_scan = false; else a.plan.n_parts = parts;
   }
   stage_mark(0, a.stream);
-  if (launch_qproj(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (cuda_failed(launch_qproj(a))) return S4R_ERR_CUDA;
   stage_mark(1, a.stream);
   if (fast_scan) {
-    if (launch_scan_sm100(a) != cudaSuccess) return S4R_ERR_CUDA;
+    if (cuda_failed(launch_scan_sm100(a))) return S4R_ERR_CUDA;
   } else {
-    if (launch_scan_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+    if (cuda_failed(launch_scan_generic(a))) return S4R_ERR_CUDA;
   }
   stage_mark(2, a.stream);
-  if (launch_relevance(a) != cudaSuccess) return S4R_ERR_CUDA;
-  if (launch_select(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (cuda_failed(launch_relevance(a))) return S4R_ERR_CUDA;
+  if (cuda_failed(launch_select(a))) return S4R_ERR_CUDA;
   stage_mark(3, a.stream);
-  if (att_fast_supported(ly)) {
-    if (launch_attend_sm100(a) != cudaSuccess) return S4R_ERR_CUDA;
+  const bool absorb = att_fast_supported(ly) && a.value_path == S4R_VALUE_AUTO;
+  if (absorb) {
+    if (cuda_failed(launch_attend_absorb(a))) return S4R_ERR_CUDA;
+  } else if (att_fast_supported(ly)) {
+    if (cuda_failed(launch_attend_sm100(a))) return S4R_ERR_CUDA;
   } else {
-    if (launch_attend_generic(a) != cudaSuccess) return S4R_ERR_CUDA;
+    if (cuda_failed(launch_attend_generic(a))) return S4R_ERR_CUDA;
   }
   stage_mark(4, a.stream);
-  if (launch_merge(a) != cudaSuccess) return S4R_ERR_CUDA;
+  if (absorb) {
+    if (cuda_failed(launch_merge_absorb(a))) return S4R_ERR_CUDA;
+  } else {
+    if (cuda_failed(launch_merge(a))) return S4R_ERR_CUDA;
+  }
   stage_mark(5, a.stream);
   return S4R_OK;
 }
@@ -359,6 +376,8 @@ int s4r_stage_times(float *ms_out, int n) {
     if (cudaEventElapsedTime(&ms_out[i], t.ev[i], t.ev[i + 1]) != cudaSuccess) return S4R_ERR_CUDA;
   return m;
 }
+
+const char *s4r_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 const char *s4r_strerror(int status) {
   switch (status) {

@@ -18,7 +18,7 @@ struct StepArgs {
   const void *k_t = nullptr, *v_t = nullptr;
   void *coef_k_w = nullptr, *coef_v_w = nullptr;
   int32_t *coef_len_w = nullptr;
-  int window, top_k, kappa, pool_mode, group_mode;
+  int window, top_k, kappa, pool_mode, group_mode, value_path;
   float theta;
   void *out;
   int out_dtype;
@@ -49,6 +49,9 @@ inline bool att_fast_supported(const Layer &ly) {
          (size_t)((ly.rk + ly.rv) / 64 + 3) * 16384 + 65536 + 8192 + (size_t)4 * ly.G * 128 * 4 + 2048 <= 232448;
 }
 cudaError_t launch_attend_sm100(const StepArgs &a);
+// value side absorbed: (P C^V)(B^V)^T; needs the same geometry as the reconstructing kernel
+cudaError_t launch_attend_absorb(const StepArgs &a);
+cudaError_t launch_merge_absorb(const StepArgs &a);
 
 cudaError_t launch_attend_generic(const StepArgs &a);
 cudaError_t launch_merge(const StepArgs &a);

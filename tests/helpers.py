@@ -100,7 +100,7 @@ class Problem:
 
 def run_gpu_step(p: Problem, W_: int | None = None, k: int | None = None, theta: float | None = None,
                  kappa: int | None = None, pool_mode: str | None = None, group_mode: str | None = None,
-                 out_dtype: torch.dtype | None = None, max_len: int | None = None):
+                 out_dtype: torch.dtype | None = None, max_len: int | None = None, value_path: int = 0):
     import paper_2608_00528_b200 as s4r
     cfg = p.cfg
     W_ = cfg.window if W_ is None else W_
@@ -118,7 +118,7 @@ def run_gpu_step(p: Problem, W_: int | None = None, k: int | None = None, theta:
     gm = {"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode if group_mode is None else group_mode]
     s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, max_len, W_, k,
                     out, sel_buf, cnt, ws, pool_kernel=cfg.pool_kernel if kappa is None else kappa, pool_mode=pm,
-                    group_mode=gm, rope_theta=theta, dev_status=status)
+                    group_mode=gm, rope_theta=theta, value_path=value_path, dev_status=status)
     torch.cuda.synchronize()
     return out, sel, cnt, int(status.item())
 

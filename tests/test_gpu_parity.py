@@ -31,20 +31,24 @@ def test_decode_config0_fp32(theta):
 
 
 @pytest.mark.parametrize("theta", [None, 0.0])
-def test_decode_llama_shape_bf16_8k(theta):
-    # config 1's layer at a context that spans several scan chunks and a ragged tail, batch 2
+@pytest.mark.parametrize("value_path", [0, 1])
+def test_decode_llama_shape_bf16_8k(theta, value_path):
+    # config 1's layer at a context that spans several scan chunks and a ragged tail, batch 2;
+    # value_path 1 = values reconstructed as in Eq. 16, 0 = library's choice (absorbed on this geometry)
     p = Problem(_cfg(1, context=8192 + 333, batch=2), device="cuda").upload()
-    out, sel, cnt, status = run_gpu_step(p, theta=theta)
+    out, sel, cnt, status = run_gpu_step(p, theta=theta, value_path=value_path)
     assert status == 0
     err = check_step(p, out, sel, cnt, theta=theta)
-    print(f"llama 8k theta={theta}: max rel err {err:.3e}")
+    print(f"llama 8k theta={theta} value_path={value_path}: max rel err {err:.3e}")
 
 
-def test_decode_qwen_shape_bf16_8k_group7():
+@pytest.mark.parametrize("value_path", [0, 1])
+def test_decode_qwen_shape_bf16_8k_group7(value_path):
     p = Problem(_cfg(3, context=8192 + 77, batch=2, top_k=512), device="cuda").upload()
-    out, sel, cnt, status = run_gpu_step(p)
+    out, sel, cnt, status = run_gpu_step(p, value_path=value_path)
     assert status == 0
-    check_step(p, out, sel, cnt)
+    err = check_step(p, out, sel, cnt)
+    print(f"qwen 8k value_path={value_path}: max rel err {err:.3e}")
 
 
 def test_decode_config1_full_size():
