@@ -28,6 +28,11 @@ import torch  # noqa: E402
 
 import workloads as W  # noqa: E402
 
+# DRAM bytes (read + write) of one latent-scoring launch per algorithmic byte, from an `ncu --set full` capture of
+# the same launch configuration at 64K context (207.40 MB moved for 201.33 MB of key coefficients); the traffic
+# grows in proportion to the rows scanned, so the ratio carries to the 128K launch.
+SCAN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 207.40 / 201.33
+
 METRIC = "decode steps/sec at 128K context (one layer, whole batch)"
 UNIT = "steps/s"
 
@@ -41,54 +46,89 @@ def _peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons through NVML (read-only queries) every few milliseconds from a
+    thread while the timed region runs; falls back to an `nvidia-smi -lms` child process without NVML."""
 
-    def __init__(self, index: int):
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40}
+
+    def __init__(self, index: int, period_s: float = 0.002):
         self.index = index
-        self.rows = []
+        self.period = period_s
+        self.sm, self.mx, self.reasons = [], [], set()
+        self.stop_flag = threading.Event()
+        self.thread = None
         self.proc = None
+        self.source = None
+
+    def _nvml_loop(self, nv, handle):
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(handle))
+                for name, bit in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:       # noqa: BLE001  (a failed read-only query just skips the sample)
+                pass
+            time.sleep(self.period)
+
+    def _smi_loop(self):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.proc.stdout:
+            r = [c.strip() for c in line.split(",")]
+            if len(r) < 6:
+                continue
+            try:
+                self.sm.append(float(r[0])); self.mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    self.reasons.add(n)
 
     def start(self):
-        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            # NVML enumerates physical devices; map through CUDA_VISIBLE_DEVICES when it lists plain indices
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            idx = self.index
+            parts = [v for v in vis.split(",") if v.strip()]
+            if parts and all(v.strip().isdigit() for v in parts) and self.index < len(parts):
+                idx = int(parts[self.index])
+            handle = nv.nvmlDeviceGetHandleByIndex(idx)
+            self.mx.append(float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM)))
+            self.source = "nvml"
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nv, handle), daemon=True)
+            self.thread.start()
+            return
+        except Exception:           # noqa: BLE001
+            pass
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.source = "nvidia-smi"
+            self.thread = threading.Thread(target=self._smi_loop, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
-
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            if len(r) < 7:
-                continue
+        self.stop_flag.set()
+        if self.proc is not None:
+            self.proc.terminate()
             try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        sm = sorted(self.sm)
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(self.mx) if self.mx else None,
+                "reasons": sorted(self.reasons), "samples": len(sm), "source": self.source}
 
 
 def build_cache(cfg, s4r, device, capacity):
@@ -182,7 +222,7 @@ def run_reference(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
@@ -261,6 +301,7 @@ def main():
         step(Wm + i)
     e1.record()
     barrier()
+    clocks = sampler.stop() if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
     gpu_launches = launches[0]
     if dist is not None:
@@ -281,7 +322,6 @@ def main():
             stage_sum[k_] = stage_sum.get(k_, 0.0) + v_
     s4r.stage_timing(False)
     stage_ms = {k_: v_ / n_prof for k_, v_ in stage_sum.items()}
-    clocks = sampler.stop() if rank == 0 else None
 
     # ---- end to end through the host-buffer entry point: q from pinned host memory, results read back
     c["len"].fill_(cfg.cache_len)
@@ -342,7 +382,9 @@ def main():
                    "l2": "inputs larger than L2 (key coefficients %.0f MB per step)" % (scan_bytes / 1e6),
                    "parallelism": f"dp{world} (independent sequences, no collective)"},
         "roofline": {"bound": "hbm", "kernel": "latent_scoring", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                     "frac": achieved / peak, "peak_kind": peak_kind,
+                     "traffic": scan_bytes * SCAN_DRAM_BYTES_PER_ALGORITHMIC_BYTE,
+                     "traffic_source": "ncu capture at 64K context scaled by rows (profiles/)",
                      "bytes_per_launch": scan_bytes, "ms_per_launch": scan_ms},
         "step_roofline": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_bytes / (ms_step * 1e-3) / 1e9,
                           "frac_of_8TBs": step_bytes / (ms_step * 1e-3) / 8e12,

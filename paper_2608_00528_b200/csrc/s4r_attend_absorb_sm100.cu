@@ -53,6 +53,7 @@ __device__ __forceinline__ void cp_async16_zfill(void *dst, const void *src, boo
 
 __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_constant__ CUtensorMap tmap_bk,
                                                                const __grid_constant__ AbsorbParams p) {
+  grid_dependency_sync();
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int kbk = p.rk >> 6, kbv = p.rv >> 6, G = p.G;
@@ -398,6 +399,7 @@ __device__ __forceinline__ void cp_async8(void *dst, const void *src) {
 constexpr int kMgTiles = 32;
 
 __global__ void __launch_bounds__(128) k_merge_absorb(const __grid_constant__ MergeAbsorbParams p) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) uint8_t msm[];
   const int h = blockIdx.x, b = blockIdx.y, i = threadIdx.x;
   const int kv = h / p.G, lane = i & 31, warp = i >> 5;
@@ -576,7 +578,8 @@ cudaError_t launch_attend_absorb(const StepArgs &a) {
     smem_set = smem;
   }
   dim3 grid(p.n_tiles, split, ly.B);
-  k_attend_absorb<<<grid, kThreads, smem, a.stream>>>(tm_k, p);
+  cudaError_t le = launch_chained(k_attend_absorb, grid, dim3(kThreads), smem, a.stream, 1, tm_k, p);
+  if (le != cudaSuccess) return le;
   ++launch_counter();
   return cudaGetLastError();
 }
@@ -604,7 +607,8 @@ cudaError_t launch_merge_absorb(const StepArgs &a) {
     smem_set = smem;
   }
   dim3 grid(ly.Hq, ly.B);
-  k_merge_absorb<<<grid, 128, smem, a.stream>>>(p);
+  cudaError_t le = launch_chained(k_merge_absorb, grid, dim3(128), smem, a.stream, 1, p);
+  if (le != cudaSuccess) return le;
   ++launch_counter();
   return cudaGetLastError();
 }

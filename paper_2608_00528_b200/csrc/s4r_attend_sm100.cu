@@ -57,6 +57,7 @@ __device__ __forceinline__ void cp_async16_zfill(void *dst, const void *src, boo
 __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_constant__ CUtensorMap tmap_bk,
                                                               const __grid_constant__ CUtensorMap tmap_bv,
                                                               const __grid_constant__ AttFastParams p) {
+  grid_dependency_sync();
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int kbk = p.rk >> 6, kbv = p.rv >> 6, G = p.G;
@@ -424,7 +425,8 @@ cudaError_t launch_attend_sm100(const StepArgs &a) {
     smem_set = smem;
   }
   dim3 grid(p.n_tiles, split, ly.B);
-  k_attend_sm100<<<grid, kThreads, smem, a.stream>>>(tm_k, tm_v, p);
+  cudaError_t le = launch_chained(k_attend_sm100, grid, dim3(kThreads), smem, a.stream, 1, tm_k, tm_v, p);
+  if (le != cudaSuccess) return le;
   ++launch_counter();
   return cudaGetLastError();
 }

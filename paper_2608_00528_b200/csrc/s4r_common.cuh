@@ -18,6 +18,42 @@ constexpr int kMaxCluster = 8;     // CTAs per sequence in the selection kernel 
 constexpr int kProjCluster = 8;    // CTAs (slices of D') per sequence in the projection kernels
 constexpr int kMaxParts = 256;     // upper bound of softmax partials per sequence written by a scan kernel
 
+// ---- programmatic dependent launch --------------------------------------------------------------------------
+// Every kernel of the decode step calls grid_dependency_sync() before its first global-memory access: it blocks
+// until the preceding kernel of the stream has completed (its writes visible) and then lets the next kernel's
+// CTAs be scheduled early, where they block at the same call.  Launch latency and CTA start-up therefore overlap
+// the predecessor; data dependencies are untouched.  Without the launch attribute both instructions are no-ops.
+__device__ inline void grid_dependency_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// cudaLaunchKernelEx with programmatic stream serialization allowed and an optional cluster width
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  int cluster_x, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // ---- storage-type helpers -------------------------------------------------------------------------
 
 template <typename T>

@@ -43,6 +43,7 @@ __device__ __forceinline__ void online_update(float &m, float &s, float z) {
 
 __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_constant__ CUtensorMap tmap,
                                                                 ScanFastParams p) {
+  grid_dependency_sync();
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int kblocks = p.r >> 6;                    // 64-column blocks per row
@@ -316,7 +317,8 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
     smem_set = smem;
   }
   dim3 grid(p.cps, ly.B);
-  k_scan_sm100<<<grid, kScanThreads, smem, a.stream>>>(tmap, p);
+  cudaError_t le = launch_chained(k_scan_sm100, grid, dim3(kScanThreads), smem, a.stream, 1, tmap, p);
+  if (le != cudaSuccess) return le;
   ++launch_counter();
   return cudaGetLastError();
 }

@@ -76,6 +76,7 @@ __device__ __forceinline__ void pool_group(const float (&f)[12], float (&acc)[4]
 
 template <int MAXG>
 __global__ void __launch_bounds__(kRelThreads, 4) k_relevance(RelParams p) {
+  grid_dependency_sync();
   __shared__ float s_c[kMaxGroup];  // p = exp2(z * log2e + c), c = -M log2e - log2 S
   __shared__ float s_M[kMaxGroup], s_iS[kMaxGroup];
   __shared__ unsigned s_hist[2048];
@@ -290,6 +291,7 @@ __device__ inline unsigned find_bin(cg::cluster_group &cluster, unsigned *s_hist
 }
 
 __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
+  grid_dependency_sync();
   cg::cluster_group cluster = cg::this_cluster();
   const int CL = cluster.num_blocks();
   const int rank = cluster.block_rank();
@@ -461,10 +463,12 @@ cudaError_t launch_relevance(const StepArgs &a) {
   p.z_stride = a.plan.z_stride;
   const int per_cta = (kRelThreads / 32) * kRelOut * kRelChunks;
   dim3 grid((unsigned)((a.plan.max_len + per_cta - 1) / per_cta), a.ly.B);
+  cudaError_t le;
   if (a.ly.G <= 4)
-    k_relevance<4><<<grid, kRelThreads, 0, a.stream>>>(p);
+    le = launch_chained(k_relevance<4>, grid, dim3(kRelThreads), 0, a.stream, 1, p);
   else
-    k_relevance<8><<<grid, kRelThreads, 0, a.stream>>>(p);
+    le = launch_chained(k_relevance<8>, grid, dim3(kRelThreads), 0, a.stream, 1, p);
+  if (le != cudaSuccess) return le;
   ++launch_counter();
   return cudaGetLastError();
 }
@@ -488,19 +492,8 @@ cudaError_t launch_select(const StepArgs &a) {
     if (e != cudaSuccess) return e;
     smem_set = smem;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(a.plan.cluster, a.ly.B);
-  cfg.blockDim = dim3(kSelThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = a.stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = a.plan.cluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, k_select, p);
+  cudaError_t e = launch_chained(k_select, dim3(a.plan.cluster, a.ly.B), dim3(kSelThreads), smem, a.stream,
+                                 a.plan.cluster, p);
   if (e != cudaSuccess) return e;
   ++launch_counter();
   return cudaGetLastError();

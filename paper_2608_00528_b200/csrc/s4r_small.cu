@@ -65,6 +65,7 @@ __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4 &t, float (&
 
 template <typename T>
 __global__ void __launch_bounds__(256) k_project(ProjParams p) {
+  grid_dependency_sync();
   constexpr int V = Store<T>::kVec;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = cluster.block_rank(), CL = cluster.num_blocks();
@@ -217,19 +218,7 @@ static cudaError_t project_launch(const ProjParams &p, int B, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     smem_set = smem;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(kProjCluster, B);
-  cfg.blockDim = dim3(256);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = kProjCluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, k_project<T>, p);
+  cudaError_t e = launch_chained(k_project<T>, dim3(kProjCluster, B), dim3(256), smem, st, kProjCluster, p);
   if (e != cudaSuccess) return e;
   ++launch_counter();
   return cudaGetLastError();
@@ -269,6 +258,7 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // grid (Hq, B), block dh threads: thread i owns channel i of the head
 template <typename T>
 __global__ void __launch_bounds__(128) k_merge(MergeParams p) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) uint8_t msm[];
   const int h = blockIdx.x, b = blockIdx.y, i = threadIdx.x, dh = p.dh, nthr = dh;
   const int kv = h / p.G, half = dh >> 1, lane = i & 31, warp = i >> 5, nwarp = dh >> 5;
@@ -453,21 +443,23 @@ cudaError_t launch_merge(const StepArgs &a) {
   const size_t smem = esz * (size_t)ly.dh * (1 + 2 * (size_t)ly.s) + sizeof(float) * kMergeTiles * ly.dh +
                       sizeof(float2) * kMergeTiles + sizeof(float) * (4 * 64 + 64) + 16;
   dim3 grid(ly.Hq, ly.B);
+  cudaError_t le;
   if (ly.dtype == S4R_BF16) {
     static size_t set_b = 0;
     if (smem > 48 * 1024 && smem > set_b) {
       cudaFuncSetAttribute(k_merge<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       set_b = smem;
     }
-    k_merge<__nv_bfloat16><<<grid, ly.dh, smem, a.stream>>>(p);
+    le = launch_chained(k_merge<__nv_bfloat16>, grid, dim3(ly.dh), smem, a.stream, 1, p);
   } else {
     static size_t set_f = 0;
     if (smem > 48 * 1024 && smem > set_f) {
       cudaFuncSetAttribute(k_merge<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       set_f = smem;
     }
-    k_merge<float><<<grid, ly.dh, smem, a.stream>>>(p);
+    le = launch_chained(k_merge<float>, grid, dim3(ly.dh), smem, a.stream, 1, p);
   }
+  if (le != cudaSuccess) return le;
   ++launch_counter();
   return cudaGetLastError();
 }
