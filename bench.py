@@ -131,7 +131,7 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(sm), "source": self.source}
 
 
-def build_cache(cfg, s4r, device, capacity):
+def build_cache(cfg, s4r, device, capacity, seq_ids):
     """Synthetic prompt -> bases (set-up) -> s4r_compress.  Returns the device-resident cache and timings."""
     st = W.storage_dtype(cfg)
     B, s, D = cfg.batch, cfg.sink_count, cfg.d_kv
@@ -142,13 +142,12 @@ def build_cache(cfg, s4r, device, capacity):
     BK = torch.empty(B, D, cfg.rank_k, dtype=st, device=device)
     BV = torch.empty(B, D, cfg.rank_v, dtype=st, device=device)
     q = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=st, device=device)
-    rank_off = int(os.environ.get("RANK", "0")) * B          # every rank draws its own sequences
-    for b in range(B):
-        K[b] = W.make_kv(cfg, 0, rank_off + b, "k", device=device)
-        V[b] = W.make_kv(cfg, 0, rank_off + b, "v", device=device)
-        BK[b] = W.make_bench_basis(K[b][W.sample_rows(cfg, 0, rank_off + b, "k").to(device)], cfg.rank_k, st)
-        BV[b] = W.make_bench_basis(V[b][W.sample_rows(cfg, 0, rank_off + b, "v").to(device)], cfg.rank_v, st)
-        q[b] = W.make_query(cfg, K[b], 0, rank_off + b)
+    for b, sid in enumerate(seq_ids):                        # every rank draws its own sequences
+        K[b] = W.make_kv(cfg, 0, sid, "k", device=device)
+        V[b] = W.make_kv(cfg, 0, sid, "v", device=device)
+        BK[b] = W.make_bench_basis(K[b][W.sample_rows(cfg, 0, sid, "k").to(device)], cfg.rank_k, st)
+        BV[b] = W.make_bench_basis(V[b][W.sample_rows(cfg, 0, sid, "v").to(device)], cfg.rank_v, st)
+        q[b] = W.make_query(cfg, K[b], 0, sid)
     sink_k = torch.empty(B, s, D, dtype=st, device=device)
     sink_v = torch.empty_like(sink_k)
     CK = torch.zeros(B, capacity, cfg.rank_k, dtype=st, device=device)
@@ -242,9 +241,9 @@ def main():
         return run_reference(args, cfg)
 
     import paper_2608_00528_b200 as s4r
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2608_00528_b200 import replicas
+    rep = replicas.replica_from_env()
+    rank, local_rank, world = rep.rank, rep.local_rank, rep.world
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -257,7 +256,8 @@ def main():
     K_steps, Wm = args.steps, max(args.warmup, 3)
     n_append = 2 * (K_steps + Wm) + 8
     capacity = cfg.cache_len + n_append
-    c = build_cache(cfg, s4r, device, capacity)
+    seq_ids = replicas.sequence_ids(rep, cfg.batch)
+    c = build_cache(cfg, s4r, device, capacity, seq_ids)
     ly, B = c["ly"], cfg.batch
     st = W.storage_dtype(cfg)
     n_sel = cfg.window + cfg.top_k
@@ -267,8 +267,8 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=device)
     # per-step inputs: one new (k_t, v_t, q) triple per step, cycled from a small pool
     pool = 4
-    kt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "k", i + 1, device) for b in range(B)]) for i in range(pool)])
-    vt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "v", i + 1, device) for b in range(B)]) for i in range(pool)])
+    kt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "k", i + 1, device) for b in seq_ids]) for i in range(pool)])
+    vt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "v", i + 1, device) for b in seq_ids]) for i in range(pool)])
     qs = torch.stack([c["q"] * (1.0 + 0.01 * i) for i in range(pool)]).to(st)
     kw = dict(pool_kernel=cfg.pool_kernel, pool_mode={"max": s4r.POOL_MAX, "avg": s4r.POOL_AVG}[cfg.pool_mode],
               group_mode={"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode], rope_theta=cfg.rope_theta,
@@ -304,10 +304,7 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
     gpu_launches = launches[0]
-    if dist is not None:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = replicas.max_over_ranks(ms_total, dist, device)
     ms_step = ms_total / K_steps
 
     # ---- per-stage device times of the same steps (second pass; events recorded inside the library on the
@@ -349,10 +346,7 @@ def main():
         step_e2e(3 + i)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = replicas.max_over_ranks(e2e_s, dist, device)
     esz = cfg.elem_bytes
     h2d = B * (cfg.n_q_heads * cfg.head_dim + 2 * cfg.d_kv) * esz
     d2h = B * (cfg.n_q_heads * cfg.head_dim * 4 + n_sel * 4 + 4)
@@ -372,7 +366,7 @@ def main():
     m = cfg.window + cfg.top_k
     step_bytes = B * (L_now * cfg.rank_k + m * (cfg.rank_k + cfg.rank_v) + 2 * cfg.sink_count * cfg.d_kv) * esz
     line = {
-        "metric": METRIC, "value": world * 1e3 / ms_step, "unit": UNIT, "n_gpus": world, "steps": K_steps,
+        "metric": METRIC, "value": replicas.whole_job_rate(K_steps, world, ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K_steps,
         "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "batch_per_gpu": B, "global_batch": B * world, "context": cfg.context,
@@ -392,7 +386,7 @@ def main():
         "stage_ms": stage_ms,
         "compress": {"ms": c["compress_ms"], "tokens_per_s": B * (cfg.context - cfg.sink_count) / (c["compress_ms"] * 1e-3),
                      "launches": c["compress_launches"]},
-        "e2e": {"value": world * K_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": {"value": replicas.whole_job_rate(K_steps, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": gpu_launches, "clocks": clocks, "dev_status": dev_flags,
     }
     if not args.no_cpu_baseline and world == 1:
