@@ -218,7 +218,8 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (cuda_failed(launch_relevance(a))) return S4R_ERR_CUDA;
   if (cuda_failed(launch_select(a))) return S4R_ERR_CUDA;
   stage_mark(3, a.stream);
-  const bool absorb = att_fast_supported(ly) && a.value_path == S4R_VALUE_AUTO;
+  // the absorbed kernel keeps U in tensor-memory columns [256, 256 + r_v) below the logit buffers at 480
+  const bool absorb = att_fast_supported(ly) && ly.rv <= 192 && a.value_path == S4R_VALUE_AUTO;
   if (absorb) {
     if (cuda_failed(launch_attend_absorb(a))) return S4R_ERR_CUDA;
   } else if (att_fast_supported(ly)) {

@@ -12,7 +12,8 @@
 //   K^[tokens x d_h] = C^K[rows] (B^K slice)^T   tcgen05.mma, basis slice streamed through a TMA ring
 //   logits, tile softmax                         16 epilogue warps, RoPE angles held in registers
 //   U[2G x r_v]      = [P_hi; P_lo]^T C^V[rows]  tcgen05.mma, probabilities as two bf16 terms (hi + lo)
-// Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-17 = epilogue.
+// Warp 0 = key-basis TMA stream + issuer of the key product, warp 1 = issuer of the logit product,
+// warps 2-17 = epilogue, warp 18 = issuer of the P C^V product.
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
 
@@ -20,17 +21,20 @@ namespace s4r {
 
 using namespace sm100;
 
-void fill_inv_freq(double *dst, int head_dim, float theta);
+void fill_rope_turns(uint64_t *dst, int head_dim, float theta);
 
 namespace {
 
 constexpr int kTok = 128;
 constexpr int kDh = 128;
-constexpr int kRing = 3;
+constexpr int kRing = 6;                 // key-basis blocks in flight (two heads at r_k = 192)
+constexpr int kPopBlk = 16 * 128;        // stored part of one 64-token block of the probability operand: 16 rows
 constexpr int kBlkBytes = 128 * 128;
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kThreads = 64 + kEpiThreads;
+constexpr int kThreads = 64 + kEpiThreads + 32;
+constexpr int kQopBytes = 2 * 16 * 128;  // one head's query operand: two 64-channel blocks of 16 rows
+constexpr uint32_t kUCol = 256, kZCol = 480;  // tensor-memory columns of U and of the two logit buffers
 
 struct AbsorbParams {
   const __nv_bfloat16 *q, *coef_k, *coef_v;
@@ -41,8 +45,22 @@ struct AbsorbParams {
   int64_t cap, max_len;
   float theta;
   int32_t *dev_status;
-  double inv_freq[64];
+  uint64_t rope_turns[64];
 };
+
+// (sin, cos) of pos * inv_freq as two biased 16-bit fixed-point numbers, value = (u - 32768) / 32768, with no
+// integer<->float conversion instruction: the top 23 bits of the turn fraction become the mantissa of a float in
+// [1, 2), the angle minus pi follows from one FMA, and the rounding to fixed point uses the 2^23 trick.
+__device__ __forceinline__ uint32_t pack_sincos(int pos, uint64_t turns) {
+  const uint64_t ph = (uint64_t)(uint32_t)pos * turns;                     // fraction of a turn, 0.64 fixed point
+  const float x = __uint_as_float(0x3F800000u | (uint32_t)(ph >> 41));     // 1 + fraction
+  float sn, cs;
+  __sincosf(fmaf(x, 6.28318530718f, -9.42477796077f), &sn, &cs);           // angle - pi: both signs flip
+  const float kTop = 8388608.f + 65535.f;
+  const float fs = fminf(fmaf(-sn, 32768.f, 8388608.f + 32768.f), kTop);
+  const float fc = fminf(fmaf(-cs, 32768.f, 8388608.f + 32768.f), kTop);
+  return (__float_as_uint(fs) & 0xffffu) | (__float_as_uint(fc) << 16);
+}
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 __device__ __forceinline__ float2 bcast2(float v) { return make_float2(v, v); }
@@ -53,33 +71,34 @@ __device__ __forceinline__ void cp_async16_zfill(void *dst, const void *src, boo
 
 __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_constant__ CUtensorMap tmap_bk,
                                                                const __grid_constant__ AbsorbParams p) {
-  grid_dependency_sync();
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int kbk = p.rk >> 6, kbv = p.rv >> 6, G = p.G;
   uint8_t *ck = smem;                                   // [kbk][128 tokens][128 B]   A of the K^ product
   uint8_t *cv = ck + (size_t)kbk * kBlkBytes;           // [kbv][128 tokens][128 B]   B (N-contiguous) of P C^V
-  uint8_t *ring = cv + (size_t)kbv * kBlkBytes;         // [kRing][128 d][128 B]      key-basis blocks
-  uint8_t *pop = ring + (size_t)kRing * kBlkBytes;      // [2][128 rows][128 B]       A of P C^V: rows g / G+g = hi / lo
-  float *qs = reinterpret_cast<float *>(pop + 2 * kBlkBytes);   // [128 cols][8]
-  float *xch = qs + kDh * kMaxGroup;                             // [4 quarters][G][128]
-  uint64_t *bars = reinterpret_cast<uint64_t *>(xch + 4 * G * 128);
+  // A of P C^V: rows g / G+g = hi / lo part of the probabilities.  Only 16 of the operand's 128 rows are stored;
+  // the product reads the other rows from whatever follows (the ring), and their output lanes are never read.
+  // Two copies, alternating by head, so that a head's softmax does not wait for the previous head's product.
+  uint8_t *pop = cv + (size_t)kbv * kBlkBytes;          // [2 heads][2 x 64 tokens][16 rows][128 B]
+  uint8_t *ring = pop + 4 * kPopBlk;                    // [kRing][128 d][128 B]      key-basis blocks
+  uint8_t *qop = ring + (size_t)kRing * kBlkBytes;      // [2 heads][2 x 64 d][16 rows][128 B]  B of the logit product:
+                                                        //   rows g / 8+g = hi / lo part of q'[g]
+  float *xch = reinterpret_cast<float *>(qop + 2 * kQopBytes);   // [2 heads][G][128 tokens] logits
+  uint64_t *bars = reinterpret_cast<uint64_t *>(xch + 2 * G * 128);
   uint64_t *full = bars, *empty = bars + kRing;
-  uint64_t *k_full = bars + 2 * kRing, *k_empty = k_full + 2;
-  uint64_t *p_ready = k_empty + 2, *u_full = p_ready + 1, *u_empty = u_full + 1;
+  uint64_t *k_full = bars + 2 * kRing, *rope_done = k_full + 2;
+  uint64_t *z_full = rope_done + 2, *z_empty = z_full + 2;
+  uint64_t *p_ready = z_empty + 2, *u_full = p_ready + 1, *u_empty = u_full + 2;  // u_full[2]: by head parity
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(u_empty + 1);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   int *rows = reinterpret_cast<int *>(tmem_slot + 2);   // [128]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, kv0 = blockIdx.y * p.nkv, b = blockIdx.z;
-  const int count = min(p.sel_count[b], p.sel_stride);
-  const int t0 = tile * kTok;
-  if (t0 >= count) return;  // uniform over the CTA
-  const int nt = min(kTok, count - t0);
-  int L = p.coef_len[b];
-  L = L < 0 ? 0 : (L > p.max_len ? (int)p.max_len : L);
+  // the ring holds whole heads: stage s = blocks [s kbk, (s+1) kbk), one full/empty barrier pair per stage
+  const int n_stages = kRing / kbk > 0 ? kRing / kbk : 1;
 
+  // ---- set-up that touches no global memory runs before the wait on the preceding kernel
   if (tid == 0) {
     for (int i = 0; i < kRing; ++i) {
       mbar_init(&full[i], 1);
@@ -87,17 +106,27 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&k_full[i], 1);
-      mbar_init(&k_empty[i], kEpiWarps);
+      mbar_init(&rope_done[i], kEpiWarps);
+      mbar_init(&z_full[i], 1);
+      mbar_init(&z_empty[i], 4);  // one warp per lane quadrant reads the logits
     }
-    mbar_init(p_ready, 1);
-    mbar_init(u_full, 1);
-    mbar_init(u_empty, 4);  // the four warps of lane quadrant 0 read U
+    mbar_init(p_ready, (uint32_t)G);  // one softmax warp per query head of the group
+    mbar_init(&u_full[0], 1);
+    mbar_init(&u_full[1], 1);
+    mbar_init(u_empty, 3);  // three warps of lane quadrant 0 read U
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tmap_bk);
   }
   if (warp == 1) tmem_alloc(tmem_slot, 512);
-  if (tid < kTok) {
+  grid_dependency_sync();
+  const int count = min(p.sel_count[b], p.sel_stride);
+  const int t0 = tile * kTok;
+  const bool active = t0 < count;  // uniform over the CTA
+  const int nt = min(kTok, count - t0);
+  int L = p.coef_len[b];
+  L = L < 0 ? 0 : (L > p.max_len ? (int)p.max_len : L);
+  if (tid < kTok && active) {
     int rix = (tid < nt) ? p.sel_idx[(size_t)b * p.sel_stride + t0 + tid] : -1;
     rows[tid] = rix < 0 ? -1 : min(rix, max(L - 1, 0));
   }
@@ -105,10 +134,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (!active) {
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+    return;
+  }
 
   if (warp != 0) {
     // ---- gather the selected coefficient rows (asynchronous 16-byte pieces, all in flight at once; rows past
-    //      the tile's end are zero) and clear the probability operand, while the producer fills the ring
+    //      the tile's end are zero) and clear the probability and query operands, while the producer fills the ring
     constexpr int kWorkers = kThreads - 32;
     const int wt = tid - 32;
     const int cpr_k = p.rk >> 3, cpr_v = p.rv >> 3;
@@ -125,75 +158,128 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
                        reinterpret_cast<const uint4 *>(cvb + (size_t)max(rix, 0) * p.rv) + c, rix >= 0);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int i = wt; i < 2 * kBlkBytes / 16; i += kWorkers) reinterpret_cast<uint4 *>(pop)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = wt; i < 4 * kPopBlk / 16; i += kWorkers) reinterpret_cast<uint4 *>(pop)[i] = make_uint4(0, 0, 0, 0);
   }
 
+  // Three threads issue the tensor-core work, one per product and each in a warp of a different SM
+  // sub-partition, so that no product waits behind another one's barrier or issue slots.  Tensor-memory columns:
+  // [0, 256) two K^ buffers (fp32, then overwritten in place by the rotated rows as hi + lo bf16),
+  // [256, 256 + r_v) U, [480, 512) two logit buffers of 16 columns.
   if (warp == 0) {
-    // ---------------- TMA producer: key-basis slices in 64-column blocks ----------------
+    // ---------------- key-basis stream (TMA, 64-column blocks, whole heads per stage) and K^ = C^K_tile (B^K)^T
     if (lane == 0) {
-      int it = 0, issued = 0;
-      bool ok = true;
-      for (int h = 0; h < p.nkv && ok; ++h) {
-        const int y = b * p.D + (kv0 + h) * kDh;
-        for (int blk = 0; blk < kbk; ++blk, ++it) {
-          const int slot = it % kRing;
-          if (!mbar_wait(&empty[slot], ((uint32_t)(it / kRing) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(&full[slot], kBlkBytes);
-          tma_load_2d(ring + (size_t)slot * kBlkBytes, &tmap_bk, blk * 64, y, &full[slot]);
-          issued = it + 1;
+      const int pre = min(n_stages, p.nkv);
+      for (int h = 0; h < pre; ++h) {  // fresh stages: no wait
+        mbar_expect_tx(&full[h], (uint32_t)kbk * kBlkBytes);
+        for (int blk = 0; blk < kbk; ++blk)
+          tma_load_2d(ring + (size_t)(h * kbk + blk) * kBlkBytes, &tmap_bk, blk * 64, b * p.D + (kv0 + h) * kDh, &full[h]);
+      }
+    }
+    __syncwarp();
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");  // tiles gathered, operands cleared, q' of head 0 set
+    if (lane == 0) {
+      const uint32_t idesc_k = umma_idesc_bf16(128, 128);
+      const uint64_t ck_desc = umma_desc_sw128(smem_u32(ck));
+      int hp = min(n_stages, p.nkv), hk = 0;  // next head to load / to multiply
+      unsigned long long t_idle = 0;
+      int spins = 0;
+      while (hk < p.nkv) {
+        bool progress = false;
+        if (hp < p.nkv) {
+          const int st = hp % n_stages;
+          if (mbar_test(&empty[st], ((uint32_t)(hp / n_stages) & 1u) ^ 1u)) {
+            mbar_expect_tx(&full[st], (uint32_t)kbk * kBlkBytes);
+            for (int blk = 0; blk < kbk; ++blk)
+              tma_load_2d(ring + (size_t)(st * kbk + blk) * kBlkBytes, &tmap_bk, blk * 64, b * p.D + (kv0 + hp) * kDh,
+                          &full[st]);
+            ++hp;
+            progress = true;
+          }
+        }
+        {
+          // K^ of head hk overwrites the buffer that the logit product of head hk - 2 reads: wait for that product
+          const int buf = hk & 1, st = hk % n_stages;
+          if (mbar_test(&full[st], (uint32_t)(hk / n_stages) & 1u) &&
+              (hk < 2 || mbar_test(&z_full[buf], (uint32_t)((hk - 2) >> 1) & 1u))) {
+            tc_fence_after();
+            const uint64_t bs_desc = umma_desc_sw128(smem_u32(ring + (size_t)st * kbk * kBlkBytes));
+            for (int blk = 0; blk < kbk; ++blk) {
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4)
+                umma_bf16(tmem_base + (uint32_t)buf * 128, ck_desc + (uint64_t)((blk * kBlkBytes + k4 * 32) >> 4),
+                          bs_desc + (uint64_t)((blk * kBlkBytes + k4 * 32) >> 4), idesc_k, (blk | k4) != 0);
+            }
+            umma_commit(&empty[st]);
+            umma_commit(&k_full[buf]);
+            ++hk;
+            progress = true;
+          }
+        }
+        if (progress) {
+          spins = 0;
+        } else {
+          const int st = hk % n_stages;
+          if (!mbar_test(&full[st], (uint32_t)(hk / n_stages) & 1u))
+            mbar_try_wait_ns(&full[st], (uint32_t)(hk / n_stages) & 1u, 500u);
+          else
+            mbar_try_wait_ns(&z_full[hk & 1], (uint32_t)((hk - 2) >> 1) & 1u, 500u);
+          if ((++spins & 15) == 0) {
+            if (*abort_flag) break;
+            const unsigned long long now = global_ns();
+            if (spins == 16) t_idle = now;
+            if (now - t_idle > kWaitLimitNs) { *abort_flag = 1; break; }
+          }
         }
       }
-      if (*abort_flag) {
-        for (int i = max(0, issued - kRing); i < issued; ++i) {
+      if (*abort_flag) {  // let the copies in flight land before the CTA leaves
+        for (int h = max(0, hp - n_stages); h < hp; ++h) {
           const unsigned long long t_0 = global_ns();
-          while (!mbar_try_wait(&full[i % kRing], (uint32_t)(i / kRing) & 1u))
+          while (!mbar_try_wait(&full[h % n_stages], (uint32_t)(h / n_stages) & 1u))
             if (global_ns() - t_0 > kWaitLimitNs) break;
         }
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+    // ---------------- logits[token, n] = sum_d K'[token, d] q'[n, d]; K' = rotated K^ as hi + lo bf16 in tensor memory
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     fence_proxy_async_smem();
-    asm volatile("bar.sync 2, %0;" ::"n"(kThreads - 32) : "memory");  // tiles gathered, operand cleared
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
     if (lane == 0) {
-      const uint32_t idesc_k = umma_idesc_bf16(128, 128);
+      const uint32_t idesc_z = umma_idesc_bf16(128, 16);
+      for (int h = 0; h < p.nkv; ++h) {
+        const int buf = h & 1;
+        const uint32_t ph = (uint32_t)(h >> 1) & 1u;
+        if (!mbar_wait(&rope_done[buf], ph, abort_flag)) break;
+        if (!mbar_wait(&z_empty[buf], ph ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint64_t q_desc = umma_desc_sw128(smem_u32(qop + (size_t)buf * kQopBytes));
+#pragma unroll
+        for (int st = 0; st < 16; ++st) {
+          const int ks = st >> 1, part = st & 1;  // K-step ks = channels {8 ks .. +7, 64 + 8 ks .. +7}; hi or lo
+          umma_bf16_ts(tmem_base + kZCol + (uint32_t)buf * 16, tmem_base + (uint32_t)(buf * 128 + part * 64 + ks * 8),
+                       q_desc + (uint64_t)(((ks >> 2) * 2048 + (ks & 3) * 32) >> 4), idesc_z, st != 0);
+        }
+        umma_commit(&z_full[buf]);
+      }
+    }
+  } else if (warp == 2 + kEpiWarps) {
+    // ---------------- U = [P_hi; P_lo]^T C^V over the 128 tokens of the tile (8 steps of 16 tokens)
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    fence_proxy_async_smem();
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
+    if (lane == 0) {
       const uint32_t idesc_u = umma_idesc_bf16(128, p.rv) | (1u << 16);  // B operand N-contiguous
-      const uint64_t ck_desc = umma_desc_sw128(smem_u32(ck));
       const uint64_t cv_desc = umma_desc_mn_sw128(smem_u32(cv), kBlkBytes);
       const uint64_t pop_desc = umma_desc_sw128(smem_u32(pop));
-      int it = 0;
-      bool ok = true;
-      auto issue_k = [&](int h) {
-        const int buf = h & 1;
-        if (!mbar_wait(&k_empty[buf], ((uint32_t)(h >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; return; }
-        tc_fence_after();
-        for (int blk = 0; blk < kbk; ++blk, ++it) {
-          const int slot = it % kRing;
-          if (!mbar_wait(&full[slot], (uint32_t)(it / kRing) & 1u, abort_flag)) { ok = false; return; }
-          tc_fence_after();
-          const uint64_t bs_desc = umma_desc_sw128(smem_u32(ring + (size_t)slot * kBlkBytes));
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            umma_bf16(tmem_base + (uint32_t)buf * 128, ck_desc + (uint64_t)((blk * kBlkBytes + k4 * 32) >> 4),
-                      bs_desc + (uint64_t)((k4 * 32) >> 4), idesc_k, (blk | k4) != 0);
-          umma_commit(&empty[slot]);
-        }
-        umma_commit(&k_full[buf]);
-      };
-      issue_k(0);
-      for (int h = 0; h < p.nkv && ok; ++h) {
-        if (h + 1 < p.nkv) issue_k(h + 1);  // the key product runs one head ahead of the epilogue
-        if (!ok) break;
-        // U = [P_hi; P_lo]^T C^V over the 128 tokens of the tile (8 steps of 16 tokens)
+      for (int h = 0; h < p.nkv; ++h) {
         if (!mbar_wait(p_ready, (uint32_t)h & 1u, abort_flag)) break;
         if (!mbar_wait(u_empty, ((uint32_t)h & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          umma_bf16(tmem_base + 256u, pop_desc + (uint64_t)(((kk >> 2) * kBlkBytes + (kk & 3) * 32) >> 4),
+          umma_bf16(tmem_base + kUCol, pop_desc + (uint64_t)((((h & 1) * 2 + (kk >> 2)) * kPopBlk + (kk & 3) * 32) >> 4),
                     cv_desc + (uint64_t)((kk * 2048) >> 4), idesc_u, kk != 0);
-        umma_commit(u_full);
+        umma_commit(&u_full[h & 1]);
       }
     }
   } else {
@@ -202,61 +288,132 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
     const int quad = warp & 3, qt = e >> 2;
     const int lane_row = quad * 32 + lane;   // token owned by this thread
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const int npair = (G + 1) >> 1;
     const bool rope = p.theta > 0.f;
+    const int nsync = (G > 4 ? 8 : 4 + G) * 32;  // threads of the logit readers (4 <= e < 8) and the softmax warps (e < G)
     // RoPE angles of this thread's token for its 16 pairs, kept in registers for all heads
-    // (sin, cos) packed as two 16-bit fixed-point numbers (absolute error 1.5e-5, far below bf16 resolution)
+    // (sin, cos) packed as two biased 16-bit fixed-point numbers, value = (u - 32768) / 32768 (absolute error
+    // 1.5e-5, far below bf16 resolution); unpacked with a byte permute and one FMA, no integer conversion
     uint32_t sc[16];
     {
       const int rix = rows[lane_row];
 #pragma unroll
-      for (int ii = 0; ii < 16; ++ii) {
-        float sn = 0.f, cs = 1.f;
-        if (rope && rix >= 0) rope_sincos(p.s + rix, p.inv_freq[qt * 16 + ii], sn, cs);
-        sc[ii] = ((uint32_t)__float2int_rn(sn * 32767.f) & 0xffffu) | ((uint32_t)__float2int_rn(cs * 32767.f) << 16);
-      }
+      for (int ii = 0; ii < 16; ++ii)
+        sc[ii] = (rope && rix >= 0) ? pack_sincos(p.s + rix, p.rope_turns[qt * 16 + ii]) : 0xffff8000u;  // (0, 1)
     }
-    // q' = RoPE(q) / sqrt(d_h), laid out [col][g]; this thread prepares column qc for the heads g = qg0, qg0 + 4.
-    // The raw values of the next KV head are fetched one head ahead.
+    // q' = RoPE(q) / sqrt(d_h) as hi + lo bf16 rows of the logit product's B operand; this thread prepares column
+    // qc for the heads g = qg0, qg0 + 4.  The raw values are fetched one head ahead of their use.
     const int qc = et & 127, qg0 = et >> 7;
     float q_sn = 0.f, q_cs = 1.f;
-    if (rope) rope_sincos(p.s + L - 1, p.inv_freq[qc & 63], q_sn, q_cs);
+    if (rope) rope_sincos(p.s + L - 1, p.rope_turns[qc & 63], q_sn, q_cs);
     const float q_scale = rsqrtf((float)kDh);
-    float q_raw[2][2];  // [g slot][own, partner]
+    // raw bf16 bits; widened only where they are used, so that the loads stay in flight across a whole head
+    unsigned short q_raw[2][2];  // [g slot][own, partner]
     auto fetch_q = [&](int h) {
 #pragma unroll
       for (int sl = 0; sl < 2; ++sl) {
         const int g = qg0 + 4 * sl;
-        q_raw[sl][0] = q_raw[sl][1] = 0.f;
+        q_raw[sl][0] = q_raw[sl][1] = 0;
         if (g < G && h < p.nkv) {
-          const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)(kv0 + h) * G + g) * kDh;
-          q_raw[sl][0] = __bfloat162float(qp[qc]);
-          q_raw[sl][1] = __bfloat162float(qp[qc ^ 64]);
+          const unsigned short *qp =
+              reinterpret_cast<const unsigned short *>(p.q + ((size_t)b * p.Hq + (size_t)(kv0 + h) * G + g) * kDh);
+          q_raw[sl][0] = __ldg(qp + qc);
+          q_raw[sl][1] = __ldg(qp + (qc ^ 64));
         }
       }
     };
-    auto store_q = [&]() {
+    // position of channel qc in the K order of the logit product: steps of {8 channels of the lower half of the
+    // head, their 8 rotation partners}
+    const int q_col = ((qc & 63) >> 3) * 16 + (qc >> 6) * 8 + (qc & 7);
+    auto store_q = [&](int h) {
+      uint8_t *qb = qop + (size_t)(h & 1) * kQopBytes + (size_t)(q_col >> 6) * 2048;
 #pragma unroll
       for (int sl = 0; sl < 2; ++sl) {
-        float v = q_raw[sl][0];
-        if (rope) v = (qc < 64) ? v * q_cs - q_raw[sl][1] * q_sn : v * q_cs + q_raw[sl][1] * q_sn;
-        qs[qc * kMaxGroup + qg0 + 4 * sl] = v * q_scale;
+        const int g = qg0 + 4 * sl;
+        if (g < G) {
+          float v = __uint_as_float((uint32_t)q_raw[sl][0] << 16);
+          const float o = __uint_as_float((uint32_t)q_raw[sl][1] << 16);
+          if (rope) v = (qc < 64) ? v * q_cs - o * q_sn : v * q_cs + o * q_sn;
+          v *= q_scale;
+          const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+          *reinterpret_cast<__nv_bfloat16 *>(qb + sw128_offset(g, q_col & 63)) = hi;
+          *reinterpret_cast<__nv_bfloat16 *>(qb + sw128_offset(8 + g, q_col & 63)) = lo;
+        }
       }
     };
-    // U of one head: TMEM lanes 0..G-1 hold the hi part, G..2G-1 the lo part; the four warps of quadrant 0 split
-    // the columns and store both parts (k_merge_absorb adds them)
-    auto read_u = [&](int h, bool ok_in) -> bool {
+    // K^ row of this thread's token, pairs [16 qt, +16), in two halves of 8 pairs (d1 = 16 qt + 8 half + j,
+    // d2 = d1 + 64): rotate, split into hi + lo bf16 by truncation (hi = upper 16 bits of the fp32 value, lo =
+    // upper 16 bits of the exact remainder; together 16 significand bits) and write back over the half's own 16
+    // accumulator columns: [c, c+4) hi of d1, [c+4, c+8) hi of d2, [c+64, c+68) lo of d1, [c+68, c+72) lo of d2,
+    // two values per column with the even channel in the low half.  A K-step of the logit product is therefore
+    // the 16 channels {d1 .. d1+7, d2 .. d2+7}; q' is stored in the same order (q_col).
+    auto rotate = [&](int h, bool ok_in) -> bool {
+      const int buf = h & 1;
       bool ok2 = ok_in;
-      if (ok2) ok2 = mbar_wait(u_full, (uint32_t)h & 1u, abort_flag);
+      if (ok2) ok2 = mbar_wait(&k_full[buf], (uint32_t)(h >> 1) & 1u, abort_flag);
       ok2 = __all_sync(0xffffffffu, ok2);
       tc_fence_after();
       if (ok2) {
-        const int cper = p.rv >> 2;  // columns per warp, a multiple of 16
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t ka[8], kb[8];
+          const uint32_t base = tmem_base + (uint32_t)buf * 128 + lane_addr + (uint32_t)(qt * 16 + half * 8);
+          tmem_ld8(base, ka);
+          tmem_ld8(base + 64, kb);
+          tmem_ld_wait();
+          if (rope) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t w = sc[half * 8 + j];
+              // 0x4B000000 | u is the float 2^23 + u; times 2^-15 minus 257 gives (u - 32768) / 32768 exactly
+              const float2 scf = __ffma2_rn(make_float2(__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7410)),
+                                                        __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7432))),
+                                            bcast2(1.f / 32768.f), bcast2(-257.f));
+              const float2 k12 = make_float2(__uint_as_float(ka[j]), __uint_as_float(kb[j]));
+              const float2 r = __ffma2_rn(make_float2(-k12.y, k12.x), bcast2(scf.x), __fmul2_rn(k12, bcast2(scf.y)));
+              ka[j] = __float_as_uint(r.x);
+              kb[j] = __float_as_uint(r.y);
+            }
+          }
+          uint32_t hi[8], lo[8];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t a0 = ka[2 * j], a1 = ka[2 * j + 1], b0 = kb[2 * j], b1 = kb[2 * j + 1];
+            hi[j] = __byte_perm(a0, a1, 0x7632);
+            hi[4 + j] = __byte_perm(b0, b1, 0x7632);
+            const float ra0 = __uint_as_float(a0) - __uint_as_float(a0 & 0xffff0000u);
+            const float ra1 = __uint_as_float(a1) - __uint_as_float(a1 & 0xffff0000u);
+            const float rb0 = __uint_as_float(b0) - __uint_as_float(b0 & 0xffff0000u);
+            const float rb1 = __uint_as_float(b1) - __uint_as_float(b1 & 0xffff0000u);
+            lo[j] = __byte_perm(__float_as_uint(ra0), __float_as_uint(ra1), 0x7632);
+            lo[4 + j] = __byte_perm(__float_as_uint(rb0), __float_as_uint(rb1), 0x7632);
+          }
+          tmem_st8(base, hi);
+          tmem_st8(base + 64, lo);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&rope_done[buf]);
+      return ok2;
+    };
+    // U of one head: TMEM lanes 0..G-1 hold the hi part, G..2G-1 the lo part; three warps of lane quadrant 0 that
+    // have no part in the softmax (e = 6, 10, 14) split the columns and store both parts
+    // (k_merge_absorb adds them)
+    const bool u_reader = (e == 6 || e == 10 || e == 14);
+    const int u_part = (e - 6) >> 2;
+    auto read_u = [&](int h, bool ok_in) -> bool {
+      bool ok2 = ok_in;
+      if (ok2) ok2 = mbar_wait(&u_full[h & 1], (uint32_t)(h >> 1) & 1u, abort_flag);
+      ok2 = __all_sync(0xffffffffu, ok2);
+      tc_fence_after();
+      if (ok2) {
         const int part = lane < G ? 0 : 1, g = lane < G ? lane : lane - G;
         float *dst = p.part_u + ((((size_t)b * p.Hq + (size_t)(kv0 + h) * G + min(g, G - 1)) * p.n_tiles + tile) * 2 + part) * p.rv;
-        for (int c0 = qt * cper; c0 < (qt + 1) * cper; c0 += 16) {
+        for (int c0 = u_part * 16; c0 < p.rv; c0 += 48) {
           uint32_t v[16];
-          tmem_ld16(tmem_base + 256u + (uint32_t)c0, v);
+          tmem_ld16(tmem_base + kUCol + (uint32_t)c0, v);
           tmem_ld_wait();
           if (lane < 2 * G) {
 #pragma unroll
@@ -272,73 +429,59 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
       return ok2;
     };
     fetch_q(0);
+    for (int i = et; i < 2 * kQopBytes / 16; i += kEpiThreads) reinterpret_cast<uint4 *>(qop)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    fence_proxy_async_smem();
-    store_q();
+    epi_sync();  // query operand cleared (rows past G stay zero)
+    store_q(0);
     fetch_q(1);
-    asm volatile("bar.sync 2, %0;" ::"n"(kThreads - 32) : "memory");  // tiles gathered, operand cleared, q' of head 0 set
+    fence_proxy_async_smem();
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");  // tiles gathered, operands cleared, q' of head 0 set
     bool ok = true;  // warp-uniform; after a failed wait the loop keeps its shape but touches tensor memory no more
+    ok = rotate(0, ok);
     for (int h = 0; h < p.nkv; ++h) {
-      const int kv = kv0 + h, buf = h & 1;
-      const uint32_t aph = (uint32_t)(h >> 1) & 1u;
-      // ---- K^ row of this thread's token: pairs [16*qt, +16)
-      if (ok) ok = mbar_wait(&k_full[buf], aph, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      tc_fence_after();
-      float2 lg[4];
+      const int kv = kv0 + h, zb = h & 1;
+      if (h + 1 < p.nkv) {
+        // the other q' buffer was last read by the logit product of head h - 1
+        if (h >= 1) {
+          if (ok) ok = mbar_wait(&z_full[zb ^ 1], (uint32_t)((h - 1) >> 1) & 1u, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+        }
+        store_q(h + 1);
+        fetch_q(h + 2);
+        fence_proxy_async_smem();
+        ok = rotate(h + 1, ok);  // runs one head ahead of the softmax
+      }
+      // ---- logits of this head: one warp per lane quadrant (e = 4..7) moves them from tensor memory to shared memory
+      if (qt == 1) {
+        if (ok) ok = mbar_wait(&z_full[zb], (uint32_t)(h >> 1) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+        if (ok) {
+          uint32_t v[16];
+          tmem_ld16(tmem_base + kZCol + (uint32_t)zb * 16 + lane_addr, v);
+          tmem_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&z_empty[zb]);
 #pragma unroll
-      for (int gp = 0; gp < 4; ++gp) lg[gp] = make_float2(0.f, 0.f);
-      if (ok) {
-        uint32_t ka[16], kb[16];
-        const uint32_t base = tmem_base + (uint32_t)buf * 128 + lane_addr + (uint32_t)qt * 16;
-        tmem_ld16(base, ka);
-        tmem_ld16(base + 64, kb);
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&k_empty[buf]);
-#pragma unroll
-        for (int ii = 0; ii < 16; ++ii) {
-          const int i = qt * 16 + ii;
-          float2 k12 = make_float2(__uint_as_float(ka[ii]), __uint_as_float(kb[ii]));
-          if (rope) {
-            const float sn = (float)(short)(sc[ii] & 0xffffu) * (1.f / 32767.f);
-            const float cs = (float)((int)sc[ii] >> 16) * (1.f / 32767.f);
-            k12 = __ffma2_rn(make_float2(-k12.y, k12.x), bcast2(sn), __fmul2_rn(k12, bcast2(cs)));
-          }
-          const float2 k1 = bcast2(k12.x), k2 = bcast2(k12.y);
-          const float4 qa = *reinterpret_cast<const float4 *>(qs + i * kMaxGroup);
-          const float4 qb = *reinterpret_cast<const float4 *>(qs + (i + 64) * kMaxGroup);
-          lg[0] = __ffma2_rn(make_float2(qa.x, qa.y), k1, __ffma2_rn(make_float2(qb.x, qb.y), k2, lg[0]));
-          lg[1] = __ffma2_rn(make_float2(qa.z, qa.w), k1, __ffma2_rn(make_float2(qb.z, qb.w), k2, lg[1]));
-          if (npair > 2) {
-            const float4 qc4 = *reinterpret_cast<const float4 *>(qs + i * kMaxGroup + 4);
-            const float4 qd4 = *reinterpret_cast<const float4 *>(qs + (i + 64) * kMaxGroup + 4);
-            lg[2] = __ffma2_rn(make_float2(qc4.x, qc4.y), k1, __ffma2_rn(make_float2(qd4.x, qd4.y), k2, lg[2]));
-            lg[3] = __ffma2_rn(make_float2(qc4.z, qc4.w), k1, __ffma2_rn(make_float2(qd4.z, qd4.w), k2, lg[3]));
-          }
+          for (int g = 0; g < kMaxGroup; ++g)
+            if (g < G) xch[(zb * G + g) * 128 + lane_row] = __uint_as_float(v[g]) + __uint_as_float(v[8 + g]);
         }
       }
-#pragma unroll
-      for (int gp = 0; gp < 4; ++gp) {
-        if (2 * gp < G) xch[(qt * G + 2 * gp) * 128 + lane_row] = lg[gp].x;
-        if (2 * gp + 1 < G) xch[(qt * G + 2 * gp + 1) * 128 + lane_row] = lg[gp].y;
-      }
-      epi_sync();  // logits exchanged; q' of this head is no longer read
+      if (qt == 1 || e < G) asm volatile("bar.sync 3, %0;" ::"r"(nsync) : "memory");
       // ---- tile softmax by warp e for head g = e; probabilities go into the MMA operand as hi + lo bf16
       if (e < G) {
         float l4[4], m = -INFINITY;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int t = u * 32 + lane;
-          l4[u] = (t < nt) ? (xch[e * 128 + t] + xch[(G + e) * 128 + t]) + (xch[(2 * G + e) * 128 + t] + xch[(3 * G + e) * 128 + t])
-                           : -INFINITY;
+          l4[u] = (t < nt) ? xch[(zb * G + e) * 128 + t] : -INFINITY;
           m = fmaxf(m, l4[u]);
         }
         m = warp_max(m);
         float ssum = 0.f;
-        // the previous head's P C^V must have read the operand before it is overwritten
-        if (ok && h > 0) ok = mbar_wait(u_full, (uint32_t)(h - 1) & 1u, abort_flag);
+        // the operand copy of this head was last read by the P C^V product of head h - 2
+        if (ok && h > 1) ok = mbar_wait(&u_full[h & 1], ((uint32_t)(h >> 1) & 1u) ^ 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -347,21 +490,19 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
           ssum += pe;
           const __nv_bfloat16 hi = __float2bfloat16_rn(pe);
           const __nv_bfloat16 lo = __float2bfloat16_rn(pe - __bfloat162float(hi));
-          uint8_t *blk = pop + (size_t)(t >> 6) * kBlkBytes;
+          uint8_t *blk = pop + (size_t)((h & 1) * 2 + (t >> 6)) * kPopBlk;
           *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(e, t & 63)) = hi;
           *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(G + e, t & 63)) = lo;
         }
         ssum = warp_sum(ssum);
         if (lane == 0) p.part_ms[((size_t)b * p.Hq + (size_t)kv * G + e) * p.n_tiles + tile] = make_float2(m, ssum);
         fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_ready);
       }
-      store_q();       // q' of the next head
-      fetch_q(h + 2);  // raw values two heads ahead
-      if (quad == 0 && h > 0) ok = read_u(h - 1, ok);  // the previous head's U, whose MMA ran during this head's K loop
-      epi_sync();
-      if (et == 0) mbar_arrive(p_ready);
+      if (u_reader && h > 0) ok = read_u(h - 1, ok);  // the previous head's U
     }
-    if (quad == 0) ok = read_u(p.nkv - 1, ok);
+    if (u_reader) ok = read_u(p.nkv - 1, ok);
   }
   tc_fence_before();
   __syncthreads();
@@ -386,7 +527,7 @@ struct MergeAbsorbParams {
   int out_dtype, Hq, G, D, rv, s, n_tiles, sel_stride;
   int64_t max_len;
   float theta;
-  double inv_freq[64];
+  uint64_t rope_turns[64];
 };
 
 __device__ __forceinline__ void cp_async16(void *dst, const void *src) {
@@ -457,7 +598,7 @@ __global__ void __launch_bounds__(128) k_merge_absorb(const __grid_constant__ Me
   // ---- rotated, scaled query channel and the sink logits
   const bool rope = p.theta > 0.f;
   const int partner = i < 64 ? i + 64 : i - 64;
-  const double inv_freq = p.inv_freq[i & 63];
+  const uint64_t inv_freq = p.rope_turns[i & 63];
   float qi = __bfloat162float(q_s[i]);
   if (rope) {
     const float o = __bfloat162float(q_s[partner]);
@@ -568,9 +709,9 @@ cudaError_t launch_attend_absorb(const StepArgs &a) {
   p.max_len = a.plan.max_len;
   p.theta = a.theta;
   p.dev_status = a.dev_status;
-  fill_inv_freq(p.inv_freq, kDh, a.theta);
-  const size_t smem = 1024 + (size_t)(ly.rk / 64 + ly.rv / 64 + kRing + 2) * kBlkBytes +
-                      sizeof(float) * (kDh * kMaxGroup + 4 * ly.G * 128) + 1024;
+  fill_rope_turns(p.rope_turns, kDh, a.theta);
+  const size_t smem = 1024 + (size_t)(ly.rk / 64 + ly.rv / 64 + kRing) * kBlkBytes + 4 * kPopBlk + 2 * kQopBytes +
+                      sizeof(float) * (2 * ly.G * 128) + 1024;
   static size_t smem_set = 0;
   if (smem > smem_set) {
     cudaError_t e = cudaFuncSetAttribute(k_attend_absorb, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -597,7 +738,7 @@ cudaError_t launch_merge_absorb(const StepArgs &a) {
   p.part_ms = (const float2 *)(a.ws + a.plan.off_att_ms);
   p.out = a.out; p.out_dtype = a.out_dtype; p.Hq = ly.Hq; p.G = ly.G; p.D = ly.D; p.rv = ly.rv; p.s = ly.s;
   p.n_tiles = a.plan.n_att_tiles; p.sel_stride = a.window + a.top_k; p.max_len = a.plan.max_len; p.theta = a.theta;
-  fill_inv_freq(p.inv_freq, kDh, a.theta);
+  fill_rope_turns(p.rope_turns, kDh, a.theta);
   const size_t smem = sizeof(__nv_bfloat16) * ((size_t)kDh * (ly.rv + 8) + kDh + 2 * (size_t)ly.s * kDh) +
                       sizeof(float) * ((size_t)kMgTiles * 2 * ly.rv + ly.rv + 4 * 64 + 64) + sizeof(float2) * kMgTiles + 16;
   static size_t smem_set = 0;

@@ -20,7 +20,7 @@ namespace s4r {
 
 using namespace sm100;
 
-void fill_inv_freq(double *dst, int head_dim, float theta);
+void fill_rope_turns(uint64_t *dst, int head_dim, float theta);
 
 namespace {
 
@@ -41,7 +41,7 @@ struct AttFastParams {
   int64_t cap, max_len;
   float theta;
   int32_t *dev_status;
-  double inv_freq[64];
+  uint64_t rope_turns[64];
 };
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
       for (int i = wt; i < 64 * kTok; i += kWorkers) {
         const int pair = i >> 7, t = i & (kTok - 1);
         float sn = 0.f, cs = 1.f;
-        if (rows[t] >= 0) rope_sincos(p.s + rows[t], p.inv_freq[pair], sn, cs);
+        if (rows[t] >= 0) rope_sincos(p.s + rows[t], p.rope_turns[pair], sn, cs);
         sc[i] = make_float2(sn, cs);
       }
     }
@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_sm100(const __grid_const
     // RoPE of the query: this thread prepares column qc of q' for the heads g = qg0, qg0 + 4
     const int qc = et & 127, qg0 = et >> 7;
     float q_sn = 0.f, q_cs = 1.f;
-    if (rope) rope_sincos(p.s + L - 1, p.inv_freq[qc & 63], q_sn, q_cs);
+    if (rope) rope_sincos(p.s + L - 1, p.rope_turns[qc & 63], q_sn, q_cs);
     const float q_scale = rsqrtf((float)kDh);
     // `ok` stays warp-uniform; after a failed wait the loop keeps its shape (every epi_sync is still reached)
     // but touches tensor memory no more
@@ -415,7 +415,7 @@ cudaError_t launch_attend_sm100(const StepArgs &a) {
   p.max_len = a.plan.max_len;
   p.theta = a.theta;
   p.dev_status = a.dev_status;
-  fill_inv_freq(p.inv_freq, kDh, a.theta);
+  fill_rope_turns(p.rope_turns, kDh, a.theta);
   const size_t smem = 1024 + (size_t)(ly.rk / 64 + ly.rv / 64 + kRing) * kBlkBytes + sizeof(float2) * 64 * kTok +
                       sizeof(float) * (kDh * kMaxGroup + kTok * kMaxGroup + 4 * ly.G * 128) + 1024;
   static size_t smem_set = 0;

@@ -129,6 +129,15 @@ __device__ inline void rope_sincos(int pos, double inv_freq, float &sn, float &c
   __sincosf((float)red, &sn, &cs);  // |red| <= pi: the fast approximations are accurate to ~2^-21 there
 }
 
+// Same angle without fp64 arithmetic (slow on this part): `turns` = inv_freq / (2 pi) as a 0.64 fixed-point
+// fraction of a turn (host-computed).  The 64-bit product wraps modulo one turn exactly; its top 32 bits, read as
+// a signed number, are the reduced angle in [-1/2, 1/2) turns with 2^-32 resolution.
+__device__ inline void rope_sincos(int pos, uint64_t turns, float &sn, float &cs) {
+  const uint64_t ph = (uint64_t)(uint32_t)pos * turns;
+  const float red = (float)(int32_t)(uint32_t)(ph >> 32) * 1.4629180792671596e-9f;  // 2 pi / 2^32
+  __sincosf(red, &sn, &cs);
+}
+
 // ---- host-side plan of one decode step -------------------------------------------------------------
 
 struct DecodePlan {

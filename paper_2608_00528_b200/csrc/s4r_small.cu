@@ -240,7 +240,7 @@ struct MergeParams {
   int out_dtype, B, Hq, G, dh, D, s, n_tiles, att_tok, sel_stride;
   int64_t max_len;
   float theta;
-  double inv_freq[64];
+  uint64_t rope_turns[64];
 };
 
 __device__ __forceinline__ void cp_async16(void *dst, const void *src) {
@@ -313,7 +313,7 @@ __global__ void __launch_bounds__(128) k_merge(MergeParams p) {
   // ---- rotated, scaled query channel and the sink logits
   const bool rope = p.theta > 0.f;
   const int partner = i < half ? i + half : i - half;
-  const double inv_freq = p.inv_freq[i % half];
+  const uint64_t inv_freq = p.rope_turns[i % half];
   float qi = to_float(q_s[i]);
   if (rope) {
     const float o = to_float(q_s[partner]);
@@ -375,10 +375,13 @@ __global__ void __launch_bounds__(128) k_merge(MergeParams p) {
 
 }  // namespace
 
-void fill_inv_freq(double *dst, int head_dim, float theta) {
-  for (int i = 0; i < 64; ++i) dst[i] = 0.0;
+void fill_rope_turns(uint64_t *dst, int head_dim, float theta) {
+  for (int i = 0; i < 64; ++i) dst[i] = 0;
   if (theta > 0.f)
-    for (int i = 0; i < head_dim / 2 && i < 64; ++i) dst[i] = pow((double)theta, -2.0 * (double)i / (double)head_dim);
+    for (int i = 0; i < head_dim / 2 && i < 64; ++i) {
+      const double f = pow((double)theta, -2.0 * (double)i / (double)head_dim) / 6.283185307179586476925;  // < 0.16
+      dst[i] = (uint64_t)ldexp(f, 64);
+    }
 }
 
 // Query projection; when a.k_t is set, the new token's key and value rows are projected and appended too.
@@ -438,7 +441,7 @@ cudaError_t launch_merge(const StepArgs &a) {
   p.out = a.out; p.out_dtype = a.out_dtype; p.B = ly.B; p.Hq = ly.Hq; p.G = ly.G; p.dh = ly.dh; p.D = ly.D;
   p.s = ly.s; p.n_tiles = a.plan.n_att_tiles; p.att_tok = a.plan.att_tok; p.sel_stride = a.window + a.top_k;
   p.max_len = a.plan.max_len; p.theta = a.theta;
-  fill_inv_freq(p.inv_freq, ly.dh, a.theta);
+  fill_rope_turns(p.rope_turns, ly.dh, a.theta);
   const size_t esz = ly.dtype == S4R_BF16 ? 2 : 4;
   const size_t smem = esz * (size_t)ly.dh * (1 + 2 * (size_t)ly.s) + sizeof(float) * kMergeTiles * ly.dh +
                       sizeof(float2) * kMergeTiles + sizeof(float) * (4 * 64 + 64) + 16;
