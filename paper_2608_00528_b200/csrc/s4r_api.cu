@@ -52,6 +52,8 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   p->off_att = off;     off = align_up(off + sizeof(float) * ly.B * ly.Hq * (size_t)p->n_att_tiles *
                                              (att_fast_supported(ly) && 2 * ly.rv > ly.dh ? 2 * ly.rv : ly.dh), 256);
   p->off_att_ms = off;  off = align_up(off + sizeof(float2) * ly.B * ly.Hq * (size_t)p->n_att_tiles, 256);
+  p->off_proj = off;    off = align_up(off + sizeof(float) * ly.B * kProjMaxParts * (size_t)(((ly.G + 1) * ly.rk + ly.rv + 3) & ~3), 256);
+  p->off_flag = off;    off = align_up(off + sizeof(unsigned long long) * ly.B * (kMaxParts + 1), 256);
   p->off_basis_t = off;
   p->total = off > 256 ? off : 256;
   if (ly.dtype == S4R_BF16 && compress_fast_workspace(ly) > p->total) p->total = compress_fast_workspace(ly);
@@ -206,8 +208,9 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
     const int parts = scan_fast_parts(ly);
     if (parts < 1 || parts > a.plan.parts_cap) fast_scan = false; else a.plan.n_parts = parts;
   }
+  a.fuse_projection = fast_scan && scan_fuse_supported(ly);
   stage_mark(0, a.stream);
-  if (cuda_failed(launch_qproj(a))) return S4R_ERR_CUDA;
+  if (!a.fuse_projection && cuda_failed(launch_qproj(a))) return S4R_ERR_CUDA;
   stage_mark(1, a.stream);
   if (fast_scan) {
     if (cuda_failed(launch_scan_sm100(a))) return S4R_ERR_CUDA;

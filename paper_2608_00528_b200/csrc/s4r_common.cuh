@@ -17,6 +17,7 @@ constexpr int kSelThreads = 1024;  // threads per CTA of the selection kernel (o
 constexpr int kMaxCluster = 8;     // CTAs per sequence in the selection kernel (8 is the portable cluster size)
 constexpr int kProjCluster = 8;    // CTAs (slices of D') per sequence in the projection kernels
 constexpr int kMaxParts = 256;     // upper bound of softmax partials per sequence written by a scan kernel
+constexpr int kProjMaxParts = 16;  // CTAs per sequence that share the per-step projections inside the scan kernel
 
 // ---- programmatic dependent launch --------------------------------------------------------------------------
 // Every kernel of the decode step calls grid_dependency_sync() before its first global-memory access: it blocks
@@ -149,7 +150,7 @@ struct DecodePlan {
   int n_att_tiles;      // row tiles per sequence in the attention kernel
   int cluster;          // CTAs per sequence in the selection kernel
   int att_tok;          // selected rows per attention tile
-  size_t off_cq, off_z, off_part, off_score, off_hist, off_att, off_att_ms, off_basis_t, total;
+  size_t off_cq, off_z, off_part, off_score, off_hist, off_att, off_att_ms, off_proj, off_flag, off_basis_t, total;
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -18,6 +18,7 @@ struct StepArgs {
   const void *k_t = nullptr, *v_t = nullptr;
   void *coef_k_w = nullptr, *coef_v_w = nullptr;
   int32_t *coef_len_w = nullptr;
+  bool fuse_projection = false;  // Eq. 5-6 run inside the scan kernel; no projection kernel is launched
   int window, top_k, kappa, pool_mode, group_mode, value_path;
   float theta;
   void *out;
@@ -42,6 +43,10 @@ cudaError_t launch_select(const StepArgs &a);
 bool scan_fast_supported(const Layer &ly);
 int scan_fast_parts(const Layer &ly);  // CTAs (= softmax partials) per sequence; 0 on error
 cudaError_t launch_scan_sm100(const StepArgs &a);
+// projection fused into the scan kernel (cooperating CTAs of one sequence)
+struct ScanFuse { int npj, slot, groups_k, groups_v, rows_per; };
+bool scan_fuse_plan(const Layer &ly, int cps, ScanFuse *f);
+bool scan_fuse_supported(const Layer &ly);
 inline bool att_fast_supported(const Layer &ly) {
   return ly.dtype == S4R_BF16 && ly.dh == 128 && ly.rk % 64 == 0 && ly.rv % 64 == 0 && ly.rk >= 64 && ly.rv >= 64 &&
          (ly.rk + ly.rv) / 64 <= 6 && (int64_t)ly.B * ly.D < 0x7fffffffLL &&

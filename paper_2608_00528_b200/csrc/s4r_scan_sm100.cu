@@ -8,6 +8,18 @@
 // 32 columns); four epilogue warps read them back, scale by 1/sqrt(r), store Z[b][g][row] and keep the
 // running (max, sum exp) of Eq. 9 for the CTA's rows.  Warp 0 = TMA producer, warp 1 = MMA issuer,
 // warps 2-5 = epilogue.  grid (CTAs per sequence, B).
+//
+// Fused projection (Eq. 5-6).  The per-step projections c^Q = Q~ B^K, c^K_t = k_t B^K, c^V_t = v_t B^V are tiny
+// but cost a kernel of their own with two dependent trips to cold memory.  In the fused mode the first CTAs of
+// a sequence each multiply a slice of D' rows of the bases while the producer already streams coefficient
+// tiles, publish their partial sums in the workspace and raise a flag (a per-call token, so the workspace
+// needs no clearing); every CTA then adds the partials in CTA order (fixed order, deterministic) and builds
+// its B operand from the result.  CTA 0 of the sequence also stores the new token's coefficient rows, raises a
+// second flag and bumps coef_len; the producer that owns the tile with row L-1 waits for that flag before it
+// loads the tile.  CTAs of one launch wait on one another here: the grid never exceeds one CTA per SM, the host
+// checks that the device holds all of them at once, and every wait is bounded.
+#include <atomic>
+
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
 
@@ -15,13 +27,27 @@ namespace s4r {
 
 using namespace sm100;
 
+bool scan_fast_supported(const Layer &ly);
+int scan_fast_parts(const Layer &ly);
+
 namespace {
 
 constexpr int kTileRows = 128;
 constexpr int kScanThreads = 192;
 constexpr int kAccCols = 32;  // accumulator columns per buffer: [hi | mid | lo | 0] x 8 group members
 
+constexpr int kWorkers = kScanThreads - 32;  // warps 1-5: projection, B operand
+
 struct ScanFastParams {
+  // fused projection
+  int fused, npj, slot, groups_k, groups_v, rows_per, D, Hq, dh, dh_shift, rv;
+  const __nv_bfloat16 *q, *basis_k, *basis_v, *k_t, *v_t;
+  __nv_bfloat16 *coef_k_w, *coef_v_w;
+  int32_t *coef_len_w;
+  float *proj_part;               // [B][npj][slot]: (G + 1) x r_k key-side sums, then r_v value-side sums
+  unsigned long long *proj_flag;  // [B][cps + 1]: one per CTA of the sequence, then "token rows stored"
+  unsigned long long token;
+  unsigned *hist;                 // [B][2048], cleared here for the relevance kernel
   const float *cq_part;
   const int32_t *coef_len;
   float *Z;
@@ -31,6 +57,106 @@ struct ScanFastParams {
   float inv_sqrt_r;
   int32_t *dev_status;
 };
+
+__device__ __forceinline__ void st_release(unsigned long long *p, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_acquire(const unsigned long long *p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+// Bounded poll of a flag written by another CTA of this launch.
+__device__ __forceinline__ bool flag_wait(const unsigned long long *p, unsigned long long token, volatile int *abort_flag) {
+  if (ld_acquire(p) == token) return true;
+  const unsigned long long t0 = global_ns();
+  while (ld_acquire(p) != token) {
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      return false;
+    }
+    __nanosleep(100);
+  }
+  return true;
+}
+__device__ __forceinline__ void unpack_bf16x8(const uint4 &t, float (&v)[8]) {
+  const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+// Projection helpers.  Thread layout of a pass over a basis slice [nrows][r]: 16-byte chunk c = wt % (r/8) of a
+// row, row group rg = wt / (r/8); a thread owns rows rg, rg + groups, ...  All loads of a batch of kProjBatch rows
+// go out before anything is consumed: under the full-bandwidth coefficient stream a dependent trip to memory
+// costs about 2 us, so the number of trips is what matters.
+constexpr int kProjBatch = 12;
+
+__device__ __forceinline__ void proj_load(uint4 (&raw)[kProjBatch], const __nv_bfloat16 *basis, int r, int nrows,
+                                          int groups, int first, int wt) {
+  const int cpr = r >> 3;
+  const int c = wt % cpr, rg = wt / cpr;
+#pragma unroll
+  for (int u = 0; u < kProjBatch; ++u) {
+    const int i = first + rg + u * groups;
+    raw[u] = (rg < groups && i < nrows) ? __ldg(reinterpret_cast<const uint4 *>(basis + (size_t)i * r) + c)
+                                        : make_uint4(0, 0, 0, 0);
+  }
+}
+template <int NV>
+__device__ __forceinline__ void proj_fma(float (&acc)[NV][8], const uint4 (&raw)[kProjBatch], int r, int nrows,
+                                         int groups, int first, int nv, const float *xs, int rows_per, int wt) {
+  const int rg = wt / (r >> 3);
+#pragma unroll
+  for (int u = 0; u < kProjBatch; ++u) {
+    const int i = first + rg + u * groups;
+    if (rg < groups && i < nrows) {
+      float bv[8];
+      unpack_bf16x8(raw[u], bv);
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        if (v < nv) {
+          const float xv = xs[v * rows_per + i];
+          const float2 x2 = make_float2(xv, xv);
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            const float2 t = __ffma2_rn(x2, make_float2(bv[e], bv[e + 1]), make_float2(acc[v][e], acc[v][e + 1]));
+            acc[v][e] = t.x;
+            acc[v][e + 1] = t.y;
+          }
+        }
+      }
+    }
+  }
+}
+// sums over the row groups (fixed order) -> dst[nv * r]
+template <int NV>
+__device__ __forceinline__ void proj_reduce(const float (&acc)[NV][8], int r, int groups, int nv, float *red, float *dst,
+                                            int wt) {
+  const int cpr = r >> 3;
+  const int c = wt % cpr, rg = wt / cpr;
+  if (rg < groups) {
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+      if (v < nv) {
+        float4 *o = reinterpret_cast<float4 *>(red + ((size_t)rg * nv + v) * r + c * 8);
+        o[0] = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
+        o[1] = make_float4(acc[v][4], acc[v][5], acc[v][6], acc[v][7]);
+      }
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");
+  for (int i = wt; i < (nv * r) >> 2; i += kWorkers) {
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int g2 = 0; g2 < groups; ++g2) {
+      const float4 t = reinterpret_cast<const float4 *>(red + (size_t)g2 * nv * r)[i];
+      sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+    }
+    reinterpret_cast<float4 *>(dst)[i] = sum;
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");  // red is reused
+}
 
 __device__ __forceinline__ void online_update(float &m, float &s, float z) {
   if (z <= m) {
@@ -52,13 +178,22 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
   uint8_t *b_op = a_tiles + (size_t)p.stages * tile_bytes;         // [kblocks][32 rows][128 B]
   uint64_t *bars = reinterpret_cast<uint64_t *>(b_op + (size_t)kblocks * kAccCols * 128);
   uint64_t *full = bars, *empty = bars + p.stages, *acc_full = bars + 2 * p.stages, *acc_empty = acc_full + 2;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+  uint64_t *proj_bar = acc_empty + 2;  // projection done: the scratch stage may be loaded
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(proj_bar + 1);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  volatile int *go = reinterpret_cast<volatile int *>(tmem_slot + 2);
   float2 *red = reinterpret_cast<float2 *>(tmem_slot + 4);       // [4 warps][kMaxGroup]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.y, j = blockIdx.x;
-  int L = p.coef_len[b];
+  const int len = p.coef_len[b];
+  // fused cache update: the new token's row goes to index len and is scanned with the rest
+  bool tok_ok = p.fused && p.k_t != nullptr;
+  if (tok_ok && (len < 0 || (int64_t)len >= p.cap)) {
+    if (p.dev_status && tid == 0 && j == 0) atomicOr(p.dev_status, S4R_DEV_BOUNDS);
+    tok_ok = false;  // cache full: the token is dropped, the query is still scored
+  }
+  int L = len + (tok_ok ? 1 : 0);
   if (L < 0 || (int64_t)L > p.max_len) {
     if (p.dev_status && tid == 0) atomicOr(p.dev_status, S4R_DEV_BOUNDS);
     L = L < 0 ? 0 : (int)p.max_len;
@@ -67,7 +202,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
   const int tpc = (tiles_total + p.cps - 1) / p.cps;
   const int t_begin = min(tiles_total, j * tpc), t_end = min(tiles_total, t_begin + tpc);
   const int n_tiles = t_end - t_begin;
-  if (n_tiles <= 0) {  // uniform over the CTA: nothing to scan
+  if (n_tiles <= 0 && !p.fused) {  // uniform over the CTA: nothing to scan
     if (tid < p.G) p.part[((size_t)b * p.cps + j) * kMaxGroup + tid] = make_float2(-INFINITY, 0.f);
     return;
   }
@@ -81,6 +216,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
       mbar_init(&acc_full[a], 1);
       mbar_init(&acc_empty[a], 4);  // one arrival per epilogue warp
     }
+    mbar_init(proj_bar, 1);
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tmap);
@@ -92,40 +228,157 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp != 0) {
-    // While the producer (warp 0) already streams tiles, the other warps build the B operand: row n = t*8 + g
-    // holds term t (0 hi, 1 mid, 2 lo, 3 zero) of c^Q[g], K-major, 128-byte swizzle.  Loads go out in batches
-    // of 8 so that their latencies overlap.
-    constexpr int kWorkers = kScanThreads - 32;
+    // While the producer (warp 0) already streams tiles, the other warps produce c^Q and build the B operand:
+    // row n = t*8 + g holds term t (0 hi, 1 mid, 2 lo, 3 zero) of c^Q[g], K-major, 128-byte swizzle.
+    const int wt = tid - 32;
     const int n_el = kMaxGroup * p.r;
-    for (int i0 = tid - 32; i0 < n_el; i0 += 8 * kWorkers) {
-      float cval[8];
+    const float *cq_src = p.cq_part + (size_t)b * p.G * p.r;   // unfused: written by the projection kernel
+    int n_src = 1;                                              // partial sums to add per value
+    size_t src_stride = 0;
+    if (p.fused) {
+      // ---- Eq. 5-6: this CTA's slice of the basis rows; scratch = the last pipeline stage, which the producer
+      //      leaves alone until proj_bar
+      float *xs = reinterpret_cast<float *>(a_tiles + (size_t)(p.stages - 1) * tile_bytes);  // [G + 2][rows_per]
+      float *pred = xs + (size_t)(p.G + 2) * p.rows_per;  // row-group sums of one pass
+      const int d_lo = min(p.D, j * p.rows_per), d_hi = min(p.D, d_lo + p.rows_per);
+      const int nrows = j < p.npj ? d_hi - d_lo : 0;
+      const int nvk = p.G + (tok_ok ? 1 : 0);
+      if (j == 0)
+        for (int i = wt; i < 2048; i += kWorkers) p.hist[(size_t)b * 2048 + i] = 0;
+      if (j < p.npj) {
+        float *part = p.proj_part + ((size_t)b * p.npj + j) * p.slot;
+        const __nv_bfloat16 *bk = p.basis_k + ((size_t)b * p.D + d_lo) * p.r;
+        const __nv_bfloat16 *bv = p.basis_v + ((size_t)b * p.D + d_lo) * p.rv;
+        // one trip to memory: first batches of both bases, then the vectors
+        uint4 raw_k[kProjBatch], raw_v[kProjBatch];
+        proj_load(raw_k, bk, p.r, nrows, p.groups_k, 0, wt);
+        if (tok_ok) proj_load(raw_v, bv, p.rv, nrows, p.groups_v, 0, wt);
+        for (int di = wt; di < nrows; di += kWorkers) {
+          const int d = d_lo + di;
+          const __nv_bfloat16 *qd = p.q + ((size_t)b * p.Hq + (size_t)(d >> p.dh_shift) * p.G) * p.dh + (d & (p.dh - 1));
+          float x[kMaxGroup + 2];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int i = i0 + u * kWorkers;
-        const int g = i / p.r, k = i - g * p.r;
-        cval[u] = (i < n_el && g < p.G) ? __ldcg(p.cq_part + ((size_t)b * p.G + g) * p.r + k) : 0.f;
+          for (int v = 0; v < kMaxGroup; ++v) x[v] = v < p.G ? __bfloat162float(qd[(size_t)v * p.dh]) : 0.f;
+          x[kMaxGroup] = tok_ok ? __bfloat162float(p.k_t[(size_t)b * p.D + d]) : 0.f;
+          x[kMaxGroup + 1] = tok_ok ? __bfloat162float(p.v_t[(size_t)b * p.D + d]) : 0.f;
+#pragma unroll
+          for (int v = 0; v < kMaxGroup; ++v)
+            if (v < p.G) xs[v * p.rows_per + di] = x[v];
+          xs[p.G * p.rows_per + di] = x[kMaxGroup];
+          xs[(p.G + 1) * p.rows_per + di] = x[kMaxGroup + 1];
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");
+        {
+          float acc[kMaxGroup + 1][8];
+#pragma unroll
+          for (int v = 0; v < kMaxGroup + 1; ++v)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
+          proj_fma<kMaxGroup + 1>(acc, raw_k, p.r, nrows, p.groups_k, 0, nvk, xs, p.rows_per, wt);
+          for (int first = kProjBatch * p.groups_k; first < nrows; first += kProjBatch * p.groups_k) {
+            proj_load(raw_k, bk, p.r, nrows, p.groups_k, first, wt);
+            proj_fma<kMaxGroup + 1>(acc, raw_k, p.r, nrows, p.groups_k, first, nvk, xs, p.rows_per, wt);
+          }
+          proj_reduce<kMaxGroup + 1>(acc, p.r, p.groups_k, nvk, pred, part, wt);
+        }
+        if (tok_ok) {
+          float acc[1][8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[0][e] = 0.f;
+          const float *xv = xs + (size_t)(p.G + 1) * p.rows_per;
+          proj_fma<1>(acc, raw_v, p.rv, nrows, p.groups_v, 0, 1, xv, p.rows_per, wt);
+          for (int first = kProjBatch * p.groups_v; first < nrows; first += kProjBatch * p.groups_v) {
+            proj_load(raw_v, bv, p.rv, nrows, p.groups_v, first, wt);
+            proj_fma<1>(acc, raw_v, p.rv, nrows, p.groups_v, first, 1, xv, p.rows_per, wt);
+          }
+          proj_reduce<1>(acc, p.rv, p.groups_v, 1, pred, part + (size_t)(p.G + 1) * p.r, wt);
+        }
+        // the barrier at the end of proj_reduce orders every worker's stores before thread 0's release below
       }
+      // flag j: this CTA has read coef_len and (if it contributes) published its partial sums
+      unsigned long long *flags = p.proj_flag + (size_t)b * (p.cps + 1);
+      if (wt == 0) st_release(flags + j, p.token);
+      for (int i = wt; i < p.npj; i += kWorkers) flag_wait(flags + i, p.token, abort_flag);
+      asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");
+      if (wt == 0) *go = *abort_flag ? 0 : 1;
+      asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");
+      cq_src = p.proj_part + (size_t)b * p.npj * p.slot;
+      n_src = p.npj;
+      src_stride = (size_t)p.slot;
+      if (j == 0 && tok_ok && *go) {
+        // the new token's coefficient rows (Eq. 6), rounded once to the storage type
+        for (int i = wt; i < p.r + p.rv; i += kWorkers) {
+          const int off = i < p.r ? p.G * p.r + i : (p.G + 1) * p.r + (i - p.r);
+          float sum = 0.f;
+          for (int jj0 = 0; jj0 < n_src; jj0 += 16) {
+            float t[16];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int i = i0 + u * kWorkers;
-        if (i < n_el) {
-          const int g = i / p.r, k = i - g * p.r;
-          const float c = cval[u];
-          const __nv_bfloat16 hi = __float2bfloat16_rn(c);
-          const float r1 = c - __bfloat162float(hi);
-          const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-          const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-          uint8_t *blk = b_op + (size_t)(k >> 6) * (kAccCols * 128);
-          const int kc = k & 63;
-          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(g, kc)) = hi;
-          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(8 + g, kc)) = mid;
-          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(16 + g, kc)) = lo;
-          *reinterpret_cast<__nv_bfloat16 *>(blk + sw128_offset(24 + g, kc)) = __float2bfloat16_rn(0.f);
+            for (int q = 0; q < 16; ++q) t[q] = jj0 + q < n_src ? __ldcg(cq_src + (size_t)(jj0 + q) * src_stride + off) : 0.f;
+#pragma unroll
+            for (int q = 0; q < 16; ++q) sum += t[q];
+          }
+          if (i < p.r)
+            p.coef_k_w[((size_t)b * p.cap + len) * p.r + i] = __float2bfloat16_rn(sum);
+          else
+            p.coef_v_w[((size_t)b * p.cap + len) * p.rv + (i - p.r)] = __float2bfloat16_rn(sum);
+        }
+        // coef_len moves only after every CTA of the sequence has read the old value
+        for (int i = p.npj + wt; i < p.cps; i += kWorkers) flag_wait(flags + i, p.token, abort_flag);
+        asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");
+        if (wt == 0) {
+          st_release(flags + p.cps, p.token);
+          p.coef_len_w[b] = len + 1;
         }
       }
     }
+    // c^Q[g][k] = sum over the partials in CTA order, four consecutive k per thread (16-byte loads: the phase is
+    // bound by the instructions the five worker warps have to issue, not by bytes); up to sixteen partials are in
+    // flight at once.  Rows g >= G of the operand are zero.
+    const int n_q4 = n_el >> 2, r4 = p.r >> 2;
+    for (int i4 = wt; i4 < n_q4; i4 += kWorkers) {
+      const int g = i4 / r4, k = (i4 - g * r4) * 4;
+      float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (g < p.G) {
+        const float *src = cq_src + (size_t)g * p.r + k;
+        for (int jj0 = 0; jj0 < n_src; jj0 += 16) {
+          float4 t[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q)
+            t[q] = jj0 + q < n_src ? __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(jj0 + q) * src_stride))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            c4.x += t[q].x; c4.y += t[q].y; c4.z += t[q].z; c4.w += t[q].w;
+          }
+        }
+      }
+      const float cv[4] = {c4.x, c4.y, c4.z, c4.w};
+      uint32_t w[3][2];  // packed bf16 pairs of the hi / mid / lo terms
+#pragma unroll
+      for (int e2 = 0; e2 < 2; ++e2) {
+        __nv_bfloat16 term[3][2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float c = cv[2 * e2 + e];
+          term[0][e] = __float2bfloat16_rn(c);
+          const float r1 = c - __bfloat162float(term[0][e]);
+          term[1][e] = __float2bfloat16_rn(r1);
+          term[2][e] = __float2bfloat16_rn(r1 - __bfloat162float(term[1][e]));
+        }
+#pragma unroll
+        for (int t3 = 0; t3 < 3; ++t3)
+          w[t3][e2] = (uint32_t)__bfloat16_as_ushort(term[t3][0]) | ((uint32_t)__bfloat16_as_ushort(term[t3][1]) << 16);
+      }
+      uint8_t *blk = b_op + (size_t)(k >> 6) * (kAccCols * 128);
+      const int kc = k & 63;  // a multiple of 4: the four values share one 16-byte chunk of the swizzled row
+#pragma unroll
+      for (int t3 = 0; t3 < 3; ++t3)
+        *reinterpret_cast<uint2 *>(blk + sw128_offset(t3 * 8 + g, kc)) = make_uint2(w[t3][0], w[t3][1]);
+      *reinterpret_cast<uint2 *>(blk + sw128_offset(24 + g, kc)) = make_uint2(0u, 0u);
+    }
     fence_proxy_async_smem();
-    asm volatile("bar.sync 1, %0;" ::"n"(kScanThreads - 32) : "memory");  // B operand complete (producer not involved)
+    asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");  // B operand complete (producer not involved)
+    if (wt == 0) mbar_arrive(proj_bar);
   }
 
   if (warp == 0) {
@@ -133,9 +386,15 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
     if (lane == 0) {
       const uint64_t pol = policy_evict_first();
       int issued = 0;
+      const int tok_tile = tok_ok ? len / kTileRows : -1;  // tile that holds the row stored by CTA 0 of the sequence
       for (int it = 0; it < n_tiles; ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+        if (p.fused && it == p.stages - 1 && !mbar_wait(proj_bar, 0, abort_flag)) break;  // scratch stage released
+        if (t_begin + it == tok_tile) {
+          if (!flag_wait(p.proj_flag + (size_t)b * (p.cps + 1) + p.cps, p.token, abort_flag)) break;
+          asm volatile("fence.proxy.async;" ::: "memory");  // the row was written through the generic proxy
+        }
         if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag)) break;
         mbar_expect_tx(&full[s], tile_bytes);
         const int y = (int)((int64_t)b * p.cap) + (t_begin + it) * kTileRows;
@@ -266,6 +525,30 @@ bool make_tmap_bf16_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Geometry of the fused projection for `cps` CTAs per sequence; false when the scratch stage cannot hold it.
+bool scan_fuse_plan(const Layer &ly, int cps, ScanFuse *f) {
+  if (!scan_fast_supported(ly) || ly.rv % 8 || cps < 1) return false;
+  f->npj = cps < kProjMaxParts ? cps : kProjMaxParts;
+  f->rows_per = (ly.D + f->npj - 1) / f->npj;
+  f->slot = ((ly.G + 1) * ly.rk + ly.rv + 3) & ~3;
+  const long long scratch = (long long)(ly.rk / 64) * kTileRows * 128 / 4 - (long long)(ly.G + 2) * f->rows_per;  // floats
+  const int cpr_k = ly.rk / 8, cpr_v = ly.rv / 8;
+  if (scratch <= 0 || cpr_k > kWorkers || cpr_v > kWorkers) return false;
+  long long gk = kWorkers / cpr_k, gv = kWorkers / cpr_v;
+  if (gk > scratch / ((long long)(ly.G + 1) * ly.rk)) gk = scratch / ((long long)(ly.G + 1) * ly.rk);
+  if (gv > scratch / ly.rv) gv = scratch / ly.rv;
+  if (gk < 1 || gv < 1) return false;
+  f->groups_k = (int)gk;
+  f->groups_v = (int)gv;
+  return true;
+}
+
+bool scan_fuse_supported(const Layer &ly) {
+  ScanFuse f;
+  const int cps = scan_fast_parts(ly);
+  return cps >= 1 && scan_fuse_plan(ly, cps, &f);
+}
+
 bool scan_fast_supported(const Layer &ly) {
   return ly.dtype == S4R_BF16 && ly.rk % 64 == 0 && ly.rk >= 64 && ly.rk <= 512 && ly.cap > 0 &&
          (int64_t)ly.B * ly.cap < 0x7fffffffLL - 256;
@@ -304,6 +587,25 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
   p.inv_sqrt_r = (float)(1.0 / sqrt((double)ly.rk));
   p.dev_status = a.dev_status;
   const size_t tile_bytes = (size_t)(ly.rk / 64) * kTileRows * 128;
+  ScanFuse fz;
+  p.fused = a.fuse_projection && scan_fuse_plan(ly, p.cps, &fz) ? 1 : 0;
+  if (a.fuse_projection && !p.fused) return cudaErrorInvalidValue;  // the caller skipped the projection kernel
+  p.npj = fz.npj; p.slot = fz.slot; p.groups_k = fz.groups_k; p.groups_v = fz.groups_v; p.rows_per = fz.rows_per;
+  p.D = ly.D; p.Hq = ly.Hq; p.dh = ly.dh; p.rv = ly.rv;
+  p.dh_shift = ly.dh == 128 ? 7 : 6;  // head_dim is 64 or 128
+  p.q = (const __nv_bfloat16 *)a.q;
+  p.basis_k = (const __nv_bfloat16 *)a.basis_k;
+  p.basis_v = (const __nv_bfloat16 *)a.basis_v;
+  p.k_t = (const __nv_bfloat16 *)a.k_t;
+  p.v_t = (const __nv_bfloat16 *)a.v_t;
+  p.coef_k_w = (__nv_bfloat16 *)a.coef_k_w;
+  p.coef_v_w = (__nv_bfloat16 *)a.coef_v_w;
+  p.coef_len_w = a.coef_len_w;
+  p.proj_part = (float *)(a.ws + a.plan.off_proj);
+  p.proj_flag = (unsigned long long *)(a.ws + a.plan.off_flag);
+  p.hist = (unsigned *)(a.ws + a.plan.off_hist);
+  static std::atomic<unsigned long long> token_source{0x9e3779b97f4a7c15ull};
+  p.token = token_source.fetch_add(1) + 1;
   const size_t fixed = (size_t)(ly.rk / 64) * kAccCols * 128 + 1024 /*alignment*/ + 1024 /*barriers, flags, red*/;
   int stages = (int)((226 * 1024 - fixed) / tile_bytes);
   if (stages > 8) stages = 8;
@@ -317,6 +619,23 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
     smem_set = smem;
   }
   dim3 grid(p.cps, ly.B);
+  if (p.fused) {
+    // The CTAs of a sequence wait on one another, so all of them must be resident together.  The grid is at most
+    // one CTA per SM by construction; the occupancy query confirms that the device really holds it.  (A
+    // cooperative launch would have the runtime make the same check, but it gives up the overlap with the
+    // preceding kernel, about 5 us per step.)  Should other work keep some CTAs off the device for a while, the
+    // waits are bounded: the kernel gives up after a second and reports S4R_DEV_TIMEOUT instead of hanging.
+    static int checked_smem = -1, blocks_per_sm = 0, sms = 0;
+    if (checked_smem != (int)smem) {
+      int dev = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, k_scan_sm100, kScanThreads, smem) != cudaSuccess)
+        return cudaErrorInvalidValue;
+      checked_smem = (int)smem;
+    }
+    if ((long long)blocks_per_sm * sms < (long long)p.cps * ly.B) return cudaErrorCooperativeLaunchTooLarge;
+  }
   cudaError_t le = launch_chained(k_scan_sm100, grid, dim3(kScanThreads), smem, a.stream, 1, tmap, p);
   if (le != cudaSuccess) return le;
   ++launch_counter();

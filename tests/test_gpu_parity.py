@@ -269,7 +269,7 @@ def test_multi_layer_multi_step_generation_with_append():
             check_step(p, out, sel, cnt, L=L)
 
 
-def test_fused_append_decode_equals_separate_calls():
+def test_fused_append_decode_agrees_with_separate_calls():
     s4r = _s4r()
     cfg = _cfg(1, context=5000 + 3, batch=2)
     res = []
@@ -293,6 +293,16 @@ def test_fused_append_decode_equals_separate_calls():
                                 cfg.window, cfg.top_k, out, sel, cnt, ws, rope_theta=cfg.rope_theta)
         torch.cuda.synchronize()
         res.append((out.clone(), sel.clone(), cnt.clone(), p.d_CK.clone(), p.d_CV.clone(), p.d_len.clone()))
-    for a, b in zip(*res):
-        assert torch.equal(a, b)
-    assert res[0][5].tolist() == [cfg.cache_len + 2] * cfg.batch
+    # The two routes add the D' products of the new rows in different (each fixed) orders, so a coefficient may
+    # differ by one rounding of the storage type; everything downstream agrees to the accuracy of that rounding.
+    (out_a, sel_a, cnt_a, ck_a, cv_a, len_a), (out_b, sel_b, cnt_b, ck_b, cv_b, len_b) = res
+    assert len_a.tolist() == len_b.tolist() == [cfg.cache_len + 2] * cfg.batch
+    assert torch.equal(cnt_a, cnt_b)
+    for x, y in ((ck_a, ck_b), (cv_a, cv_b)):
+        xf, yf = x.float(), y.float()
+        assert torch.all((xf - yf).abs() <= 2.0 ** -7 * torch.maximum(xf.abs(), yf.abs()) + 1e-30)
+        assert torch.equal(x[:, :cfg.cache_len], y[:, :cfg.cache_len])           # the prompt rows are untouched
+    same = sum(len(set(sel_a[b].tolist()) & set(sel_b[b].tolist())) for b in range(cfg.batch))
+    assert same >= cfg.batch * (cfg.window + cfg.top_k) - 2 * cfg.batch           # at most a tie-band swap per sequence
+    err = (out_a - out_b).abs().amax() / out_a.abs().amax()
+    assert err <= 1e-3
