@@ -227,6 +227,9 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--context", type=int, default=None, help="override the context length (profiling only)")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling only)")
+    ap.add_argument("--rho", type=float, default=None,
+                    help="budget as a ratio of the cache (Eq. 14: top_k = floor(rho L) - window) instead of the "
+                         "configuration's top_k; the paper's setting is 0.2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = W.get_config(args.config)
@@ -237,6 +240,9 @@ def main():
         over["batch"] = args.batch
     if over:
         cfg = W.scaled_config(cfg, **over)
+    if args.rho is not None:
+        cfg = W.scaled_config(cfg, top_k=max(int(args.rho * cfg.cache_len) - cfg.window, 0),
+                              name=f"{cfg.name}_rho{args.rho:g}")
     if args.impl == "reference":
         return run_reference(args, cfg)
 

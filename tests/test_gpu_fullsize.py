@@ -123,3 +123,23 @@ def test_full_size_config(ci, checked):
         _properties(p, out, sel, cnt, b, cfg.window, cfg.top_k)
     out2, sel2, cnt2, _ = run_gpu_step(p)
     assert torch.equal(sel, sel2) and torch.equal(out, out2)          # run-to-run bitwise determinism
+
+
+def test_full_size_ratio_budget_rho_0_2():
+    """The paper's own budget at 128K: rho = 0.2 keeps about 26 000 rows per sequence, so that the reconstruction
+    and attention kernels, not the scan, carry most of the step (App. B's cost split)."""
+    import paper_2608_00528_b200 as s4r
+    base = W.get_config(2)
+    k = s4r.top_k_from_ratio(0.2, base.cache_len, base.window)
+    cfg = W.scaled_config(base, top_k=k)
+    checked = (3,)
+    p = FullSizeProblem(cfg, checked)
+    p.check_compress_and_adopt_oracle_coefficients()
+    del p.d_K, p.d_V
+    torch.cuda.empty_cache()
+    out, sel, cnt, status = run_gpu_step(p)
+    assert status == 0
+    worst = check_step(p, out, sel, cnt, seqs=list(checked))
+    print(f"{cfg.name} rho=0.2 (k={k}): selection ok, max rel output error {worst:.3e}")
+    for b in range(cfg.batch):
+        _properties(p, out, sel, cnt, b, cfg.window, cfg.top_k)

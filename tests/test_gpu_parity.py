@@ -136,6 +136,22 @@ def test_small_rank_head_dim_64_and_asymmetric_ranks():
     check_step(p, out, sel, cnt)
 
 
+@pytest.mark.parametrize("rank_k,rank_v,value_path", [(128, 192, 0), (128, 192, 1), (128, 256, 0), (64, 128, 0)])
+def test_asymmetric_ranks_with_ratio_budget_on_the_tensor_core_paths(rank_k, rank_v, value_path):
+    """Sec. 3.3 / App. D: r^K < r^V and a budget given as a ratio, k = max(floor(rho L) - W, 0) (Eq. 14).  With
+    r_v = 256 the absorbed kernel's tensor-memory plan does not fit and the reconstructing kernel runs."""
+    s4r = _s4r()
+    cfg0 = _cfg(1, context=9000 + 4, rank_k=rank_k, rank_v=rank_v)
+    k = s4r.top_k_from_ratio(0.2, cfg0.cache_len, cfg0.window)
+    assert k == int(0.2 * cfg0.cache_len) - cfg0.window
+    cfg = _cfg(1, context=9000 + 4, rank_k=rank_k, rank_v=rank_v, top_k=k)
+    p = Problem(cfg, device="cuda").upload()
+    out, sel, cnt, status = run_gpu_step(p, value_path=value_path)
+    assert status == 0
+    err = check_step(p, out, sel, cnt)
+    print(f"r_k={rank_k} r_v={rank_v} rho=0.2 (k={k}) value_path={value_path}: max rel err {err:.3e}")
+
+
 def test_decode_step_host_entry_point():
     s4r = _s4r()
     cfg = _cfg(0, context=2000)
