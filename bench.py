@@ -131,7 +131,7 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(sm), "source": self.source}
 
 
-def build_cache(cfg, s4r, device, capacity, seq_ids):
+def build_cache(cfg, s4r, device, capacity, seq_ids, layer=0, ws=None):
     """Synthetic prompt -> bases (set-up) -> s4r_compress.  Returns the device-resident cache and timings."""
     st = W.storage_dtype(cfg)
     B, s, D = cfg.batch, cfg.sink_count, cfg.d_kv
@@ -143,17 +143,18 @@ def build_cache(cfg, s4r, device, capacity, seq_ids):
     BV = torch.empty(B, D, cfg.rank_v, dtype=st, device=device)
     q = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=st, device=device)
     for b, sid in enumerate(seq_ids):                        # every rank draws its own sequences
-        K[b] = W.make_kv(cfg, 0, sid, "k", device=device)
-        V[b] = W.make_kv(cfg, 0, sid, "v", device=device)
-        BK[b] = W.make_bench_basis(K[b][W.sample_rows(cfg, 0, sid, "k").to(device)], cfg.rank_k, st)
-        BV[b] = W.make_bench_basis(V[b][W.sample_rows(cfg, 0, sid, "v").to(device)], cfg.rank_v, st)
-        q[b] = W.make_query(cfg, K[b], 0, sid)
+        K[b] = W.make_kv(cfg, layer, sid, "k", device=device)
+        V[b] = W.make_kv(cfg, layer, sid, "v", device=device)
+        BK[b] = W.make_bench_basis(K[b][W.sample_rows(cfg, layer, sid, "k").to(device)], cfg.rank_k, st)
+        BV[b] = W.make_bench_basis(V[b][W.sample_rows(cfg, layer, sid, "v").to(device)], cfg.rank_v, st)
+        q[b] = W.make_query(cfg, K[b], layer, sid)
     sink_k = torch.empty(B, s, D, dtype=st, device=device)
     sink_v = torch.empty_like(sink_k)
     CK = torch.zeros(B, capacity, cfg.rank_k, dtype=st, device=device)
     CV = torch.zeros(B, capacity, cfg.rank_v, dtype=st, device=device)
     ln = torch.zeros(B, dtype=torch.int32, device=device)
-    ws = s4r.alloc_workspace(ly, capacity, cfg.window, cfg.top_k, device)
+    if ws is None:
+        ws = s4r.alloc_workspace(ly, capacity, cfg.window, cfg.top_k, device)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s4r.compress(ly, K, V, BK, BV, sink_k, sink_v, CK, CV, ln, workspace=ws)       # warm-up
     torch.cuda.synchronize()
@@ -167,6 +168,88 @@ def build_cache(cfg, s4r, device, capacity, seq_ids):
     torch.cuda.empty_cache()
     return dict(ly=ly, BK=BK, BV=BV, q=q, sink_k=sink_k, sink_v=sink_v, CK=CK, CV=CV, len=ln, ws=ws,
                 compress_ms=compress_ms, compress_launches=compress_launches)
+
+
+def run_all_layers(args, cfg, s4r, device):
+    """Config 4's flow: every layer's prompt is compressed once, then `decode_steps` decode steps run over all
+    layers (cache update + decode per layer and step).  One JSON line with compress and decode throughput."""
+    layers = args.layers or cfg.n_layers
+    steps, B = cfg.decode_steps, cfg.batch
+    capacity = cfg.cache_len + 2 * steps + 8
+    st = W.storage_dtype(cfg)
+    seq_ids = list(range(B))
+    caches, ws, compress_ms, pool = [], None, 0.0, 2
+    for layer in range(layers):
+        c = build_cache(cfg, s4r, device, capacity, seq_ids, layer=layer, ws=ws)
+        ws = c["ws"]
+        compress_ms += c["compress_ms"]
+        c["kt"] = torch.stack([torch.stack([W.make_token(cfg, layer, b, "k", i + 1, device) for b in seq_ids]) for i in range(pool)])
+        c["vt"] = torch.stack([torch.stack([W.make_token(cfg, layer, b, "v", i + 1, device) for b in seq_ids]) for i in range(pool)])
+        caches.append(c)
+    n_sel = cfg.window + cfg.top_k
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=device)
+    sel = torch.empty(B, n_sel, dtype=torch.int32, device=device)
+    cnt = torch.empty(B, dtype=torch.int32, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    kw = dict(pool_kernel=cfg.pool_kernel, pool_mode={"max": s4r.POOL_MAX, "avg": s4r.POOL_AVG}[cfg.pool_mode],
+              group_mode={"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode], rope_theta=cfg.rope_theta,
+              dev_status=status)
+
+    def model_step(i):
+        for c in caches:
+            s4r.append_decode_step(c["ly"], c["kt"][i % pool], c["vt"][i % pool], c["q"], c["sink_k"], c["sink_v"], c["CK"],
+                                   c["CV"], c["len"], c["BK"], c["BV"], capacity, cfg.window, cfg.top_k, out, sel, cnt, ws, **kw)
+
+    for i in range(3):
+        model_step(i)
+    for c in caches:
+        c["len"].fill_(cfg.cache_len)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        model_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    s4r.stage_timing(True)
+    stage_sum = {}
+    for c in caches[:4]:
+        c["len"].fill_(cfg.cache_len + steps)
+        s4r.append_decode_step(c["ly"], c["kt"][0], c["vt"][0], c["q"], c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"],
+                               c["BK"], c["BV"], capacity, cfg.window, cfg.top_k, out, sel, cnt, ws, **kw)
+        for k_, v_ in s4r.stage_times().items():
+            stage_sum[k_] = stage_sum.get(k_, 0.0) + v_ / min(4, len(caches))
+    s4r.stage_timing(False)
+    layer_steps = steps * layers
+    esz = cfg.elem_bytes
+    L_now = cfg.cache_len + steps
+    scan_bytes = B * L_now * cfg.rank_k * esz
+    peak, peak_kind = _peaks()
+    scan_ms = stage_sum.get("latent_scoring", float("nan"))
+    prompt_tokens = B * (cfg.context - cfg.sink_count) * layers
+    line = {
+        "metric": "decode layer-steps/sec (all layers, cache update + decode per layer and step)",
+        "value": layer_steps / (ms * 1e-3), "unit": "layer-steps/s", "n_gpus": 1, "steps": steps, "warmup": 3,
+        "ms_per_step": ms / layer_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": layers, "batch": B, "context": cfg.context, "decode_steps": steps,
+                   "rank": cfg.rank_k, "window": cfg.window, "top_k": cfg.top_k,
+                   "l2": "inputs larger than L2 (%.0f MB of key coefficients per layer-step, %.1f GB of caches)"
+                         % (scan_bytes / 1e6, 2 * layers * scan_bytes / 1e9)},
+        "model_steps_per_s": steps / (ms * 1e-3), "tokens_per_s": steps * B / (ms * 1e-3),
+        "compress": {"ms_all_layers": compress_ms, "token_layers_per_s": prompt_tokens / (compress_ms * 1e-3),
+                     "prompt_tokens_per_s": prompt_tokens / layers / (compress_ms * 1e-3)},
+        "roofline": {"bound": "hbm", "kernel": "latent_scoring", "achieved": scan_bytes / (scan_ms * 1e-3) / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": scan_bytes / (scan_ms * 1e-3) / 1e9 / peak, "peak_kind": peak_kind,
+                     "traffic": scan_bytes * SCAN_DRAM_BYTES_PER_ALGORITHMIC_BYTE, "ms_per_launch": scan_ms},
+        "stage_ms": stage_sum, "gpu_launches": None, "clocks": clocks, "dev_status": int(status.item()),
+        "cpu_baseline": None, "e2e": None,
+    }
+    print(json.dumps(line), flush=True)
 
 
 def cpu_baseline(cfg, repeats=3):
@@ -230,6 +313,7 @@ def main():
     ap.add_argument("--rho", type=float, default=None,
                     help="budget as a ratio of the cache (Eq. 14: top_k = floor(rho L) - window) instead of the "
                          "configuration's top_k; the paper's setting is 0.2")
+    ap.add_argument("--layers", type=int, default=None, help="layers to run for a multi-layer configuration (default: all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = W.get_config(args.config)
@@ -259,6 +343,8 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
+    if cfg.n_layers > 1 and world == 1:
+        return run_all_layers(args, cfg, s4r, device)
     K_steps, Wm = args.steps, max(args.warmup, 3)
     n_append = 2 * (K_steps + Wm) + 8
     capacity = cfg.cache_len + n_append

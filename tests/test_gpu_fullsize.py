@@ -17,14 +17,14 @@ pytestmark = pytest.mark.gpu
 
 
 class FullSizeProblem(Problem):
-    def __init__(self, cfg, checked):
+    def __init__(self, cfg, checked, layer=0, extra_rows=0):
         import paper_2608_00528_b200 as s4r
-        self.cfg, self.layer, self.st = cfg, 0, W.storage_dtype(cfg)
+        self.cfg, self.layer, self.st = cfg, layer, W.storage_dtype(cfg)
         self.device = torch.device("cuda")
         dev, st = self.device, self.st
         B, s, D, T = cfg.batch, cfg.sink_count, cfg.d_kv, cfg.context
         self.L = cfg.cache_len
-        self.cap = self.L
+        self.cap = self.L + extra_rows
         self.checked = list(checked)
         self.d_K = torch.empty(B, T, D, dtype=st, device=dev)
         self.d_V = torch.empty_like(self.d_K)
@@ -34,12 +34,12 @@ class FullSizeProblem(Problem):
         self.K, self.V = [None] * B, [None] * B            # sink rows only (the oracle needs nothing else of them)
         self.q, self.BK, self.BV, self.CK, self.CV = ([None] * B for _ in range(5))
         for b in range(B):
-            self.d_K[b] = W.make_kv(cfg, 0, b, "k", device=dev)
-            self.d_V[b] = W.make_kv(cfg, 0, b, "v", device=dev)
-            q = W.make_query(cfg, self.d_K[b], 0, b)
+            self.d_K[b] = W.make_kv(cfg, layer, b, "k", device=dev)
+            self.d_V[b] = W.make_kv(cfg, layer, b, "v", device=dev)
+            q = W.make_query(cfg, self.d_K[b], layer, b)
             self.d_q[b] = q
-            rows_k = self.d_K[b][W.sample_rows(cfg, 0, b, "k").to(dev)]
-            rows_v = self.d_V[b][W.sample_rows(cfg, 0, b, "v").to(dev)]
+            rows_k = self.d_K[b][W.sample_rows(cfg, layer, b, "k").to(dev)]
+            rows_v = self.d_V[b][W.sample_rows(cfg, layer, b, "v").to(dev)]
             if b in self.checked:
                 bk = O.round_to_storage(O.build_basis(to_np(rows_k), cfg.rank_k)[0], cfg.dtype)
                 bv = O.round_to_storage(O.build_basis(to_np(rows_v), cfg.rank_v)[0], cfg.dtype)
@@ -89,7 +89,7 @@ class FullSizeProblem(Problem):
                 assert (np.abs(got - want) <= 2 * O.storage_ulp(np.maximum(np.abs(want), np.abs(got)), "bf16")
                         + 1e-4 * np.abs(want).max()).all()
                 assert (got != want).mean() < 0.02
-                store[b] = want
+                store[b] = np.concatenate([want, np.zeros((self.cap - self.L, want.shape[1]))])
                 d_c[b, :self.L] = from_np(want, self.st, self.device)
                 del x, got
 
@@ -143,3 +143,63 @@ def test_full_size_ratio_budget_rho_0_2():
     print(f"{cfg.name} rho=0.2 (k={k}): selection ok, max rel output error {worst:.3e}")
     for b in range(cfg.batch):
         _properties(p, out, sel, cnt, b, cfg.window, cfg.top_k)
+
+
+def test_config4_layers_and_decode_steps_at_full_shape():
+    """Config 4 (32 layers, batch 16, 64K prompt, 64 decode steps with the cache update): layers are independent
+    problems, so three of them (first, middle, last) run at the full batch and context.  Every step appends the
+    new token's rows for all 16 sequences.  For the checked sequences the oracle keeps its own cache; the
+    library's new rows are compared with the oracle's and replaced by them, and at four steps the decode output
+    and index set are compared on those identical inputs (separate append + decode calls there, the fused call
+    everywhere else)."""
+    import paper_2608_00528_b200 as s4r
+    cfg = W.get_config(4)
+    checked, check_steps = (0, 15), (1, 2, 32, 64)
+    for layer in (0, cfg.n_layers // 2 - 1, cfg.n_layers - 1):
+        p = FullSizeProblem(cfg, checked, layer=layer, extra_rows=cfg.decode_steps)
+        p.check_compress_and_adopt_oracle_coefficients(n_rows_abs=2048)
+        del p.d_K, p.d_V
+        torch.cuda.empty_cache()
+        ly = p.layer_desc()
+        B = cfg.batch
+        ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+        out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, device="cuda")
+        sel = torch.empty(B, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+        cnt = torch.empty(B, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        kw = dict(rope_theta=cfg.rope_theta, dev_status=status)
+        worst = 0.0
+        for step in range(1, cfg.decode_steps + 1):
+            L = p.L + step
+            kt = torch.stack([W.make_token(cfg, layer, b, "k", step, "cuda") for b in range(B)])
+            vt = torch.stack([W.make_token(cfg, layer, b, "v", step, "cuda") for b in range(B)])
+            if step in check_steps:
+                s4r.append(ly, kt, vt, p.d_BK, p.d_BV, p.d_CK, p.d_CV, p.d_len, dev_status=status)
+            else:
+                s4r.append_decode_step(ly, kt, vt, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV,
+                                       p.cap, cfg.window, cfg.top_k, out, sel, cnt, ws, **kw)
+            torch.cuda.synchronize()
+            assert status.item() == 0 and p.d_len.tolist() == [L] * B
+            for b in checked:
+                for x_t, basis, d_c, store in ((kt, p.BK, p.d_CK, p.CK), (vt, p.BV, p.d_CV, p.CV)):
+                    want = O.project_token(to_np(x_t[b]), basis[b], "bf16")
+                    got = to_np(d_c[b, L - 1])
+                    absdot = np.abs(to_np(x_t[b])) @ np.abs(basis[b])
+                    assert (np.abs(got - want) <= O.storage_ulp(want, "bf16") * 1.0001 + 2.0 ** -18 * absdot).all()
+                    store[b][L - 1] = want
+                    d_c[b, L - 1] = from_np(want, p.st, p.device)
+            if step in check_steps:
+                s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                cfg.window, cfg.top_k, out, sel, cnt, ws, **kw)
+                torch.cuda.synchronize()
+                assert status.item() == 0
+                worst = max(worst, check_step(p, out, sel, cnt, seqs=list(checked), L=L))
+            if step in (check_steps[0], cfg.decode_steps):
+                p.L, keep = L, p.L
+                for b in range(B):
+                    _properties(p, out, sel, cnt, b, cfg.window, cfg.top_k)
+                p.L = keep
+        print(f"{cfg.name} layer {layer}: {cfg.decode_steps} steps, checked steps {check_steps}, "
+              f"max rel output error {worst:.3e}")
+        del p, ws
+        torch.cuda.empty_cache()
