@@ -17,7 +17,16 @@
  *     stage timing below) and never synchronises the stream (except
  *     s4r_decode_step_host and s4r_stage_times, see there).
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
- *     work of a call is enqueued on it, in order.
+ *     work of a call is enqueued on it, in order.  The device-pointer calls
+ *     may be captured into a CUDA graph (after one uncaptured call on the
+ *     device): while the stream is capturing, the decode step projects the
+ *     query in a kernel of its own instead of inside the scoring kernel, so
+ *     that nothing in the captured arguments is specific to one call.
+ *   - On sm_100 with bf16 storage the scoring kernel's CTAs of one sequence
+ *     exchange partial sums of the per-step projections and wait for one
+ *     another (bounded).  The launch is sized to one CTA per SM and the host
+ *     checks that the device can hold all of them; if other work keeps them
+ *     apart for more than a second the call ends with S4R_DEV_TIMEOUT.
  *   - Every entry point returns S4R_OK or a negative s4r_status_t.  Misuse
  *     that the host can see is rejected before anything is launched.
  *   - `dev_status` (may be NULL) is a device int32 the kernels OR flags into
@@ -156,7 +165,8 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
 
 /* s4r_append followed by s4r_decode_step as one call (Sec. 3.2.1 then 3.2.2-3.2.3): the new token's key and
  * value rows are projected in the same pass over the bases that projects the query (Eq. 5), appended
- * (Eq. 6), and the step then runs on the grown cache.  Results are bit-identical to the two separate calls.
+ * (Eq. 6), and the step then runs on the grown cache.  The new rows may differ from those of s4r_append by one
+ * rounding of the storage type (the D' products are added in a different, equally fixed order).
  * k_t, v_t [B, D'] pre-RoPE; coef_k, coef_v, coef_len are updated; max_len must bound coef_len[b] + 1. */
 int s4r_append_decode_step(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,
                            const void *sink_k, const void *sink_v, void *coef_k, void *coef_v, int32_t *coef_len,

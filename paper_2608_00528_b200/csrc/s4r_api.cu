@@ -209,6 +209,15 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
     if (parts < 1 || parts > a.plan.parts_cap) fast_scan = false; else a.plan.n_parts = parts;
   }
   a.fuse_projection = fast_scan && scan_fuse_supported(ly);
+  if (a.fuse_projection) {
+    // The fused projection identifies each call by a fresh token in its kernel arguments.  A captured graph
+    // would replay the same token, so under stream capture the projection runs as its own kernel instead.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(a.stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+      (void)cudaGetLastError();
+      a.fuse_projection = false;
+    }
+  }
   stage_mark(0, a.stream);
   if (!a.fuse_projection && cuda_failed(launch_qproj(a))) return S4R_ERR_CUDA;
   stage_mark(1, a.stream);

@@ -322,3 +322,43 @@ def test_fused_append_decode_agrees_with_separate_calls():
     assert same >= cfg.batch * (cfg.window + cfg.top_k) - 2 * cfg.batch           # at most a tie-band swap per sequence
     err = (out_a - out_b).abs().amax() / out_a.abs().amax()
     assert err <= 1e-3
+
+
+def test_decode_step_replayed_from_a_cuda_graph():
+    """A captured step must give the same result on every replay (the per-call token of the fused projection
+    cannot be used there, so the library falls back to the separate projection kernel while capturing)."""
+    s4r = _s4r()
+    cfg = _cfg(1, context=6000 + 4, batch=2)
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+    out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(cfg.batch, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(cfg.batch, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step():
+        s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap, cfg.window,
+                        cfg.top_k, out, sel, cnt, ws, rope_theta=cfg.rope_theta, dev_status=status)
+
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step()                       # warm-up outside capture (function attributes, driver entry points)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    ref = None
+    for q_scale in (1.0, 0.5, 1.0):
+        p.d_q.copy_(torch.stack([from_np(q * q_scale, p.st, p.device) for q in p.q]))
+        out.zero_(); sel.fill_(-7); cnt.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        if q_scale == 1.0:
+            check_step(p, out, sel, cnt)
+            if ref is None:
+                ref = (out.clone(), sel.clone())
+            else:
+                assert torch.equal(out, ref[0]) and torch.equal(sel, ref[1])
