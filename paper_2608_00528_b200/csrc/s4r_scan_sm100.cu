@@ -19,6 +19,8 @@
 // loads the tile.  CTAs of one launch wait on one another here: the grid never exceeds one CTA per SM, the host
 // checks that the device holds all of them at once, and every wait is bounded.
 #include <atomic>
+#include <chrono>
+#include <random>
 
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
@@ -604,7 +606,11 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
   p.proj_part = (float *)(a.ws + a.plan.off_proj);
   p.proj_flag = (unsigned long long *)(a.ws + a.plan.off_flag);
   p.hist = (unsigned *)(a.ws + a.plan.off_hist);
-  static std::atomic<unsigned long long> token_source{0x9e3779b97f4a7c15ull};
+  // per-call token: unique within the process (counter) and seeded per process, so that flags left in recycled
+  // device memory by an earlier call or an earlier process never match
+  static std::atomic<unsigned long long> token_source{
+      0x9e3779b97f4a7c15ull ^ ((unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() << 20) ^
+      ((unsigned long long)std::random_device{}() << 32)};
   p.token = token_source.fetch_add(1) + 1;
   const size_t fixed = (size_t)(ly.rk / 64) * kAccCols * 128 + 1024 /*alignment*/ + 1024 /*barriers, flags, red*/;
   int stages = (int)((226 * 1024 - fixed) / tile_bytes);
