@@ -412,7 +412,7 @@ def main():
     s4r.stage_timing(False)
     stage_ms = {k_: v_ / n_prof for k_, v_ in stage_sum.items()}
 
-    # ---- end to end through the host-buffer entry point: q from pinned host memory, results read back
+    # ---- end to end: q, k_t, v_t from pinned host memory every step, results read back every step
     c["len"].fill_(cfg.cache_len)
     q_h = [qs[j].cpu().pin_memory() for j in range(pool)]
     kt_h = [kt[j].cpu().pin_memory() for j in range(pool)]
@@ -423,12 +423,18 @@ def main():
     q_d, kt_d, vt_d = torch.empty_like(qs[0]), torch.empty_like(kt[0]), torch.empty_like(vt[0])
 
     def step_e2e(i):
+        # the call a user makes for one generated token: inputs from pinned host memory, one fused library call
+        # (cache update + decode step), results read back to the host before the next token
         j = i % pool
         kt_d.copy_(kt_h[j], non_blocking=True)
         vt_d.copy_(vt_h[j], non_blocking=True)
-        s4r.append(ly, kt_d, vt_d, c["BK"], c["BV"], c["CK"], c["CV"], c["len"], dev_status=status)
-        s4r.decode_step_host(ly, q_h[j], q_d, c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"],
-                             capacity, cfg.window, cfg.top_k, out_h, out, sel_h, sel, cnt_h, cnt, c["ws"], **kw)
+        q_d.copy_(q_h[j], non_blocking=True)
+        s4r.append_decode_step(ly, kt_d, vt_d, q_d, c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"],
+                               capacity, cfg.window, cfg.top_k, out, sel, cnt, c["ws"], **kw)
+        out_h.copy_(out, non_blocking=True)
+        sel_h.copy_(sel, non_blocking=True)
+        cnt_h.copy_(cnt, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
 
     for i in range(3):
         step_e2e(i)

@@ -120,14 +120,18 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
   }
   if (warp == 1) tmem_alloc(tmem_slot, 512);
   grid_dependency_sync();
-  const int count = min(p.sel_count[b], p.sel_stride);
+  // One trip to memory for everything the gather depends on: the index list, its length and the cache length
+  // are fetched side by side (entries past the list's end read as -1, the selection kernel pads with -1).
   const int t0 = tile * kTok;
-  const bool active = t0 < count;  // uniform over the CTA
-  const int nt = min(kTok, count - t0);
+  int rix_raw = -1;
+  if (tid < kTok && t0 + tid < p.sel_stride) rix_raw = p.sel_idx[(size_t)b * p.sel_stride + t0 + tid];
+  const int count = min(p.sel_count[b], p.sel_stride);
   int L = p.coef_len[b];
   L = L < 0 ? 0 : (L > p.max_len ? (int)p.max_len : L);
+  const bool active = t0 < count;  // uniform over the CTA
+  const int nt = min(kTok, count - t0);
   if (tid < kTok && active) {
-    int rix = (tid < nt) ? p.sel_idx[(size_t)b * p.sel_stride + t0 + tid] : -1;
+    const int rix = tid < nt ? rix_raw : -1;
     rows[tid] = rix < 0 ? -1 : min(rix, max(L - 1, 0));
   }
   tc_fence_before();
@@ -147,15 +151,15 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
     const int cpr_k = p.rk >> 3, cpr_v = p.rv >> 3;
     const __nv_bfloat16 *ckb = p.coef_k + (size_t)b * p.cap * p.rk;
     const __nv_bfloat16 *cvb = p.coef_v + (size_t)b * p.cap * p.rv;
-    for (int i = wt; i < kTok * cpr_k; i += kWorkers) {
-      const int t = i / cpr_k, c = i - t * cpr_k, rix = rows[t];
-      cp_async16_zfill(ck + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8),
-                       reinterpret_cast<const uint4 *>(ckb + (size_t)max(rix, 0) * p.rk) + c, rix >= 0);
-    }
-    for (int i = wt; i < kTok * cpr_v; i += kWorkers) {
-      const int t = i / cpr_v, c = i - t * cpr_v, rix = rows[t];
-      cp_async16_zfill(cv + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8),
-                       reinterpret_cast<const uint4 *>(cvb + (size_t)max(rix, 0) * p.rv) + c, rix >= 0);
+    // a warp per row, a lane per 16-byte piece (no index arithmetic beyond adds)
+    for (int t = warp - 1; t < kTok; t += kWorkers / 32) {
+      const int rix = rows[t];
+      const uint4 *srck = reinterpret_cast<const uint4 *>(ckb + (size_t)max(rix, 0) * p.rk);
+      const uint4 *srcv = reinterpret_cast<const uint4 *>(cvb + (size_t)max(rix, 0) * p.rv);
+      for (int c = lane; c < cpr_k; c += 32)
+        cp_async16_zfill(ck + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8), srck + c, rix >= 0);
+      for (int c = lane; c < cpr_v; c += 32)
+        cp_async16_zfill(cv + (size_t)(c >> 3) * kBlkBytes + sw128_offset(t, (c & 7) * 8), srcv + c, rix >= 0);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
     for (int i = wt; i < 4 * kPopBlk / 16; i += kWorkers) reinterpret_cast<uint4 *>(pop)[i] = make_uint4(0, 0, 0, 0);

@@ -160,6 +160,26 @@ __device__ __forceinline__ void proj_reduce(const float (&acc)[NV][8], int r, in
   asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");  // red is reused
 }
 
+// One pass: multiply-accumulate the batch already in `raw`, then any further batches, then reduce into dst.
+template <int NV>
+__device__ __forceinline__ void proj_pass(uint4 (&raw)[kProjBatch], const __nv_bfloat16 *basis, int r, int nrows,
+                                          int groups, int nv, const float *xs, int rows_per, float *red, float *dst,
+                                          int wt) {
+  float acc[NV][8];
+#pragma unroll
+  for (int v = 0; v < NV; ++v)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
+  int first = 0;
+  while (true) {
+    proj_fma<NV>(acc, raw, r, nrows, groups, first, nv, xs, rows_per, wt);
+    first += kProjBatch * groups;
+    if (first >= nrows) break;
+    proj_load(raw, basis, r, nrows, groups, first, wt);
+  }
+  proj_reduce<NV>(acc, r, groups, nv, red, dst, wt);
+}
+
 __device__ __forceinline__ void online_update(float &m, float &s, float z) {
   if (z <= m) {
     s += __expf(z - m);
@@ -270,31 +290,14 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
           xs[(p.G + 1) * p.rows_per + di] = x[kMaxGroup + 1];
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");
-        {
-          float acc[kMaxGroup + 1][8];
-#pragma unroll
-          for (int v = 0; v < kMaxGroup + 1; ++v)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
-          proj_fma<kMaxGroup + 1>(acc, raw_k, p.r, nrows, p.groups_k, 0, nvk, xs, p.rows_per, wt);
-          for (int first = kProjBatch * p.groups_k; first < nrows; first += kProjBatch * p.groups_k) {
-            proj_load(raw_k, bk, p.r, nrows, p.groups_k, first, wt);
-            proj_fma<kMaxGroup + 1>(acc, raw_k, p.r, nrows, p.groups_k, first, nvk, xs, p.rows_per, wt);
-          }
-          proj_reduce<kMaxGroup + 1>(acc, p.r, p.groups_k, nvk, pred, part, wt);
-        }
-        if (tok_ok) {
-          float acc[1][8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[0][e] = 0.f;
-          const float *xv = xs + (size_t)(p.G + 1) * p.rows_per;
-          proj_fma<1>(acc, raw_v, p.rv, nrows, p.groups_v, 0, 1, xv, p.rows_per, wt);
-          for (int first = kProjBatch * p.groups_v; first < nrows; first += kProjBatch * p.groups_v) {
-            proj_load(raw_v, bv, p.rv, nrows, p.groups_v, first, wt);
-            proj_fma<1>(acc, raw_v, p.rv, nrows, p.groups_v, first, 1, xv, p.rows_per, wt);
-          }
-          proj_reduce<1>(acc, p.rv, p.groups_v, 1, pred, part + (size_t)(p.G + 1) * p.r, wt);
-        }
+        // (the executed code is kept short: the scan kernel starts with cold instruction caches every step)
+        if (nvk <= 5)
+          proj_pass<5>(raw_k, bk, p.r, nrows, p.groups_k, nvk, xs, p.rows_per, pred, part, wt);
+        else
+          proj_pass<kMaxGroup + 1>(raw_k, bk, p.r, nrows, p.groups_k, nvk, xs, p.rows_per, pred, part, wt);
+        if (tok_ok)
+          proj_pass<1>(raw_v, bv, p.rv, nrows, p.groups_v, 1, xs + (size_t)(p.G + 1) * p.rows_per, p.rows_per, pred,
+                       part + (size_t)(p.G + 1) * p.r, wt);
         // the barrier at the end of proj_reduce orders every worker's stores before thread 0's release below
       }
       // flag j: this CTA has read coef_len and (if it contributes) published its partial sums
