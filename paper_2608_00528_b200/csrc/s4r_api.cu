@@ -54,6 +54,7 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   p->off_att_ms = off;  off = align_up(off + sizeof(float2) * ly.B * ly.Hq * (size_t)p->n_att_tiles, 256);
   p->off_proj = off;    off = align_up(off + sizeof(float) * ly.B * kProjMaxParts * (size_t)(((ly.G + 1) * ly.rk + ly.rv + 3) & ~3), 256);
   p->off_flag = off;    off = align_up(off + sizeof(unsigned long long) * ly.B * (kMaxParts + 1), 256);
+  p->off_qop = off;     off = align_up(off + (size_t)ly.B * ly.Hkv * 4096, 256);
   p->off_basis_t = off;
   p->total = off > 256 ? off : 256;
   if (ly.dtype == S4R_BF16 && compress_fast_workspace(ly) > p->total) p->total = compress_fast_workspace(ly);
@@ -208,6 +209,10 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
     const int parts = scan_fast_parts(ly);
     if (parts < 1 || parts > a.plan.parts_cap) fast_scan = false; else a.plan.n_parts = parts;
   }
+  // the absorbed kernel keeps U in tensor-memory columns [256, 256 + r_v) below the logit buffers at 480, and it
+  // takes its rotated-query operand from the scan kernel
+  const bool absorb = fast_scan && att_fast_supported(ly) && ly.rv <= 192 && a.value_path == S4R_VALUE_AUTO;
+  a.query_operand = absorb;
   a.fuse_projection = fast_scan && scan_fuse_supported(ly);
   if (a.fuse_projection) {
     // The fused projection identifies each call by a fresh token in its kernel arguments.  A captured graph
@@ -230,8 +235,6 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (cuda_failed(launch_relevance(a))) return S4R_ERR_CUDA;
   if (cuda_failed(launch_select(a))) return S4R_ERR_CUDA;
   stage_mark(3, a.stream);
-  // the absorbed kernel keeps U in tensor-memory columns [256, 256 + r_v) below the logit buffers at 480
-  const bool absorb = att_fast_supported(ly) && ly.rv <= 192 && a.value_path == S4R_VALUE_AUTO;
   if (absorb) {
     if (cuda_failed(launch_attend_absorb(a))) return S4R_ERR_CUDA;
   } else if (att_fast_supported(ly)) {

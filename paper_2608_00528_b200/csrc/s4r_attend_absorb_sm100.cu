@@ -13,7 +13,7 @@
 //   logits, tile softmax                         16 epilogue warps, RoPE angles held in registers
 //   U[2G x r_v]      = [P_hi; P_lo]^T C^V[rows]  tcgen05.mma, probabilities as two bf16 terms (hi + lo)
 // Warp 0 = key-basis TMA stream + issuer of the key product, warp 1 = issuer of the logit product,
-// warps 2-17 = epilogue, warp 18 = issuer of the P C^V product.
+// warps 2-17 = epilogue, warp 18 = issuer and reader of the P C^V product.
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
 
@@ -33,11 +33,12 @@ constexpr int kBlkBytes = 128 * 128;
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kThreads = 64 + kEpiThreads + 32;
-constexpr int kQopBytes = 2 * 16 * 128;  // one head's query operand: two 64-channel blocks of 16 rows
+constexpr int kQopBytes = kQueryOperandBytes;  // one head's query operand: two 64-channel blocks of 16 rows
 constexpr uint32_t kUCol = 256, kZCol = 480;  // tensor-memory columns of U and of the two logit buffers
 
 struct AbsorbParams {
   const __nv_bfloat16 *q, *coef_k, *coef_v;
+  const uint8_t *qimg;  // [B][Hkv][kQueryOperandBytes]: rotated-query operands prepared by the scan kernel
   const int32_t *coef_len, *sel_idx, *sel_count;
   float *part_u;    // [B][Hq][tiles][2 (hi, lo part of P)][rv]
   float2 *part_ms;  // [B][Hq][tiles]
@@ -88,8 +89,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
   uint64_t *full = bars, *empty = bars + kRing;
   uint64_t *k_full = bars + 2 * kRing, *rope_done = k_full + 2;
   uint64_t *z_full = rope_done + 2, *z_empty = z_full + 2;
-  uint64_t *p_ready = z_empty + 2, *u_full = p_ready + 1, *u_empty = u_full + 2;  // u_full[2]: by head parity
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(u_empty + 1);
+  // p_ready[2], u_full[2]: one barrier per head parity.  A waiter that checks phase parity must never fall two
+  // phases behind; with one barrier per parity the next completion always depends on the waiter's own progress.
+  uint64_t *p_ready = z_empty + 2, *u_full = p_ready + 2;
+  uint64_t *q_full = u_full + 2;                            // q_full[2]: query operand of a head has landed
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   int *rows = reinterpret_cast<int *>(tmem_slot + 2);   // [128]
 
@@ -109,11 +113,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
       mbar_init(&rope_done[i], kEpiWarps);
       mbar_init(&z_full[i], 1);
       mbar_init(&z_empty[i], 4);  // one warp per lane quadrant reads the logits
+      mbar_init(&q_full[i], 1);
     }
-    mbar_init(p_ready, (uint32_t)G);  // one softmax warp per query head of the group
+    mbar_init(&p_ready[0], (uint32_t)G);  // one softmax warp per query head of the group
+    mbar_init(&p_ready[1], (uint32_t)G);
     mbar_init(&u_full[0], 1);
     mbar_init(&u_full[1], 1);
-    mbar_init(u_empty, 3);  // three warps of lane quadrant 0 read U
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tmap_bk);
@@ -172,6 +177,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
   if (warp == 0) {
     // ---------------- key-basis stream (TMA, 64-column blocks, whole heads per stage) and K^ = C^K_tile (B^K)^T
     if (lane == 0) {
+      for (int h = 0; h < min(2, p.nkv); ++h) {  // query operands of the first two heads (fresh buffers)
+        mbar_expect_tx(&q_full[h], kQopBytes);
+        bulk_load(qop + (size_t)h * kQopBytes, p.qimg + ((size_t)b * p.Hkv + kv0 + h) * kQopBytes, kQopBytes, &q_full[h]);
+      }
       const int pre = min(n_stages, p.nkv);
       for (int h = 0; h < pre; ++h) {  // fresh stages: no wait
         mbar_expect_tx(&full[h], (uint32_t)kbk * kBlkBytes);
@@ -206,6 +215,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
           if (mbar_test(&full[st], (uint32_t)(hk / n_stages) & 1u) &&
               (hk < 2 || mbar_test(&z_full[buf], (uint32_t)((hk - 2) >> 1) & 1u))) {
             tc_fence_after();
+            if (hk >= 2) {  // the logit product of head hk - 2 has also released this query-operand buffer
+              mbar_expect_tx(&q_full[buf], kQopBytes);
+              bulk_load(qop + (size_t)buf * kQopBytes, p.qimg + ((size_t)b * p.Hkv + kv0 + hk) * kQopBytes, kQopBytes,
+                        &q_full[buf]);
+            }
             const uint64_t bs_desc = umma_desc_sw128(smem_u32(ring + (size_t)st * kbk * kBlkBytes));
             for (int blk = 0; blk < kbk; ++blk) {
 #pragma unroll
@@ -255,6 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
         const uint32_t ph = (uint32_t)(h >> 1) & 1u;
         if (!mbar_wait(&rope_done[buf], ph, abort_flag)) break;
         if (!mbar_wait(&z_empty[buf], ph ^ 1u, abort_flag)) break;
+        if (!mbar_wait(&q_full[buf], ph, abort_flag)) break;
         tc_fence_after();
         const uint64_t q_desc = umma_desc_sw128(smem_u32(qop + (size_t)buf * kQopBytes));
 #pragma unroll
@@ -267,24 +282,50 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
       }
     }
   } else if (warp == 2 + kEpiWarps) {
-    // ---------------- U = [P_hi; P_lo]^T C^V over the 128 tokens of the tile (8 steps of 16 tokens)
+    // ---------------- U = [P_hi; P_lo] C^V over the 128 tokens of the tile (8 steps of 16 tokens), issued and
+    // read back by this warp.  The probability rows sit at M index 64.. of the A operand (the descriptor starts
+    // 8 KB before the stored rows; the rows in front of them read whatever is there and land in lanes nobody
+    // reads), so the result occupies tensor-memory lanes 64.., the quadrant this warp may load.
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     fence_proxy_async_smem();
     asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
-    if (lane == 0) {
-      const uint32_t idesc_u = umma_idesc_bf16(128, p.rv) | (1u << 16);  // B operand N-contiguous
-      const uint64_t cv_desc = umma_desc_mn_sw128(smem_u32(cv), kBlkBytes);
-      const uint64_t pop_desc = umma_desc_sw128(smem_u32(pop));
-      for (int h = 0; h < p.nkv; ++h) {
-        if (!mbar_wait(p_ready, (uint32_t)h & 1u, abort_flag)) break;
-        if (!mbar_wait(u_empty, ((uint32_t)h & 1u) ^ 1u, abort_flag)) break;
-        tc_fence_after();
+    const uint32_t idesc_u = umma_idesc_bf16(128, p.rv) | (1u << 16);  // B operand N-contiguous
+    const uint64_t cv_desc = umma_desc_mn_sw128(smem_u32(cv), kBlkBytes);
+    const uint64_t pop_desc = umma_desc_sw128(smem_u32(pop) - 8192u);
+    const int part = lane < G ? 0 : 1, g = lane < G ? lane : lane - G;
+    bool ok = true;
+    for (int h = 0; h < p.nkv; ++h) {
+      if (ok) ok = mbar_wait(&p_ready[h & 1], (uint32_t)(h >> 1) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      if (lane == 0) {
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           umma_bf16(tmem_base + kUCol, pop_desc + (uint64_t)((((h & 1) * 2 + (kk >> 2)) * kPopBlk + (kk & 3) * 32) >> 4),
                     cv_desc + (uint64_t)((kk * 2048) >> 4), idesc_u, kk != 0);
         umma_commit(&u_full[h & 1]);
       }
+      __syncwarp();
+      ok = mbar_wait(&u_full[h & 1], (uint32_t)(h >> 1) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      // lanes 0..G-1 hold the hi part, G..2G-1 the lo part of head kv*G + g (k_merge_absorb adds them)
+      float *dst = p.part_u + ((((size_t)b * p.Hq + (size_t)(kv0 + h) * G + min(g, G - 1)) * p.n_tiles + tile) * 2 + part) * p.rv;
+      for (int c0 = 0; c0 < p.rv; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem_base + kUCol + (uint32_t)c0 + (64u << 16), v);
+        tmem_ld_wait();
+        if (lane < 2 * G) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4 *>(dst + c0 + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                    __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
     }
   } else {
     // ---------------- epilogue: 16 warps; warps e, e+4, e+8, e+12 share a TMEM lane quadrant ----------------
@@ -304,47 +345,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
       for (int ii = 0; ii < 16; ++ii)
         sc[ii] = (rope && rix >= 0) ? pack_sincos(p.s + rix, p.rope_turns[qt * 16 + ii]) : 0xffff8000u;  // (0, 1)
     }
-    // q' = RoPE(q) / sqrt(d_h) as hi + lo bf16 rows of the logit product's B operand; this thread prepares column
-    // qc for the heads g = qg0, qg0 + 4.  The raw values are fetched one head ahead of their use.
-    const int qc = et & 127, qg0 = et >> 7;
-    float q_sn = 0.f, q_cs = 1.f;
-    if (rope) rope_sincos(p.s + L - 1, p.rope_turns[qc & 63], q_sn, q_cs);
-    const float q_scale = rsqrtf((float)kDh);
-    // raw bf16 bits; widened only where they are used, so that the loads stay in flight across a whole head
-    unsigned short q_raw[2][2];  // [g slot][own, partner]
-    auto fetch_q = [&](int h) {
-#pragma unroll
-      for (int sl = 0; sl < 2; ++sl) {
-        const int g = qg0 + 4 * sl;
-        q_raw[sl][0] = q_raw[sl][1] = 0;
-        if (g < G && h < p.nkv) {
-          const unsigned short *qp =
-              reinterpret_cast<const unsigned short *>(p.q + ((size_t)b * p.Hq + (size_t)(kv0 + h) * G + g) * kDh);
-          q_raw[sl][0] = __ldg(qp + qc);
-          q_raw[sl][1] = __ldg(qp + (qc ^ 64));
-        }
-      }
-    };
-    // position of channel qc in the K order of the logit product: steps of {8 channels of the lower half of the
-    // head, their 8 rotation partners}
-    const int q_col = ((qc & 63) >> 3) * 16 + (qc >> 6) * 8 + (qc & 7);
-    auto store_q = [&](int h) {
-      uint8_t *qb = qop + (size_t)(h & 1) * kQopBytes + (size_t)(q_col >> 6) * 2048;
-#pragma unroll
-      for (int sl = 0; sl < 2; ++sl) {
-        const int g = qg0 + 4 * sl;
-        if (g < G) {
-          float v = __uint_as_float((uint32_t)q_raw[sl][0] << 16);
-          const float o = __uint_as_float((uint32_t)q_raw[sl][1] << 16);
-          if (rope) v = (qc < 64) ? v * q_cs - o * q_sn : v * q_cs + o * q_sn;
-          v *= q_scale;
-          const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-          const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-          *reinterpret_cast<__nv_bfloat16 *>(qb + sw128_offset(g, q_col & 63)) = hi;
-          *reinterpret_cast<__nv_bfloat16 *>(qb + sw128_offset(8 + g, q_col & 63)) = lo;
-        }
-      }
-    };
     // K^ row of this thread's token, pairs [16 qt, +16), in two halves of 8 pairs (d1 = 16 qt + 8 half + j,
     // d2 = d1 + 64): rotate, split into hi + lo bf16 by truncation (hi = upper 16 bits of the fp32 value, lo =
     // upper 16 bits of the exact remainder; together 16 significand bits) and write back over the half's own 16
@@ -402,59 +402,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
       if (lane == 0) mbar_arrive(&rope_done[buf]);
       return ok2;
     };
-    // U of one head: TMEM lanes 0..G-1 hold the hi part, G..2G-1 the lo part; three warps of lane quadrant 0 that
-    // have no part in the softmax (e = 6, 10, 14) split the columns and store both parts
-    // (k_merge_absorb adds them)
-    const bool u_reader = (e == 6 || e == 10 || e == 14);
-    const int u_part = (e - 6) >> 2;
-    auto read_u = [&](int h, bool ok_in) -> bool {
-      bool ok2 = ok_in;
-      if (ok2) ok2 = mbar_wait(&u_full[h & 1], (uint32_t)(h >> 1) & 1u, abort_flag);
-      ok2 = __all_sync(0xffffffffu, ok2);
-      tc_fence_after();
-      if (ok2) {
-        const int part = lane < G ? 0 : 1, g = lane < G ? lane : lane - G;
-        float *dst = p.part_u + ((((size_t)b * p.Hq + (size_t)(kv0 + h) * G + min(g, G - 1)) * p.n_tiles + tile) * 2 + part) * p.rv;
-        for (int c0 = u_part * 16; c0 < p.rv; c0 += 48) {
-          uint32_t v[16];
-          tmem_ld16(tmem_base + kUCol + (uint32_t)c0, v);
-          tmem_ld_wait();
-          if (lane < 2 * G) {
-#pragma unroll
-            for (int j = 0; j < 16; j += 4)
-              *reinterpret_cast<float4 *>(dst + c0 + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                                      __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-          }
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(u_empty);
-      }
-      return ok2;
-    };
-    fetch_q(0);
-    for (int i = et; i < 2 * kQopBytes / 16; i += kEpiThreads) reinterpret_cast<uint4 *>(qop)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    epi_sync();  // query operand cleared (rows past G stay zero)
-    store_q(0);
-    fetch_q(1);
     fence_proxy_async_smem();
-    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");  // tiles gathered, operands cleared, q' of head 0 set
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");  // tiles gathered, probability operand cleared
     bool ok = true;  // warp-uniform; after a failed wait the loop keeps its shape but touches tensor memory no more
     ok = rotate(0, ok);
     for (int h = 0; h < p.nkv; ++h) {
       const int kv = kv0 + h, zb = h & 1;
-      if (h + 1 < p.nkv) {
-        // the other q' buffer was last read by the logit product of head h - 1
-        if (h >= 1) {
-          if (ok) ok = mbar_wait(&z_full[zb ^ 1], (uint32_t)((h - 1) >> 1) & 1u, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);
-        }
-        store_q(h + 1);
-        fetch_q(h + 2);
-        fence_proxy_async_smem();
-        ok = rotate(h + 1, ok);  // runs one head ahead of the softmax
-      }
+      if (h + 1 < p.nkv) ok = rotate(h + 1, ok);  // runs one head ahead of the softmax
       // ---- logits of this head: one warp per lane quadrant (e = 4..7) moves them from tensor memory to shared memory
       if (qt == 1) {
         if (ok) ok = mbar_wait(&z_full[zb], (uint32_t)(h >> 1) & 1u, abort_flag);
@@ -502,11 +457,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_absorb(const __grid_cons
         if (lane == 0) p.part_ms[((size_t)b * p.Hq + (size_t)kv * G + e) * p.n_tiles + tile] = make_float2(m, ssum);
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(p_ready);
+        if (lane == 0) mbar_arrive(&p_ready[h & 1]);
       }
-      if (u_reader && h > 0) ok = read_u(h - 1, ok);  // the previous head's U
     }
-    if (u_reader) ok = read_u(p.nkv - 1, ok);
   }
   tc_fence_before();
   __syncthreads();
@@ -697,6 +650,8 @@ cudaError_t launch_attend_absorb(const StepArgs &a) {
   if (!make_tmap_bf16_2d(&tm_k, a.basis_k, (uint64_t)ly.B * ly.D, (uint64_t)ly.rk, 128)) return cudaErrorInvalidValue;
   AbsorbParams p;
   p.q = (const __nv_bfloat16 *)a.q;
+  p.qimg = (const uint8_t *)(a.ws + a.plan.off_qop);
+  if (!a.query_operand) return cudaErrorInvalidValue;  // the scan kernel must have prepared the operands
   p.coef_k = (const __nv_bfloat16 *)a.coef_k;
   p.coef_v = (const __nv_bfloat16 *)a.coef_v;
   p.coef_len = a.coef_len;

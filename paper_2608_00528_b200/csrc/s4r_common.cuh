@@ -150,7 +150,7 @@ struct DecodePlan {
   int n_att_tiles;      // row tiles per sequence in the attention kernel
   int cluster;          // CTAs per sequence in the selection kernel
   int att_tok;          // selected rows per attention tile
-  size_t off_cq, off_z, off_part, off_score, off_hist, off_att, off_att_ms, off_proj, off_flag, off_basis_t, total;
+  size_t off_cq, off_z, off_part, off_score, off_hist, off_att, off_att_ms, off_proj, off_flag, off_qop, off_basis_t, total;
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -19,6 +19,7 @@ struct StepArgs {
   void *coef_k_w = nullptr, *coef_v_w = nullptr;
   int32_t *coef_len_w = nullptr;
   bool fuse_projection = false;  // Eq. 5-6 run inside the scan kernel; no projection kernel is launched
+  bool query_operand = false;    // the scan kernel also prepares the attention kernel's rotated-query operand
   int window, top_k, kappa, pool_mode, group_mode, value_path;
   float theta;
   void *out;

@@ -31,6 +31,7 @@ using namespace sm100;
 
 bool scan_fast_supported(const Layer &ly);
 int scan_fast_parts(const Layer &ly);
+void fill_rope_turns(uint64_t *dst, int head_dim, float theta);
 
 namespace {
 
@@ -50,6 +51,11 @@ struct ScanFastParams {
   unsigned long long *proj_flag;  // [B][cps + 1]: one per CTA of the sequence, then "token rows stored"
   unsigned long long token;
   unsigned *hist;                 // [B][2048], cleared here for the relevance kernel
+  // rotated-query operand of the attention kernel (nullptr: not wanted)
+  uint8_t *qimg;                  // [B][Hkv][kQueryOperandBytes]
+  int Hkv, sinks;
+  float theta;
+  uint64_t rope_turns[64];
   const float *cq_part;
   const int32_t *coef_len;
   float *Z;
@@ -384,6 +390,39 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
     fence_proxy_async_smem();
     asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");  // B operand complete (producer not involved)
     if (wt == 0) mbar_arrive(proj_bar);
+    // ---- Off the critical path: the attention kernel's logit product wants q' = RoPE(q) / sqrt(d_h) of every KV
+    //      head as a ready-made tensor-core operand (hi + lo bf16 rows, swizzled).  CTA j of the sequence prepares
+    //      heads j, j + cps, ...; the first tiles are already in flight.
+    if (p.qimg != nullptr) {
+      const bool rope = p.theta > 0.f;
+      const float scale = rsqrtf((float)p.dh);
+      for (int kv = j; kv < p.Hkv; kv += p.cps) {
+        uint8_t *img = p.qimg + ((size_t)b * p.Hkv + kv) * kQueryOperandBytes;
+        // rows that carry no query stay zero: G..7 and 8+G..15, 16 pieces of 16 bytes each
+        for (int i = wt; i < 2 * (8 - p.G) * 16; i += kWorkers) {
+          const int row = (i >> 4) < 8 - p.G ? p.G + (i >> 4) : 8 + p.G + ((i >> 4) - (8 - p.G));
+          const int piece = i & 15;
+          *reinterpret_cast<uint4 *>(img + (size_t)(piece >> 3) * 2048 + (row >> 3) * 1024 + (row & 7) * 128 + (piece & 7) * 16) =
+              make_uint4(0, 0, 0, 0);
+        }
+        for (int i = wt; i < p.G * p.dh; i += kWorkers) {
+          const int g = i >> 7, c = i & 127;  // d_h = 128 on this path
+          const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)kv * p.G + g) * p.dh;
+          float v = __bfloat162float(qp[c]);
+          if (rope) {
+            const float o = __bfloat162float(qp[c ^ 64]);
+            float sn, cs;
+            rope_sincos(p.sinks + L - 1, p.rope_turns[c & 63], sn, cs);
+            v = c < 64 ? v * cs - o * sn : v * cs + o * sn;
+          }
+          v *= scale;
+          const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+          *reinterpret_cast<__nv_bfloat16 *>(img + query_operand_offset(g, c)) = hi;
+          *reinterpret_cast<__nv_bfloat16 *>(img + query_operand_offset(8 + g, c)) = lo;
+        }
+      }
+    }
   }
 
   if (warp == 0) {
@@ -609,6 +648,10 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
   p.proj_part = (float *)(a.ws + a.plan.off_proj);
   p.proj_flag = (unsigned long long *)(a.ws + a.plan.off_flag);
   p.hist = (unsigned *)(a.ws + a.plan.off_hist);
+  p.qimg = a.query_operand && ly.dh == 128 ? (uint8_t *)(a.ws + a.plan.off_qop) : nullptr;
+  if (a.query_operand && !p.qimg) return cudaErrorInvalidValue;
+  p.Hkv = ly.Hkv; p.sinks = ly.s; p.theta = a.theta;
+  fill_rope_turns(p.rope_turns, ly.dh, a.theta);
   // per-call token: unique within the process (counter) and seeded per process, so that flags left in recycled
   // device memory by an earlier call or an earlier process never match
   static std::atomic<unsigned long long> token_source{

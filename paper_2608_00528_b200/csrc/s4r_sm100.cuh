@@ -161,6 +161,23 @@ __device__ __forceinline__ uint32_t sw128_offset(int row, int col) {
          ((uint32_t)col & 7u) * 2u;
 }
 
+// The rotated, scaled query of one KV head as the B operand of the attention kernel's logit product: two
+// swizzled blocks of 64 K-elements x 16 rows (row g: hi part of q'[g], row 8 + g: lo part).  The K order pairs
+// each channel with its rotation partner: K-step ks = channels {8 ks .. 8 ks + 7, 64 + 8 ks .. 64 + 8 ks + 7}.
+constexpr int kQueryOperandBytes = 2 * 16 * 128;
+__host__ __device__ inline uint32_t query_operand_offset(int row, int channel) {
+  const int col = ((channel & 63) >> 3) * 16 + (channel >> 6) * 8 + (channel & 7);
+  const int r = row, c = col & 63;
+  return (uint32_t)(col >> 6) * 2048u + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u +
+         ((((uint32_t)c >> 3) ^ ((uint32_t)r & 7u)) << 4) + ((uint32_t)c & 7u) * 2u;
+}
+// 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion on an mbarrier
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
 // 32 lanes x 32 columns of fp32 accumulators -> 32 registers per thread (thread = TMEM lane)
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(

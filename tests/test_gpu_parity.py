@@ -362,3 +362,39 @@ def test_decode_step_replayed_from_a_cuda_graph():
                 ref = (out.clone(), sel.clone())
             else:
                 assert torch.equal(out, ref[0]) and torch.equal(sel, ref[1])
+
+
+@pytest.mark.parametrize("theta", [None, 0.0])
+def test_many_back_to_back_steps_stay_in_step(theta):
+    """The kernels hand work between warp roles through phase-parity barriers; a role that fell two phases behind
+    would wait out its bound and raise S4R_DEV_TIMEOUT.  Several hundred steps back to back (with and without
+    the RoPE work, which changes the relative speed of the roles) must leave the status word clear and give the
+    same bits every time."""
+    s4r = _s4r()
+    cfg = _cfg(2, context=16384 + 4, batch=8)
+    p = Problem(_cfg(2, context=16384 + 4, batch=1), device="cuda").upload()      # one checked sequence ...
+    B = cfg.batch
+    rep = lambda t: t.expand(B, *t.shape[1:]).contiguous()                         # ... replicated over the batch
+    ly = s4r.Layer(B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rank_k, cfg.rank_v, cfg.sink_count, s4r.S4R_BF16,
+                   p.cap)
+    d = dict(q=rep(p.d_q), sk=rep(p.d_sink_k), sv=rep(p.d_sink_v), ck=rep(p.d_CK), cv=rep(p.d_CV), ln=rep(p.d_len),
+             bk=rep(p.d_BK), bv=rep(p.d_BV))
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(B, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(B, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    th = cfg.rope_theta if theta is None else theta
+    first = None
+    for i in range(300):
+        s4r.decode_step(ly, d["q"], d["sk"], d["sv"], d["ck"], d["cv"], d["ln"], d["bk"], d["bv"], p.cap, cfg.window,
+                        cfg.top_k, out, sel, cnt, ws, rope_theta=th, dev_status=status)
+        if i in (0, 149, 299):
+            torch.cuda.synchronize()
+            assert status.item() == 0
+            if first is None:
+                first = (out.clone(), sel.clone())
+                check_step(p, out[:1], sel[:1], cnt[:1], theta=theta)
+                assert all(torch.equal(out[b], out[0]) and torch.equal(sel[b], sel[0]) for b in range(1, B))
+            else:
+                assert torch.equal(out, first[0]) and torch.equal(sel, first[1])
