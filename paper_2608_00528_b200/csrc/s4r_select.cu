@@ -23,7 +23,7 @@ namespace {
 constexpr int kRelThreads = 256;
 constexpr int kRelOut = 120;                // positions a warp emits per chunk (128 held, 4 halo on each side)
 constexpr int kRelChunks = 2;               // consecutive chunks per warp
-constexpr int kSliceCap = 16384;            // scores of a slice kept in shared memory up to this many
+constexpr int kSliceMax = 49152;            // scores of a slice kept in shared memory up to this many (192 KB)
 
 struct RelParams {
   const float *Z;
@@ -41,6 +41,7 @@ struct SelParams {
   const unsigned *hist;
   int32_t *sel_idx, *sel_count;
   int window, top_k;
+  int slice_cap;  // floats of dynamic shared memory for the slice
   int64_t max_len, z_stride;
   int32_t *dev_status;
 };
@@ -296,7 +297,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
   const int CL = cluster.num_blocks();
   const int rank = cluster.block_rank();
   const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  extern __shared__ __align__(16) float s_score[];  // [kSliceCap]
+  extern __shared__ __align__(16) float s_score[];  // [p.slice_cap]
   __shared__ unsigned s_hist[2048];
   __shared__ unsigned s_tot[2048];              // cluster-wide histogram, used in rank 0 only
   __shared__ unsigned s_cnts[kMaxCluster][2];   // (greater, equal) counts of the lower-ranked CTAs
@@ -340,7 +341,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
   per = (per + 3) & ~3;
   const int begin = min(n_cand, rank * per), c_end = min(n_cand, begin + per);
   const float *gscore = p.score + (size_t)b * p.z_stride;
-  const bool in_smem = per <= kSliceCap;
+  const bool in_smem = per <= p.slice_cap;
   for (int l0 = begin + 4 * tid; l0 < c_end; l0 += 4 * kSelThreads) {
     float v[4] = {0.f, 0.f, 0.f, 0.f};
     if (l0 + 3 < c_end) {
@@ -485,7 +486,11 @@ cudaError_t launch_select(const StepArgs &a) {
   p.max_len = a.plan.max_len;
   p.z_stride = a.plan.z_stride;
   p.dev_status = a.dev_status;
-  const size_t smem = sizeof(float) * (size_t)kSliceCap;
+  // shared-memory room for one CTA's slice of the candidates at the largest length this launch can meet
+  int64_t per = (a.plan.max_len + a.plan.cluster - 1) / a.plan.cluster;
+  per = (per + 3) & ~(int64_t)3;
+  p.slice_cap = (int)(per < 4096 ? 4096 : (per > kSliceMax ? kSliceMax : per));
+  const size_t smem = sizeof(float) * (size_t)p.slice_cap;
   static size_t smem_set = 0;
   if (smem > smem_set) {
     cudaError_t e = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
