@@ -19,7 +19,8 @@ namespace {
 
 constexpr int kMTile = 256;
 constexpr int kStages = 3;
-constexpr int kCmpThreads = 192;
+constexpr int kCmpEpiWarps = 8;  // two warps per tensor-memory lane quadrant: even / odd chunks of 32 columns
+constexpr int kCmpThreads = 64 + 32 * kCmpEpiWarps;
 
 struct CompressParams {
   __nv_bfloat16 *coef;
@@ -69,7 +70,7 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
       mbar_init(&empty[i], 1);
     }
     mbar_init(acc_full, 1);
-    mbar_init(acc_empty, 4);  // one arrival per epilogue warp
+    mbar_init(acc_empty, kCmpEpiWarps);  // one arrival per epilogue warp
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tmap_x);
@@ -140,7 +141,10 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
       }
     }
   } else {
-    const int quad = warp & 3;
+    // The accumulators are single-buffered (two of 192 columns fill tensor memory), so the next item's products
+    // wait for this read-back: it is spread over eight warps and hands the accumulators back as soon as the last
+    // values are in registers.
+    const int quad = warp & 3, chunk_par = (warp - 2) >> 2;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     int n_done = 0;
     bool ok = true;
@@ -154,10 +158,15 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
       for (int half = 0; half < 2; ++half) {
         const int64_t row = (int64_t)mt * kMTile + half * 128 + quad * 32 + lane;
         __nv_bfloat16 *dst = p.coef + ((size_t)b * p.cap + (size_t)row) * p.r;
-        for (int c0 = 0; c0 < p.r; c0 += 32) {
+        for (int c0 = chunk_par * 32; c0 < p.r; c0 += 64) {
           uint32_t v[32];
           tmem_ld32(tmem_base + (uint32_t)half * 256u + lane_addr + (uint32_t)c0, v);
           tmem_ld_wait();
+          if (half == 1 && c0 + 64 >= p.r) {  // last read of this warp for the item
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty);
+          }
           if (row < n_rows) {
 #pragma unroll
             for (int j = 0; j < 32; j += 8) {
@@ -177,9 +186,11 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty);
+      if (chunk_par * 32 >= p.r) {  // a warp without columns (r <= 32) still owes its arrival
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty);
+      }
     }
   }
   tc_fence_before();
