@@ -92,7 +92,8 @@ typedef struct {
 /* Switches of the relevance estimate (Eq. 9-12); the paper's defaults are
  * pool_kernel 7, max pooling, mean aggregation. */
 typedef struct {
-  int32_t score_window; /* number of query-coefficient rows scored; only 1 (the current query) is built */
+  int32_t score_window; /* W_q, query-coefficient rows scored (Eq. 7, 9, 10): 1 = the current query alone; more
+                           than 1 only through s4r_decode_step_windowed */
   int32_t pool_kernel;  /* kappa, odd, 1 = no pooling, <= 31                              */
   int32_t pool_mode;    /* S4R_POOL_MAX | S4R_POOL_AVG                                    */
   int32_t group_mode;   /* S4R_GROUP_MEAN | S4R_GROUP_MAX                                 */
@@ -113,6 +114,11 @@ typedef struct {
  * than max_len non-sink rows (compress: max_len = T - s).  0 on invalid arguments.  The workspace
  * must be 256-byte aligned; its contents are undefined between calls. */
 size_t s4r_workspace_bytes(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k);
+
+/* The same for s4r_decode_step_windowed with W_q = score_window (W_q * G <= S4R_MAX_SCORE_ROWS, else 0). */
+#define S4R_MAX_SCORE_ROWS 32
+size_t s4r_workspace_bytes_windowed(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k,
+                                    int32_t score_window);
 
 /* Prefill-side projection (Sec. 3.1.1 sink split + Eq. 3), per sequence b:
  *   sink_k[b] = K[b, 0:s], sink_v[b] = V[b, 0:s]            (verbatim copies)
@@ -155,13 +161,34 @@ int s4r_append(const s4r_layer_t *layer, const void *k_t, const void *v_t, const
  *               non-sink indices (absolute position = s + index); unused tail = -1.  Sinks are always
  *               attended and never listed.
  * sel_count     [B] int32 = W_eff + k_eff
- * Returns S4R_ERR_UNSUPPORTED for score->score_window != 1. */
+ * Returns S4R_ERR_UNSUPPORTED for score->score_window != 1 (see s4r_decode_step_windowed). */
 int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
                     const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,
                     const void *value_basis, int64_t max_len, int32_t window, int32_t top_k,
                     const s4r_score_t *score, const s4r_rope_t *rope, void *out, int32_t out_dtype,
                     int32_t *sel_idx, int32_t *sel_count, void *workspace, size_t workspace_bytes,
                     int32_t *dev_status, void *stream);
+
+/* The decode step with the paper's full relevance estimator (Sec. 3.2.2): a FIFO of the W_q = score->score_window
+ * most recent projected queries scores the cache instead of the current query alone.
+ *   Eq. 7   the window drops its oldest row and appends c^Q of the current query (so it always holds W_q rows)
+ *   Eq. 8-9 window row i (0 = oldest) belongs to the token at non-sink index L - W_q + i; its latent logits are
+ *           softmax-normalised over the rows l <= L - W_q + i it may see (causal mask); rows with a negative
+ *           index see nothing
+ *   Eq. 10  the W_q probability rows of a query group are averaged (divided by W_q)
+ * followed by pooling, group aggregation, selection, reconstruction and attention exactly as in s4r_decode_step.
+ * query_window  [B, W_q, G, rank_k] fp32, caller-owned per-layer state, oldest row first; updated in place.  Before
+ *               the first step the caller fills rows 1..W_q-1 with the coefficients of the W_q - 1 preceding
+ *               queries (Eq. 4: C^Q = Q~ B^K; zeros if there are none) - row 0 is dropped by that step.
+ * Built for bf16 caches with rank_k a multiple of 64 on sm_100 (S4R_ERR_UNSUPPORTED otherwise, and for
+ * W_q * G > S4R_MAX_SCORE_ROWS).  The cache is scanned once per block of eight window rows.
+ * workspace_bytes >= s4r_workspace_bytes_windowed(...).  All other arguments as in s4r_decode_step. */
+int s4r_decode_step_windowed(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
+                             const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,
+                             const void *value_basis, int64_t max_len, int32_t window, int32_t top_k,
+                             const s4r_score_t *score, const s4r_rope_t *rope, float *query_window, void *out,
+                             int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
+                             size_t workspace_bytes, int32_t *dev_status, void *stream);
 
 /* s4r_append followed by s4r_decode_step as one call (Sec. 3.2.1 then 3.2.2-3.2.3): the new token's key and
  * value rows are projected in the same pass over the bases that projects the query (Eq. 5), appended

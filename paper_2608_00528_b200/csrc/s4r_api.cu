@@ -61,6 +61,25 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
   return true;
 }
 
+// Extra scratch of windowed scoring, laid out after the standard plan
+struct WindowPlan {
+  int rows, blocks, rows_alloc;
+  size_t off_z, off_part, off_zmean, off_unit, total;
+};
+static bool plan_window(const Layer &ly, const DecodePlan &dp, int score_window, WindowPlan *w) {
+  if (score_window < 1 || (int64_t)score_window * ly.G > kMaxScoreRows) return false;
+  w->rows = score_window * ly.G;
+  w->blocks = (w->rows + kMaxGroup - 1) / kMaxGroup;
+  w->rows_alloc = w->blocks * kMaxGroup;
+  size_t off = align_up(dp.total, 256);
+  w->off_z = off;      off = align_up(off + sizeof(float) * ly.B * (size_t)w->rows_alloc * dp.z_stride, 256);
+  w->off_part = off;   off = align_up(off + sizeof(float2) * (size_t)w->blocks * ly.B * dp.parts_cap * kMaxGroup, 256);
+  w->off_zmean = off;  off = align_up(off + sizeof(float) * ly.B * (size_t)ly.G * dp.z_stride, 256);
+  w->off_unit = off;   off = align_up(off + sizeof(float2) * ly.B * kMaxGroup, 256);
+  w->total = off;
+  return true;
+}
+
 static int check_arch() {
   static int cached[64];  // 0 unknown, 1 ok, 2 wrong architecture
   int dev = 0;
@@ -112,6 +131,16 @@ size_t s4r_workspace_bytes(const s4r_layer_t *layer, int64_t max_len, int32_t wi
   if (!layer_ok(layer, &ly) || layer_supported(ly) != S4R_OK) return 0;
   if (!plan_decode(ly, max_len, window, top_k, &p)) return 0;
   return p.total;
+}
+
+size_t s4r_workspace_bytes_windowed(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k,
+                                    int32_t score_window) {
+  Layer ly;
+  DecodePlan p;
+  WindowPlan w;
+  if (!layer_ok(layer, &ly) || layer_supported(ly) != S4R_OK) return 0;
+  if (!plan_decode(ly, max_len, window, top_k, &p) || !plan_window(ly, p, score_window, &w)) return 0;
+  return w.total;
 }
 
 int s4r_compress(const s4r_layer_t *layer, const void *K, const void *V, int64_t T, const void *key_basis,
@@ -168,7 +197,7 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
                        const int32_t *coef_len, const void *key_basis, const void *value_basis, int64_t max_len,
                        int32_t window, int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out,
                        int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
-                       size_t workspace_bytes, int32_t *dev_status, void *stream) {
+                       size_t workspace_bytes, int32_t *dev_status, void *stream, float *query_window = nullptr) {
   launch_counter() = 0;
   StepArgs a;
   if (!layer_ok(layer, &a.ly)) return S4R_ERR_INVALID_ARG;
@@ -185,13 +214,20 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (sc.pool_mode != S4R_POOL_MAX && sc.pool_mode != S4R_POOL_AVG) return S4R_ERR_INVALID_ARG;
   if (sc.group_mode != S4R_GROUP_MEAN && sc.group_mode != S4R_GROUP_MAX) return S4R_ERR_INVALID_ARG;
   if (sc.value_path != S4R_VALUE_AUTO && sc.value_path != S4R_VALUE_RECONSTRUCT) return S4R_ERR_INVALID_ARG;
-  if (sc.score_window != 1) return S4R_ERR_UNSUPPORTED;
+  if (!query_window && sc.score_window != 1) return S4R_ERR_UNSUPPORTED;  // windowed scoring has its own entry point
   if (sc.pool_kernel > 2 * kMaxPoolHalf + 1) return S4R_ERR_UNSUPPORTED;
   if (rope && rope->reserved != 0) return S4R_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(coef_k) || !aligned16(coef_v) || !aligned16(key_basis) || !aligned16(value_basis))
     return S4R_ERR_INVALID_ARG;
   if (!plan_decode(ly, max_len, window, top_k, &a.plan)) return S4R_ERR_INVALID_ARG;
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < a.plan.total)
+  WindowPlan wp = {};
+  if (query_window) {
+    if ((int64_t)sc.score_window * ly.G > kMaxScoreRows || k_t) return S4R_ERR_UNSUPPORTED;
+    if (!plan_window(ly, a.plan, sc.score_window, &wp)) return S4R_ERR_INVALID_ARG;
+    if (!scan_fast_supported(ly)) return S4R_ERR_UNSUPPORTED;  // bf16 caches with a rank that is a multiple of 64
+  }
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+      workspace_bytes < (query_window ? wp.total : a.plan.total))
     return S4R_ERR_WORKSPACE;
   if (int rc = check_arch()) return rc;
   a.q = q; a.sink_k = sink_k; a.sink_v = sink_v; a.coef_k = coef_k; a.coef_v = coef_v; a.coef_len = coef_len;
@@ -213,7 +249,8 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   // takes its rotated-query operand from the scan kernel
   const bool absorb = fast_scan && att_fast_supported(ly) && ly.rv <= 192 && a.value_path == S4R_VALUE_AUTO;
   a.query_operand = absorb;
-  a.fuse_projection = fast_scan && scan_fuse_supported(ly);
+  a.fuse_projection = fast_scan && scan_fuse_supported(ly) && !query_window;
+  if (query_window && !fast_scan) return S4R_ERR_UNSUPPORTED;
   if (a.fuse_projection) {
     // The fused projection identifies each call by a fresh token in its kernel arguments.  A captured graph
     // would replay the same token, so under stream capture the projection runs as its own kernel instead.
@@ -226,7 +263,40 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   stage_mark(0, a.stream);
   if (!a.fuse_projection && cuda_failed(launch_qproj(a))) return S4R_ERR_CUDA;
   stage_mark(1, a.stream);
-  if (fast_scan) {
+  if (query_window) {
+    // Eq. 7: shift the window and append the current query's coefficients; Eq. 8-9 for every window row in blocks
+    // of up to eight rows (one pass over C^K per block); Eq. 10: average per query group
+    const int Wq = sc.score_window;
+    if (cuda_failed(launch_window_shift(query_window, (const float *)(a.ws + a.plan.off_cq), ly.B, Wq, ly.G * ly.rk,
+                                        a.stream)))
+      return S4R_ERR_CUDA;
+    float *zw = (float *)(a.ws + wp.off_z);
+    float2 *partw = (float2 *)(a.ws + wp.off_part);
+    for (int blk = 0; blk < wp.blocks; ++blk) {
+      ScanRows sr;
+      sr.cq = query_window + (size_t)blk * kMaxGroup * ly.rk;
+      sr.cq_batch_stride = (int64_t)wp.rows * ly.rk;
+      sr.Z = zw + (size_t)blk * kMaxGroup * a.plan.z_stride;
+      sr.z_batch_stride = (int64_t)wp.rows_alloc * a.plan.z_stride;
+      sr.part = partw + (size_t)blk * ly.B * a.plan.parts_cap * kMaxGroup;
+      sr.n_rows = wp.rows - blk * kMaxGroup < kMaxGroup ? wp.rows - blk * kMaxGroup : kMaxGroup;
+      for (int g = 0; g < kMaxGroup; ++g) {
+        const int i = (blk * kMaxGroup + g) / ly.G;  // window row (oldest first) of scored row g of this block
+        sr.row_off[g] = i + 1 - Wq;
+      }
+      sr.first = blk == 0;
+      a.scan_rows = &sr;
+      const bool failed = cuda_failed(launch_scan_sm100(a));
+      a.scan_rows = nullptr;
+      if (failed) return S4R_ERR_CUDA;
+    }
+    float *zmean = (float *)(a.ws + wp.off_zmean);
+    float2 *unit = (float2 *)(a.ws + wp.off_unit);
+    if (cuda_failed(launch_window_mean(a, zw, partw, zmean, unit, Wq, wp.rows_alloc))) return S4R_ERR_CUDA;
+    a.rel_Z = zmean;
+    a.rel_part = unit;
+    a.rel_nparts = 1;
+  } else if (fast_scan) {
     if (cuda_failed(launch_scan_sm100(a))) return S4R_ERR_CUDA;
   } else {
     if (cuda_failed(launch_scan_generic(a))) return S4R_ERR_CUDA;
@@ -261,6 +331,18 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
   return decode_impl(layer, nullptr, nullptr, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,
                      max_len, window, top_k, score, rope, out, out_dtype, sel_idx, sel_count, workspace,
                      workspace_bytes, dev_status, stream);
+}
+
+int s4r_decode_step_windowed(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
+                             const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,
+                             const void *value_basis, int64_t max_len, int32_t window, int32_t top_k,
+                             const s4r_score_t *score, const s4r_rope_t *rope, float *query_window, void *out,
+                             int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
+                             size_t workspace_bytes, int32_t *dev_status, void *stream) {
+  if (!query_window || !score) return S4R_ERR_INVALID_ARG;
+  return decode_impl(layer, nullptr, nullptr, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,
+                     max_len, window, top_k, score, rope, out, out_dtype, sel_idx, sel_count, workspace,
+                     workspace_bytes, dev_status, stream, query_window);
 }
 
 int s4r_append_decode_step(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,

@@ -56,7 +56,10 @@ struct ScanFastParams {
   int Hkv, sinks;
   float theta;
   uint64_t rope_turns[64];
-  const float *cq_part;
+  const float *cq_part;           // unfused: rows of projected queries, [b][row][r], cq_batch_stride floats per b
+  int64_t cq_batch_stride, z_batch_stride;
+  int Gq;                         // query heads per KV head (G is the number of scored rows of this launch)
+  int row_off[kMaxGroup];         // scored row g sees cache rows l < L + row_off[g] (0: all; windowed scoring: <= 0)
   const int32_t *coef_len;
   float *Z;
   float2 *part;
@@ -230,7 +233,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
   const int tpc = (tiles_total + p.cps - 1) / p.cps;
   const int t_begin = min(tiles_total, j * tpc), t_end = min(tiles_total, t_begin + tpc);
   const int n_tiles = t_end - t_begin;
-  if (n_tiles <= 0 && !p.fused) {  // uniform over the CTA: nothing to scan
+  if (n_tiles <= 0 && !p.fused && p.qimg == nullptr) {  // uniform over the CTA: nothing to scan, nothing to prepare
     if (tid < p.G) p.part[((size_t)b * p.cps + j) * kMaxGroup + tid] = make_float2(-INFINITY, 0.f);
     return;
   }
@@ -260,7 +263,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
     // row n = t*8 + g holds term t (0 hi, 1 mid, 2 lo, 3 zero) of c^Q[g], K-major, 128-byte swizzle.
     const int wt = tid - 32;
     const int n_el = kMaxGroup * p.r;
-    const float *cq_src = p.cq_part + (size_t)b * p.G * p.r;   // unfused: written by the projection kernel
+    const float *cq_src = p.cq_part + (size_t)b * p.cq_batch_stride;   // unfused: written by the projection kernel
     int n_src = 1;                                              // partial sums to add per value
     size_t src_stride = 0;
     if (p.fused) {
@@ -399,15 +402,15 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
       for (int kv = j; kv < p.Hkv; kv += p.cps) {
         uint8_t *img = p.qimg + ((size_t)b * p.Hkv + kv) * kQueryOperandBytes;
         // rows that carry no query stay zero: G..7 and 8+G..15, 16 pieces of 16 bytes each
-        for (int i = wt; i < 2 * (8 - p.G) * 16; i += kWorkers) {
-          const int row = (i >> 4) < 8 - p.G ? p.G + (i >> 4) : 8 + p.G + ((i >> 4) - (8 - p.G));
+        for (int i = wt; i < 2 * (8 - p.Gq) * 16; i += kWorkers) {
+          const int row = (i >> 4) < 8 - p.Gq ? p.Gq + (i >> 4) : 8 + p.Gq + ((i >> 4) - (8 - p.Gq));
           const int piece = i & 15;
           *reinterpret_cast<uint4 *>(img + (size_t)(piece >> 3) * 2048 + (row >> 3) * 1024 + (row & 7) * 128 + (piece & 7) * 16) =
               make_uint4(0, 0, 0, 0);
         }
-        for (int i = wt; i < p.G * p.dh; i += kWorkers) {
+        for (int i = wt; i < p.Gq * p.dh; i += kWorkers) {
           const int g = i >> 7, c = i & 127;  // d_h = 128 on this path
-          const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)kv * p.G + g) * p.dh;
+          const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)kv * p.Gq + g) * p.dh;
           float v = __bfloat162float(qp[c]);
           if (rope) {
             const float o = __bfloat162float(qp[c ^ 64]);
@@ -490,7 +493,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
       m[g] = -INFINITY;
       sm[g] = 0.f;
     }
-    float *zb = p.Z + (size_t)b * p.G * p.z_stride;
+    float *zb = p.Z + (size_t)b * p.z_batch_stride;
     for (int it = 0; it < n_tiles; ++it) {
       const int a = it & 1;
       const uint32_t aph = (uint32_t)(it >> 1) & 1u;
@@ -510,7 +513,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
             const float z = ((__uint_as_float(v[16 + g]) + __uint_as_float(v[8 + g])) + __uint_as_float(v[g])) *
                             p.inv_sqrt_r;
             zb[(size_t)g * p.z_stride + row] = z;
-            online_update(m[g], sm[g], z);
+            if (row < L + p.row_off[g]) online_update(m[g], sm[g], z);
           }
         }
       }
@@ -619,11 +622,25 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
     return cudaErrorInvalidValue;
   ScanFastParams p;
   p.cq_part = (const float *)(a.ws + a.plan.off_cq);
+  p.cq_batch_stride = (int64_t)ly.G * ly.rk;
   p.coef_len = a.coef_len;
   p.Z = (float *)(a.ws + a.plan.off_z);
+  p.z_batch_stride = (int64_t)ly.G * a.plan.z_stride;
   p.part = (float2 *)(a.ws + a.plan.off_part);
   p.r = ly.rk;
   p.G = ly.G;
+  p.Gq = ly.G;
+  for (int g = 0; g < kMaxGroup; ++g) p.row_off[g] = 0;
+  if (a.scan_rows) {  // windowed scoring: this launch scores a block of rows of the query-coefficient window
+    const ScanRows &sr = *a.scan_rows;
+    p.cq_part = sr.cq;
+    p.cq_batch_stride = sr.cq_batch_stride;
+    p.Z = sr.Z;
+    p.z_batch_stride = sr.z_batch_stride;
+    p.part = sr.part;
+    p.G = sr.n_rows;
+    for (int g = 0; g < kMaxGroup; ++g) p.row_off[g] = sr.row_off[g];
+  }
   p.cps = a.plan.n_parts;
   p.cap = ly.cap;
   p.max_len = a.plan.max_len;
@@ -650,6 +667,7 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
   p.hist = (unsigned *)(a.ws + a.plan.off_hist);
   p.qimg = a.query_operand && ly.dh == 128 ? (uint8_t *)(a.ws + a.plan.off_qop) : nullptr;
   if (a.query_operand && !p.qimg) return cudaErrorInvalidValue;
+  if (a.scan_rows && !a.scan_rows->first) p.qimg = nullptr;  // prepared once, by the first block of rows
   p.Hkv = ly.Hkv; p.sinks = ly.s; p.theta = a.theta;
   fill_rope_turns(p.rope_turns, ly.dh, a.theta);
   // per-call token: unique within the process (counter) and seeded per process, so that flags left in recycled

@@ -449,13 +449,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select(SelParams p) {
 cudaError_t launch_relevance(const StepArgs &a) {
   if (a.plan.max_len <= 0) return cudaSuccess;
   RelParams p;
-  p.Z = (const float *)(a.ws + a.plan.off_z);
-  p.part = (const float2 *)(a.ws + a.plan.off_part);
+  p.Z = a.rel_Z ? a.rel_Z : (const float *)(a.ws + a.plan.off_z);
+  p.part = a.rel_part ? a.rel_part : (const float2 *)(a.ws + a.plan.off_part);
   p.coef_len = a.coef_len;
   p.score = (float *)(a.ws + a.plan.off_score);
   p.hist = (unsigned *)(a.ws + a.plan.off_hist);
   p.G = a.ly.G;
-  p.n_parts = a.plan.n_parts;
+  p.n_parts = a.rel_part ? a.rel_nparts : a.plan.n_parts;
   p.window = a.window;
   p.kappa = a.kappa;
   p.pool_mode = a.pool_mode;

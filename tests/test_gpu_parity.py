@@ -364,6 +364,34 @@ def test_decode_step_replayed_from_a_cuda_graph():
                 assert torch.equal(out, ref[0]) and torch.equal(sel, ref[1])
 
 
+@pytest.mark.parametrize("rows", [1, 50, 300])
+def test_captured_step_on_a_cache_shorter_than_the_grid(rows):
+    """With fewer 128-row tiles than scan CTAs some CTAs have nothing to scan; on the path with the separate
+    projection kernel (taken under capture) they must still prepare their share of the query operand."""
+    s4r = _s4r()
+    cfg = _cfg(1, context=2000 + 4, batch=2)
+    p = Problem(cfg, device="cuda").upload()
+    p.d_len.fill_(rows)
+    ly = p.layer_desc()
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+    ws.fill_(0x7f)                                # whatever a skipped CTA leaves behind is far from a valid operand
+    out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(cfg.batch, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(cfg.batch, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                            cfg.window, cfg.top_k, out, sel, cnt, ws, rope_theta=cfg.rope_theta, dev_status=status)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    err = check_step(p, out, sel, cnt, L=rows)
+    assert err <= 1e-4, f"output error {err:.3e} on a {rows}-row cache"
+
+
 @pytest.mark.parametrize("theta", [None, 0.0])
 def test_many_back_to_back_steps_stay_in_step(theta):
     """The kernels hand work between warp roles through phase-parity barriers; a role that fell two phases behind

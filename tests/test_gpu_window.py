@@ -1,0 +1,144 @@
+"""Windowed relevance estimation (Eq. 7, 9, 10): a FIFO of the W_q most recent projected queries scores the cache,
+each row under its own causal limit, and the probabilities are averaged.  The oracle keeps its own window; the
+library's window is seeded from the oracle's rows and afterwards maintained by the library itself."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import s4r_oracle as O
+from tests.helpers import Problem, to_np, from_np, TOL, BAND
+
+pytestmark = pytest.mark.gpu
+
+
+def _s4r():
+    import paper_2608_00528_b200 as s4r
+    return s4r
+
+
+def _queries(cfg, p, b, n):
+    """n successive queries of sequence b (oldest first), as stored (bf16) tensors."""
+    return [W.make_query(cfg, p.K[b], p.layer, b, step=i) for i in range(n)]
+
+
+def _run_case(cfg, Wq, steps=2, theta=None, cache_rows=None):
+    s4r = _s4r()
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    B, G, r, s = cfg.batch, cfg.group, cfg.rank_k, cfg.sink_count
+    th = cfg.rope_theta if theta is None else theta
+    L = p.L if cache_rows is None else cache_rows        # a shorter cache: only the first rows count
+    p.d_len.fill_(L)
+    n_q = Wq + steps - 1
+    qs = [_queries(cfg, p, b, n_q) for b in range(B)]
+    cq = [[O.project_query(to_np(q), p.BK[b], cfg.n_kv_heads) for q in qs[b]] for b in range(B)]     # [G, r] each
+    # library window: rows 1..W_q-1 hold the W_q - 1 queries before the first scored one; row 0 is dropped
+    win = torch.full((B, Wq, G, r), 7.0, dtype=torch.float32, device="cuda")
+    for b in range(B):
+        for i in range(Wq - 1):
+            win[b, i + 1] = torch.from_numpy(cq[b][i]).float()
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=Wq)
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(B, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(B, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    worst = 0.0
+    for t in range(steps):
+        cur = Wq - 1 + t
+        d_q = torch.stack([qs[b][cur].to("cuda") for b in range(B)])
+        before = win.clone()
+        s4r.decode_step_windowed(ly, d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                 cfg.window, cfg.top_k, win, out, sel, cnt, ws, score_window=Wq, rope_theta=th,
+                                 dev_status=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        assert torch.equal(win[:, :-1], before[:, 1:])                       # Eq. 7: shifted by one row
+        for b in range(B):
+            window_rows = np.stack(cq[b][cur - Wq + 1:cur + 1], axis=1)      # [G, W_q, r], oldest first
+            got_last = win[b, -1].double().cpu().numpy()
+            assert np.abs(got_last - cq[b][cur]).max() <= 2e-5 * np.abs(cq[b][cur]).max()
+            res = O.decode_step(to_np(qs[b][cur]), to_np(p.K[b][:s]), to_np(p.V[b][:s]), p.CK[b][:L], p.CV[b][:L], p.BK[b],
+                                p.BV[b], cfg.window, cfg.top_k, kappa=cfg.pool_kernel, pool_mode=cfg.pool_mode,
+                                group_mode=cfg.group_mode, theta=th, CQ_window=window_rows)
+            n = int(cnt[b].item())
+            got = sel[b, :n].cpu().numpy().astype(np.int64)
+            assert n == res["W_eff"] + res["k_eff"] and np.all(sel[b, n:].cpu().numpy() == -1)
+            ok, msg = O.selection_agrees(res["score"], res["idx"], got, res["W_eff"], res["k_eff"], BAND)
+            assert ok, f"W_q={Wq} step {t} seq {b}: {msg}"
+            if np.array_equal(np.sort(got), np.sort(np.asarray(res["idx"], dtype=np.int64))):
+                ref = res["out"]
+            else:
+                ref = O.sparse_attention(to_np(qs[b][cur]), to_np(p.K[b][:s]), to_np(p.V[b][:s]), p.CK[b][:L], p.CV[b][:L],
+                                         p.BK[b], p.BV[b], np.sort(got), th)
+            err = O.output_error(to_np(out[b]), ref)
+            assert err <= TOL[cfg.dtype], f"W_q={Wq} step {t} seq {b}: output error {err:.3e}"
+            worst = max(worst, err)
+    return worst
+
+
+@pytest.mark.parametrize("Wq", [2, 4, 8])
+def test_windowed_scoring_llama_shape(Wq):
+    cfg = W.scaled_config(W.get_config(1), context=6000 + 4, batch=2)
+    err = _run_case(cfg, Wq)
+    print(f"W_q={Wq} (rows {Wq * cfg.group}): max rel err {err:.3e}")
+
+
+def test_windowed_scoring_qwen_shape_group7():
+    cfg = W.scaled_config(W.get_config(3), context=5000 + 4, batch=1)
+    err = _run_case(cfg, 4)                                                   # 28 window rows, four scan blocks
+    print(f"qwen W_q=4: max rel err {err:.3e}")
+
+
+def test_window_of_one_equals_the_plain_step():
+    s4r = _s4r()
+    cfg = W.scaled_config(W.get_config(1), context=4000 + 4, batch=2)
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    B = cfg.batch
+    mk = lambda: (torch.empty(B, cfg.n_q_heads, cfg.head_dim, device="cuda"),
+                  torch.empty(B, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda"),
+                  torch.empty(B, dtype=torch.int32, device="cuda"))
+    out1, sel1, cnt1 = mk()
+    out2, sel2, cnt2 = mk()
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=2)
+    s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap, cfg.window,
+                    cfg.top_k, out1, sel1, cnt1, ws, rope_theta=cfg.rope_theta)
+    win = torch.zeros(B, 1, cfg.group, cfg.rank_k, dtype=torch.float32, device="cuda")
+    s4r.decode_step_windowed(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                             cfg.window, cfg.top_k, win, out2, sel2, cnt2, ws, score_window=1,
+                             rope_theta=cfg.rope_theta)
+    torch.cuda.synchronize()
+    assert torch.equal(cnt1, cnt2)
+    same = sum(len(set(sel1[b].tolist()) & set(sel2[b].tolist())) for b in range(B))
+    assert same >= B * (cfg.window + cfg.top_k) - 2 * B
+    assert ((out1 - out2).abs().amax() / out1.abs().amax()).item() <= 1e-3
+
+
+def test_window_longer_than_the_cache():
+    """Window rows whose token index would be negative see nothing and add nothing (Eq. 9's mask)."""
+    cfg = W.scaled_config(W.get_config(1), context=2000 + 4, batch=1, top_k=8, window=2)
+    for rows in (3, 1, 50):
+        err = _run_case(cfg, 4, steps=1, cache_rows=rows)
+        print(f"L={rows}, W_q=4: max rel err {err:.3e}")
+        assert err <= 1e-4            # every row is selected: what is left is the attention's own rounding
+
+
+def test_windowed_entry_rejects_what_it_cannot_do():
+    s4r = _s4r()
+    cfg = W.scaled_config(W.get_config(1), context=1000 + 4, batch=1)
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    out = torch.empty(1, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(1, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(1, dtype=torch.int32, device="cuda")
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=8)
+    win = torch.zeros(1, 9, cfg.group, cfg.rank_k, dtype=torch.float32, device="cuda")     # 36 rows > 32
+    with pytest.raises(s4r.S4RError) as e:
+        s4r.decode_step_windowed(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                 cfg.window, cfg.top_k, win, out, sel, cnt, ws, score_window=9)
+    assert e.value.status == -2
+    with pytest.raises(s4r.S4RError) as e:                                                  # plain entry: W_q must be 1
+        s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap, cfg.window,
+                        cfg.top_k, out, sel, cnt, ws, score_window=2)
+    assert e.value.status == -2
