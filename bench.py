@@ -253,6 +253,82 @@ def run_all_layers(args, cfg, s4r, device):
     print(json.dumps(line), flush=True)
 
 
+def run_windowed(args, cfg, s4r, device):
+    """Windowed relevance estimation (Eq. 7, 9, 10) on the bench workload: every step scores the cache with the
+    W_q most recent projected queries.  The FIFO fills itself during the warm-up steps.  One JSON line."""
+    Wq = args.score_window
+    K_steps, Wm = args.steps, max(args.warmup, 3, Wq + 2)
+    B = cfg.batch
+    capacity = cfg.cache_len + 8
+    c = build_cache(cfg, s4r, device, capacity, list(range(B)))
+    ly = c["ly"]
+    st = W.storage_dtype(cfg)
+    ws = s4r.alloc_workspace(ly, capacity, cfg.window, cfg.top_k, device, score_window=max(Wq, 2))
+    n_sel = cfg.window + cfg.top_k
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=device)
+    sel = torch.empty(B, n_sel, dtype=torch.int32, device=device)
+    cnt = torch.empty(B, dtype=torch.int32, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    win = torch.zeros(B, Wq, cfg.group, cfg.rank_k, dtype=torch.float32, device=device)
+    pool = 4
+    qs = torch.stack([c["q"] * (1.0 + 0.01 * i) for i in range(pool)]).to(st)
+    kw = dict(pool_kernel=cfg.pool_kernel, pool_mode={"max": s4r.POOL_MAX, "avg": s4r.POOL_AVG}[cfg.pool_mode],
+              group_mode={"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode], rope_theta=cfg.rope_theta,
+              dev_status=status, score_window=Wq)
+    launches = [0]
+
+    def step(i):
+        s4r.decode_step_windowed(ly, qs[i % pool], c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"],
+                                 capacity, cfg.window, cfg.top_k, win, out, sel, cnt, ws, **kw)
+        launches[0] += s4r.last_launch_count()
+
+    for i in range(Wm):
+        step(i)
+    torch.cuda.synchronize()
+    launches[0] = 0
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K_steps):
+        step(Wm + i)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_step = e0.elapsed_time(e1) / K_steps
+    gpu_launches = launches[0]
+    s4r.stage_timing(True)
+    stage_sum = {}
+    for i in range(20):
+        step(i)
+        for k_, v_ in s4r.stage_times().items():
+            stage_sum[k_] = stage_sum.get(k_, 0.0) + v_ / 20
+    s4r.stage_timing(False)
+    esz = cfg.elem_bytes
+    scan_bytes = B * cfg.cache_len * cfg.rank_k * esz
+    rows = Wq * cfg.group
+    # per pass over C^K: 2 flop per (window row, token, rank element) and per bf16 term of the split c^Q
+    scan_ms = stage_sum.get("latent_scoring", float("nan"))
+    peak, peak_kind = _peaks()
+    line = {
+        "metric": METRIC, "value": K_steps / (ms_step * K_steps * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K_steps,
+        "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": f"{cfg.name}_wq{Wq}", "batch": B, "context": cfg.context, "rank": cfg.rank_k,
+                   "window": cfg.window, "top_k": cfg.top_k, "score_window": Wq, "scored_rows": rows,
+                   "step": "s4r_decode_step_windowed (no cache update)",
+                   "l2": "inputs larger than L2 (key coefficients %.0f MB per pass)" % (scan_bytes / 1e6)},
+        "roofline": {"bound": "hbm", "kernel": "windowed latent scoring (all passes over C^K)",
+                     "achieved": scan_bytes / (scan_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": scan_bytes / (scan_ms * 1e-3) / 1e9 / peak, "peak_kind": peak_kind, "traffic": None,
+                     "bytes_per_launch": scan_bytes, "ms_per_launch": scan_ms,
+                     "note": "algorithmic bytes = one read of C^K; the stage reads it once per pass"},
+        "stage_ms": stage_sum, "gpu_launches": gpu_launches, "clocks": clocks, "dev_status": int(status.item()),
+        "cpu_baseline": None, "e2e": None,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def cpu_baseline(cfg, repeats=3):
     """The fp64 oracle, as it stands, on one sequence of the workload, timed on this host's cores."""
     import numpy as np
@@ -315,6 +391,8 @@ def main():
                     help="budget as a ratio of the cache (Eq. 14: top_k = floor(rho L) - window) instead of the "
                          "configuration's top_k; the paper's setting is 0.2")
     ap.add_argument("--layers", type=int, default=None, help="layers to run for a multi-layer configuration (default: all)")
+    ap.add_argument("--score-window", type=int, default=1,
+                    help="W_q > 1: time s4r_decode_step_windowed (Eq. 7, 9, 10) on the same workload instead")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = W.get_config(args.config)
@@ -346,6 +424,10 @@ def main():
 
     if cfg.n_layers > 1 and world == 1:
         return run_all_layers(args, cfg, s4r, device)
+    if args.score_window > 1:
+        if world > 1:
+            raise SystemExit("--score-window is a single-GPU measurement")
+        return run_windowed(args, cfg, s4r, device)
     K_steps, Wm = args.steps, max(args.warmup, 3)
     n_append = 2 * (K_steps + Wm) + 8
     capacity = cfg.cache_len + n_append
