@@ -115,8 +115,8 @@ typedef struct {
  * must be 256-byte aligned; its contents are undefined between calls. */
 size_t s4r_workspace_bytes(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k);
 
-/* The same for s4r_decode_step_windowed with W_q = score_window (W_q * G <= S4R_MAX_SCORE_ROWS, else 0). */
-#define S4R_MAX_SCORE_ROWS 32
+/* The same for s4r_decode_step_windowed with W_q = score_window (1 <= W_q <= S4R_MAX_SCORE_WINDOW, else 0). */
+#define S4R_MAX_SCORE_WINDOW 128
 size_t s4r_workspace_bytes_windowed(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k,
                                     int32_t score_window);
 
@@ -180,8 +180,11 @@ int s4r_decode_step(const s4r_layer_t *layer, const void *q, const void *sink_k,
  * query_window  [B, W_q, G, rank_k] fp32, caller-owned per-layer state, oldest row first; updated in place.  Before
  *               the first step the caller fills rows 1..W_q-1 with the coefficients of the W_q - 1 preceding
  *               queries (Eq. 4: C^Q = Q~ B^K; zeros if there are none) - row 0 is dropped by that step.
- * Built for bf16 caches with rank_k a multiple of 64 on sm_100 (S4R_ERR_UNSUPPORTED otherwise, and for
- * W_q * G > S4R_MAX_SCORE_ROWS).  The cache is scanned once per block of eight window rows.
+ * Built for bf16 caches with rank_k a multiple of 64 (at most 320) on sm_100; S4R_ERR_UNSUPPORTED otherwise and
+ * for W_q > S4R_MAX_SCORE_WINDOW.  Whole query groups with at most 128 window rows together are scored by one
+ * pair of passes over C^K (row normalisers, then the window mean): one pair for G * W_q <= 128, ceil(G /
+ * floor(128 / W_q)) pairs otherwise.  The window rows enter the tensor-core product as two bf16 terms (16
+ * mantissa bits), so a logit carries a relative error of about 2^-17.
  * workspace_bytes >= s4r_workspace_bytes_windowed(...).  All other arguments as in s4r_decode_step. */
 int s4r_decode_step_windowed(const s4r_layer_t *layer, const void *q, const void *sink_k, const void *sink_v,
                              const void *coef_k, const void *coef_v, const int32_t *coef_len, const void *key_basis,

@@ -63,17 +63,16 @@ static bool plan_decode(const Layer &ly, int64_t max_len, int window, int top_k,
 
 // Extra scratch of windowed scoring, laid out after the standard plan
 struct WindowPlan {
-  int rows, blocks, rows_alloc;
-  size_t off_z, off_part, off_zmean, off_unit, total;
+  int gpl, blocks;  // query groups per launch pair, launch pairs
+  size_t off_wimg, off_wpart, off_zmean, off_unit, total;
 };
 static bool plan_window(const Layer &ly, const DecodePlan &dp, int score_window, WindowPlan *w) {
-  if (score_window < 1 || (int64_t)score_window * ly.G > kMaxScoreRows) return false;
-  w->rows = score_window * ly.G;
-  w->blocks = (w->rows + kMaxGroup - 1) / kMaxGroup;
-  w->rows_alloc = w->blocks * kMaxGroup;
+  w->gpl = wscan_groups_per_launch(ly, score_window);
+  if (w->gpl < 1) return false;
+  w->blocks = (ly.G + w->gpl - 1) / w->gpl;
   size_t off = align_up(dp.total, 256);
-  w->off_z = off;      off = align_up(off + sizeof(float) * ly.B * (size_t)w->rows_alloc * dp.z_stride, 256);
-  w->off_part = off;   off = align_up(off + sizeof(float2) * (size_t)w->blocks * ly.B * dp.parts_cap * kMaxGroup, 256);
+  w->off_wimg = off;   off = align_up(off + (size_t)w->blocks * ly.B * wscan_image_bytes(ly), 256);
+  w->off_wpart = off;  off = align_up(off + sizeof(float2) * ly.B * (size_t)dp.parts_cap * 256, 256);
   w->off_zmean = off;  off = align_up(off + sizeof(float) * ly.B * (size_t)ly.G * dp.z_stride, 256);
   w->off_unit = off;   off = align_up(off + sizeof(float2) * ly.B * kMaxGroup, 256);
   w->total = off;
@@ -222,9 +221,8 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (!plan_decode(ly, max_len, window, top_k, &a.plan)) return S4R_ERR_INVALID_ARG;
   WindowPlan wp = {};
   if (query_window) {
-    if ((int64_t)sc.score_window * ly.G > kMaxScoreRows || k_t) return S4R_ERR_UNSUPPORTED;
+    if (k_t || !wscan_supported(ly, sc.score_window)) return S4R_ERR_UNSUPPORTED;  // bf16 caches, rank % 64 == 0, W_q <= 128
     if (!plan_window(ly, a.plan, sc.score_window, &wp)) return S4R_ERR_INVALID_ARG;
-    if (!scan_fast_supported(ly)) return S4R_ERR_UNSUPPORTED;  // bf16 caches with a rank that is a multiple of 64
   }
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
       workspace_bytes < (query_window ? wp.total : a.plan.total))
@@ -264,35 +262,22 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (!a.fuse_projection && cuda_failed(launch_qproj(a))) return S4R_ERR_CUDA;
   stage_mark(1, a.stream);
   if (query_window) {
-    // Eq. 7: shift the window and append the current query's coefficients; Eq. 8-9 for every window row in blocks
-    // of up to eight rows (one pass over C^K per block); Eq. 10: average per query group
+    // Eq. 7: shift the window and append the current query's coefficients; Eq. 8-10 per set of whole query groups
+    // with at most 128 window rows (two passes over C^K each: row normalisers, then the window mean)
     const int Wq = sc.score_window;
-    if (cuda_failed(launch_window_shift(query_window, (const float *)(a.ws + a.plan.off_cq), ly.B, Wq, ly.G * ly.rk,
-                                        a.stream)))
+    uint8_t *wimg = (uint8_t *)(a.ws + wp.off_wimg);
+    if (cuda_failed(launch_window_prepare(query_window, (const float *)(a.ws + a.plan.off_cq), wimg, ly, Wq, wp.gpl,
+                                          wp.blocks, a.stream)))
       return S4R_ERR_CUDA;
-    float *zw = (float *)(a.ws + wp.off_z);
-    float2 *partw = (float2 *)(a.ws + wp.off_part);
-    for (int blk = 0; blk < wp.blocks; ++blk) {
-      ScanRows sr;
-      sr.cq = query_window + (size_t)blk * kMaxGroup * ly.rk;
-      sr.cq_batch_stride = (int64_t)wp.rows * ly.rk;
-      sr.Z = zw + (size_t)blk * kMaxGroup * a.plan.z_stride;
-      sr.z_batch_stride = (int64_t)wp.rows_alloc * a.plan.z_stride;
-      sr.part = partw + (size_t)blk * ly.B * a.plan.parts_cap * kMaxGroup;
-      sr.n_rows = wp.rows - blk * kMaxGroup < kMaxGroup ? wp.rows - blk * kMaxGroup : kMaxGroup;
-      for (int g = 0; g < kMaxGroup; ++g) {
-        const int i = (blk * kMaxGroup + g) / ly.G;  // window row (oldest first) of scored row g of this block
-        sr.row_off[g] = i + 1 - Wq;
-      }
-      sr.first = blk == 0;
-      a.scan_rows = &sr;
-      const bool failed = cuda_failed(launch_scan_sm100(a));
-      a.scan_rows = nullptr;
-      if (failed) return S4R_ERR_CUDA;
-    }
+    float2 *wpart = (float2 *)(a.ws + wp.off_wpart);
     float *zmean = (float *)(a.ws + wp.off_zmean);
     float2 *unit = (float2 *)(a.ws + wp.off_unit);
-    if (cuda_failed(launch_window_mean(a, zw, partw, zmean, unit, Wq, wp.rows_alloc))) return S4R_ERR_CUDA;
+    for (int blk = 0; blk < wp.blocks; ++blk) {
+      const int g0 = blk * wp.gpl, ng = ly.G - g0 < wp.gpl ? ly.G - g0 : wp.gpl;
+      if (cuda_failed(launch_wscan(a, wimg + (size_t)blk * ly.B * wscan_image_bytes(ly), Wq, g0, ng, wpart, zmean, unit,
+                                   blk == 0)))
+        return S4R_ERR_CUDA;
+    }
     a.rel_Z = zmean;
     a.rel_part = unit;
     a.rel_nparts = 1;

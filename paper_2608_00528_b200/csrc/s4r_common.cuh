@@ -17,7 +17,6 @@ constexpr int kSelThreads = 1024;  // threads per CTA of the selection kernel (o
 constexpr int kMaxCluster = 8;     // CTAs per sequence in the selection kernel (8 is the portable cluster size)
 constexpr int kProjCluster = 8;    // CTAs (slices of D') per sequence in the projection kernels
 constexpr int kMaxParts = 256;     // upper bound of softmax partials per sequence written by a scan kernel
-constexpr int kMaxScoreRows = 32;   // rows of the query-coefficient window (W_q * G) in windowed scoring
 constexpr int kProjMaxParts = 16;  // CTAs per sequence that share the per-step projections inside the scan kernel
 
 // ---- programmatic dependent launch --------------------------------------------------------------------------

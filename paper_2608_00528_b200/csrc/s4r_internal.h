@@ -10,18 +10,6 @@ struct Layer {
   int64_t cap;
 };
 
-// A block of up to kMaxGroup rows of the query-coefficient window scored by one launch of the scan kernel
-struct ScanRows {
-  const float *cq;           // [b][row][r_k]
-  int64_t cq_batch_stride;   // floats between sequences
-  float *Z;                  // [b][row][z_stride] of this block
-  int64_t z_batch_stride;
-  float2 *part;              // [b][parts][kMaxGroup] of this block
-  int n_rows;
-  int row_off[kMaxGroup];    // row g sees cache rows l < L + row_off[g]
-  bool first;
-};
-
 struct StepArgs {
   Layer ly;
   const void *q, *sink_k, *sink_v, *coef_k, *coef_v, *basis_k, *basis_v;
@@ -32,7 +20,6 @@ struct StepArgs {
   int32_t *coef_len_w = nullptr;
   bool fuse_projection = false;  // Eq. 5-6 run inside the scan kernel; no projection kernel is launched
   bool query_operand = false;    // the scan kernel also prepares the attention kernel's rotated-query operand
-  const ScanRows *scan_rows = nullptr;   // windowed scoring: overrides the scan kernel's rows, outputs and limits
   // windowed scoring: the relevance kernel reads the window-averaged probabilities (as logarithms) instead of Z
   const float *rel_Z = nullptr;
   const float2 *rel_part = nullptr;
@@ -77,9 +64,13 @@ cudaError_t launch_attend_absorb(const StepArgs &a);
 cudaError_t launch_merge_absorb(const StepArgs &a);
 
 // windowed relevance estimation (Eq. 7, 9, 10)
-cudaError_t launch_window_shift(float *window, const float *cq, int B, int Wq, int n, cudaStream_t st);
-cudaError_t launch_window_mean(const StepArgs &a, const float *Z, const float2 *part, float *zmean, float2 *unit,
-                               int Wq, int rows_alloc);
+cudaError_t launch_window_prepare(float *window, const float *cq, uint8_t *wimg, const Layer &ly, int Wq, int gpl,
+                                  int sets, cudaStream_t st);
+size_t wscan_image_bytes(const Layer &ly);
+int wscan_groups_per_launch(const Layer &ly, int score_window);
+bool wscan_supported(const Layer &ly, int score_window);
+cudaError_t launch_wscan(const StepArgs &a, const uint8_t *wimg, int score_window, int g0, int ng, float2 *wpart,
+                         float *zmean, float2 *unit, bool first);
 
 cudaError_t launch_attend_generic(const StepArgs &a);
 cudaError_t launch_merge(const StepArgs &a);

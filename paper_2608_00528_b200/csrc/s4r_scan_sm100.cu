@@ -24,6 +24,7 @@
 
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
+#include "s4r_query_operand.cuh"
 
 namespace s4r {
 
@@ -51,15 +52,9 @@ struct ScanFastParams {
   unsigned long long *proj_flag;  // [B][cps + 1]: one per CTA of the sequence, then "token rows stored"
   unsigned long long token;
   unsigned *hist;                 // [B][2048], cleared here for the relevance kernel
-  // rotated-query operand of the attention kernel (nullptr: not wanted)
-  uint8_t *qimg;                  // [B][Hkv][kQueryOperandBytes]
-  int Hkv, sinks;
-  float theta;
-  uint64_t rope_turns[64];
+  QueryOperandArgs qo;            // rotated-query operand of the attention kernel (qo.qimg == nullptr: not wanted)
   const float *cq_part;           // unfused: rows of projected queries, [b][row][r], cq_batch_stride floats per b
   int64_t cq_batch_stride, z_batch_stride;
-  int Gq;                         // query heads per KV head (G is the number of scored rows of this launch)
-  int row_off[kMaxGroup];         // scored row g sees cache rows l < L + row_off[g] (0: all; windowed scoring: <= 0)
   const int32_t *coef_len;
   float *Z;
   float2 *part;
@@ -233,7 +228,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
   const int tpc = (tiles_total + p.cps - 1) / p.cps;
   const int t_begin = min(tiles_total, j * tpc), t_end = min(tiles_total, t_begin + tpc);
   const int n_tiles = t_end - t_begin;
-  if (n_tiles <= 0 && !p.fused && p.qimg == nullptr) {  // uniform over the CTA: nothing to scan, nothing to prepare
+  if (n_tiles <= 0 && !p.fused && p.qo.qimg == nullptr) {  // uniform over the CTA: nothing to scan, nothing to prepare
     if (tid < p.G) p.part[((size_t)b * p.cps + j) * kMaxGroup + tid] = make_float2(-INFINITY, 0.f);
     return;
   }
@@ -393,39 +388,8 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
     fence_proxy_async_smem();
     asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");  // B operand complete (producer not involved)
     if (wt == 0) mbar_arrive(proj_bar);
-    // ---- Off the critical path: the attention kernel's logit product wants q' = RoPE(q) / sqrt(d_h) of every KV
-    //      head as a ready-made tensor-core operand (hi + lo bf16 rows, swizzled).  CTA j of the sequence prepares
-    //      heads j, j + cps, ...; the first tiles are already in flight.
-    if (p.qimg != nullptr) {
-      const bool rope = p.theta > 0.f;
-      const float scale = rsqrtf((float)p.dh);
-      for (int kv = j; kv < p.Hkv; kv += p.cps) {
-        uint8_t *img = p.qimg + ((size_t)b * p.Hkv + kv) * kQueryOperandBytes;
-        // rows that carry no query stay zero: G..7 and 8+G..15, 16 pieces of 16 bytes each
-        for (int i = wt; i < 2 * (8 - p.Gq) * 16; i += kWorkers) {
-          const int row = (i >> 4) < 8 - p.Gq ? p.Gq + (i >> 4) : 8 + p.Gq + ((i >> 4) - (8 - p.Gq));
-          const int piece = i & 15;
-          *reinterpret_cast<uint4 *>(img + (size_t)(piece >> 3) * 2048 + (row >> 3) * 1024 + (row & 7) * 128 + (piece & 7) * 16) =
-              make_uint4(0, 0, 0, 0);
-        }
-        for (int i = wt; i < p.Gq * p.dh; i += kWorkers) {
-          const int g = i >> 7, c = i & 127;  // d_h = 128 on this path
-          const __nv_bfloat16 *qp = p.q + ((size_t)b * p.Hq + (size_t)kv * p.Gq + g) * p.dh;
-          float v = __bfloat162float(qp[c]);
-          if (rope) {
-            const float o = __bfloat162float(qp[c ^ 64]);
-            float sn, cs;
-            rope_sincos(p.sinks + L - 1, p.rope_turns[c & 63], sn, cs);
-            v = c < 64 ? v * cs - o * sn : v * cs + o * sn;
-          }
-          v *= scale;
-          const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-          const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-          *reinterpret_cast<__nv_bfloat16 *>(img + query_operand_offset(g, c)) = hi;
-          *reinterpret_cast<__nv_bfloat16 *>(img + query_operand_offset(8 + g, c)) = lo;
-        }
-      }
-    }
+    // ---- Off the critical path: the attention kernel's query operand; the first tiles are already in flight
+    if (p.qo.qimg != nullptr) build_query_operand(p.qo, b, j, p.cps, L, wt, kWorkers);
   }
 
   if (warp == 0) {
@@ -513,7 +477,7 @@ __global__ void __launch_bounds__(kScanThreads, 1) k_scan_sm100(const __grid_con
             const float z = ((__uint_as_float(v[16 + g]) + __uint_as_float(v[8 + g])) + __uint_as_float(v[g])) *
                             p.inv_sqrt_r;
             zb[(size_t)g * p.z_stride + row] = z;
-            if (row < L + p.row_off[g]) online_update(m[g], sm[g], z);
+            online_update(m[g], sm[g], z);
           }
         }
       }
@@ -629,18 +593,6 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
   p.part = (float2 *)(a.ws + a.plan.off_part);
   p.r = ly.rk;
   p.G = ly.G;
-  p.Gq = ly.G;
-  for (int g = 0; g < kMaxGroup; ++g) p.row_off[g] = 0;
-  if (a.scan_rows) {  // windowed scoring: this launch scores a block of rows of the query-coefficient window
-    const ScanRows &sr = *a.scan_rows;
-    p.cq_part = sr.cq;
-    p.cq_batch_stride = sr.cq_batch_stride;
-    p.Z = sr.Z;
-    p.z_batch_stride = sr.z_batch_stride;
-    p.part = sr.part;
-    p.G = sr.n_rows;
-    for (int g = 0; g < kMaxGroup; ++g) p.row_off[g] = sr.row_off[g];
-  }
   p.cps = a.plan.n_parts;
   p.cap = ly.cap;
   p.max_len = a.plan.max_len;
@@ -665,11 +617,10 @@ cudaError_t launch_scan_sm100(const StepArgs &a) {
   p.proj_part = (float *)(a.ws + a.plan.off_proj);
   p.proj_flag = (unsigned long long *)(a.ws + a.plan.off_flag);
   p.hist = (unsigned *)(a.ws + a.plan.off_hist);
-  p.qimg = a.query_operand && ly.dh == 128 ? (uint8_t *)(a.ws + a.plan.off_qop) : nullptr;
-  if (a.query_operand && !p.qimg) return cudaErrorInvalidValue;
-  if (a.scan_rows && !a.scan_rows->first) p.qimg = nullptr;  // prepared once, by the first block of rows
-  p.Hkv = ly.Hkv; p.sinks = ly.s; p.theta = a.theta;
-  fill_rope_turns(p.rope_turns, ly.dh, a.theta);
+  p.qo.qimg = a.query_operand && ly.dh == 128 ? (uint8_t *)(a.ws + a.plan.off_qop) : nullptr;
+  if (a.query_operand && !p.qo.qimg) return cudaErrorInvalidValue;
+  p.qo.q = p.q; p.qo.Hq = ly.Hq; p.qo.Hkv = ly.Hkv; p.qo.Gq = ly.G; p.qo.dh = ly.dh; p.qo.sinks = ly.s; p.qo.theta = a.theta;
+  fill_rope_turns(p.qo.rope_turns, ly.dh, a.theta);
   // per-call token: unique within the process (counter) and seeded per process, so that flags left in recycled
   // device memory by an earlier call or an earlier process never match
   static std::atomic<unsigned long long> token_source{

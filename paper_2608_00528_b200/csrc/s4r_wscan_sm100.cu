@@ -1,0 +1,472 @@
+// Windowed latent scoring (Eq. 8-10 with a query window W_q > 1) for bf16 coefficient caches on sm_100a.
+//
+// The W_q most recent projected queries of up to 128 / W_q query groups form the R <= 128 scored rows of one
+// launch pair; the product with a 128-token tile of C^K is a dense [128 x r] x [r x 128] contraction on the
+// tensor cores (tcgen05.mma, fp32 accumulators in tensor memory).  The projected queries enter as two bf16
+// terms per value (hi + mid: 16 mantissa bits, the logits keep a relative accuracy of 2^-17), both accumulated
+// into the same accumulator.  The softmax of Eq. 9 needs every row's normaliser before the window mean of
+// Eq. 10 can be formed, so the cache is streamed twice:
+//
+//   pass 0 (statistics)  D[window row][token]: a thread owns one window row and keeps its running
+//                        (max, sum exp) over the CTA's tiles under the row's causal limit; per-CTA partials go to
+//                        the workspace.  No logit is stored.
+//   pass 1 (mean)        D[token][window row]: a thread owns one token, turns its R logits into probabilities
+//                        with the merged normalisers, averages them per query group and stores the logarithm of
+//                        the mean, which the relevance kernel treats as a logit row with normaliser 1.
+//
+// The two-term operand image of the window is prepared once per step by the kernel that shifts the window
+// (k_window_prepare) and bulk-copied into shared memory by every CTA.  Both passes share the pipeline: warp 0 =
+// TMA producer over a ring of 16 KB pieces (one 64-column block of a 128-token tile), warps 1 and 10 = MMA
+// issuers (even and odd tiles, one accumulator each: a single thread cannot issue the 24 instructions of a tile
+// fast enough to keep up with the stream), warps 2-9 = epilogue, two per tensor-memory lane quadrant, each reading half of the accumulator columns (the
+// read-back of one warp overlaps the arithmetic of the other); grid (CTAs per sequence, B).  Two passes read C^K twice (2 r e bytes per token) instead
+// of writing and re-reading R fp32 logits per token (8 R bytes), which is less traffic from R = 48 rows on at
+// r = 192.
+#include "s4r_internal.h"
+#include "s4r_sm100.cuh"
+#include "s4r_query_operand.cuh"
+
+namespace s4r {
+
+using namespace sm100;
+
+bool scan_fast_supported(const Layer &ly);
+void fill_rope_turns(uint64_t *dst, int head_dim, float theta);
+
+namespace {
+
+constexpr int kTileRows = 128;
+constexpr int kThreads = 352;
+constexpr int kEpiThreads = 256;
+constexpr int kPieceBytes = kTileRows * 128;  // one 64-column block of a tile
+constexpr int kRows = 128;                    // rows of the query image (R padded)
+constexpr int kMaxPieces = 12;
+
+struct WScanParams {
+  const uint8_t *wimg;  // [B][2 terms][r / 64][128 rows][128 B]: operand image of this launch's groups
+  int Wq, G, g0, ng;    // this launch scores groups g0 .. g0 + ng - 1: rows rho = (g - g0) * W_q + i
+  const int32_t *coef_len;
+  float2 *wpart;        // [B][cps][2][128]: (max, sum) of z log2(e) per window row, CTA and column half
+  float *zmean;         // [B][G][z_stride]: ln of the window-averaged probability
+  float2 *unit;         // [B][kMaxGroup]: (0, 1), the relevance kernel's normalisers for zmean
+  int r, cps, pieces;
+  int64_t cap, max_len, z_stride;
+  float scale2;         // log2(e) / sqrt(r)
+  int32_t *dev_status;
+  QueryOperandArgs qo;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Pass 0, one 32-column chunk of a tile in which every column is visible to every window row.
+__device__ __forceinline__ void stats_chunk_fast(const uint32_t (&v)[32], float scale2, float &m_row, float &s_row) {
+  float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+  for (int c = 0; c < 32; ++c) cm[c & 3] = fmaxf(cm[c & 3], __uint_as_float(v[c]));
+  const float zc = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3])) * scale2;
+  if (zc > m_row) {
+    s_row *= fast_exp2(m_row - zc);
+    m_row = zc;
+  }
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int c = 0; c < 32; ++c) acc[c & 3] += fast_exp2(fmaf(__uint_as_float(v[c]), scale2, -m_row));
+  s_row += (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+// Pass 0, a chunk of which only the first nvis columns are visible to this thread's window row.
+__device__ __forceinline__ void stats_chunk_masked(const uint32_t (&v)[32], float scale2, int nvis, float &m_row,
+                                                   float &s_row) {
+  if (nvis <= 0) return;
+  float cm = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < 32; ++c)
+    if (c < nvis) cm = fmaxf(cm, __uint_as_float(v[c]));
+  const float zc = cm * scale2;
+  if (zc > m_row) {
+    s_row *= fast_exp2(m_row - zc);
+    m_row = zc;
+  }
+  float acc = 0.f;
+#pragma unroll
+  for (int c = 0; c < 32; ++c)
+    if (c < nvis) acc += fast_exp2(fmaf(__uint_as_float(v[c]), scale2, -m_row));
+  s_row += acc;
+}
+
+// Pass 1, one 32-column chunk whose group boundaries are known at compile time and whose columns are all visible:
+// SEG columns per group when SEG < 32 (W_q = SEG divides 32), the whole chunk inside one group when SEG == 32
+// (32 divides W_q).
+template <int SEG>
+__device__ __forceinline__ void mean_chunk_fast(const uint32_t (&v)[32], const float *mcc, float scale2, int n_here,
+                                                float &sum, int &i, int Wq, float *&dst, int64_t z_stride) {
+  float pr[32];
+#pragma unroll
+  for (int c = 0; c < 32; ++c) pr[c] = fast_exp2(fmaf(__uint_as_float(v[c]), scale2, -mcc[c]));
+  if (SEG == 32) {
+    float t[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 32; ++c) t[c & 3] += pr[c];
+    sum += (t[0] + t[1]) + (t[2] + t[3]);
+    i += 32;
+    if (i == Wq) {
+      *dst = __logf(sum);  // ln 0 = -inf: the position then carries no probability
+      dst += z_stride;
+      sum = 0.f;
+      i = 0;
+    }
+  } else {
+#pragma unroll
+    for (int seg = 0; seg < 32 / SEG; ++seg) {
+      if (seg * SEG < n_here) {  // uniform
+        float t = 0.f;
+#pragma unroll
+        for (int c = 0; c < SEG; ++c) t += pr[seg * SEG + c];
+        *dst = __logf(t);
+        dst += z_stride;
+      }
+    }
+  }
+}
+// Pass 1, general chunk: any W_q, and the tiles in which the causal limits of the window rows differ.
+__device__ __forceinline__ void mean_chunk_general(const uint32_t (&v)[32], const float *mcc, float scale2, int n_here,
+                                                   int age, bool in_cache, float &sum, int &i, int Wq, float *&dst,
+                                                   int64_t z_stride) {
+#pragma unroll
+  for (int c = 0; c < 32; ++c) {
+    if (c < n_here) {
+      float pr = fast_exp2(fmaf(__uint_as_float(v[c]), scale2, -mcc[c]));
+      pr = i >= age ? pr : 0.f;  // a select: logits of rows past the cache may be anything
+      sum += pr;
+      if (++i == Wq) {
+        if (in_cache) *dst = __logf(sum);
+        dst += z_stride;
+        sum = 0.f;
+        i = 0;
+      }
+    }
+  }
+}
+
+template <int PASS, int SEG>
+__global__ void __launch_bounds__(kThreads, 1) k_wscan(const __grid_constant__ CUtensorMap tmap, WScanParams p) {
+  grid_dependency_sync();
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int kblocks = p.r >> 6;
+  uint8_t *img = smem;                                            // [2 terms][kblocks][128 rows][128 B]
+  uint8_t *ring = img + (size_t)2 * kblocks * kPieceBytes;       // [pieces][128 rows][128 B]
+  uint64_t *bars = reinterpret_cast<uint64_t *>(ring + (size_t)p.pieces * kPieceBytes);
+  uint64_t *full = bars, *empty = bars + kMaxPieces, *acc_full = bars + 2 * kMaxPieces, *acc_empty = acc_full + 2;
+  uint64_t *img_bar = acc_empty + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(img_bar + 1);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  float *mc = reinterpret_cast<float *>(tmem_slot + 2);          // [128] pass 1: max + log2(sum W_q) per window row
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.y, j = blockIdx.x;
+  int L = p.coef_len[b];
+  if (L < 0 || (int64_t)L > p.max_len) {
+    if (p.dev_status && tid == 0) atomicOr(p.dev_status, S4R_DEV_BOUNDS);
+    L = L < 0 ? 0 : (int)p.max_len;
+  }
+  const int R = p.ng * p.Wq;
+  const int tiles_total = (L + kTileRows - 1) / kTileRows;
+  const int tpc = (tiles_total + p.cps - 1) / p.cps;
+  const int t_begin = min(tiles_total, j * tpc), t_end = min(tiles_total, t_begin + tpc);
+  const int n_tiles = t_end - t_begin;
+  // pass 1: the two warps of a quadrant can split the window rows only if no query group straddles column 64
+  const bool split = PASS == 0 || (64 % p.Wq) == 0;
+  if (PASS == 1 && j == 0 && tid < p.ng) p.unit[(size_t)b * kMaxGroup + p.g0 + tid] = make_float2(0.f, 1.f);
+  if (n_tiles <= 0 && (PASS == 1 || p.qo.qimg == nullptr)) {  // uniform over the CTA: nothing to scan or prepare
+    if (PASS == 0 && tid < 2 * kRows) p.wpart[((size_t)b * p.cps + j) * 2 * kRows + tid] = make_float2(-INFINITY, 0.f);
+    return;
+  }
+
+  if (tid == 0) {
+    for (int s = 0; s < p.pieces; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&acc_full[a], 1);
+      mbar_init(&acc_empty[a], split ? 8 : 4);  // one arrival per participating epilogue warp
+    }
+    mbar_init(img_bar, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&tmap);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, 256);  // two accumulators of 128 columns
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  float m_row = -INFINITY, s_row = 0.f;  // pass 0, epilogue threads
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool img_issued = false;
+      if (n_tiles > 0) {
+        // the operand image first: 2 * kblocks pieces of 16 KB on one barrier
+        const uint8_t *src = p.wimg + (size_t)b * 2 * kblocks * kPieceBytes;
+        mbar_expect_tx(img_bar, (uint32_t)(2 * kblocks * kPieceBytes));
+        for (int q = 0; q < 2 * kblocks; ++q)
+          bulk_load(img + (size_t)q * kPieceBytes, src + (size_t)q * kPieceBytes, kPieceBytes, img_bar);
+        img_issued = true;
+      }
+      const uint64_t pol = policy_evict_first();
+      const int n_pieces = n_tiles * kblocks;
+      for (int q = 0, it = 0, kb = 0; q < n_pieces; ++q) {
+        const int s = q % p.pieces;
+        const uint32_t ph = (uint32_t)(q / p.pieces) & 1u;
+        if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag)) break;
+        mbar_expect_tx(&full[s], kPieceBytes);
+        const int y = (int)((int64_t)b * p.cap) + (t_begin + it) * kTileRows;
+        tma_load_2d_hint(ring + (size_t)s * kPieceBytes, &tmap, kb * 64, y, &full[s], pol);
+        issued = q + 1;
+        if (++kb == kblocks) {
+          kb = 0;
+          ++it;
+        }
+      }
+      if (*abort_flag) {  // drain: do not leave while bulk copies may still land in this CTA's shared memory
+        for (int q = max(0, issued - p.pieces); q < issued; ++q) {
+          const unsigned long long t0 = global_ns();
+          while (!mbar_try_wait(&full[q % p.pieces], (uint32_t)(q / p.pieces) & 1u))
+            if (global_ns() - t0 > kWaitLimitNs) break;
+        }
+        if (img_issued) {
+          const unsigned long long t0 = global_ns();
+          while (!mbar_try_wait(img_bar, 0))
+            if (global_ns() - t0 > kWaitLimitNs) break;
+        }
+      }
+    }
+  } else if (warp == 1 || warp == 10) {
+    // ---------------- MMA issuers: warp 1 takes the even tiles (accumulator 0), warp 10 the odd ones ----------------
+    const int a = warp == 1 ? 0 : 1;
+    if (lane == 0 && n_tiles > a) {
+      const int n_cols = PASS == 0 ? kTileRows : ((R + 15) & ~15);
+      const uint32_t idesc = umma_idesc_bf16(128, n_cols);
+      const uint64_t img_desc0 = umma_desc_sw128(smem_u32(img));
+      const uint32_t term_step = (uint32_t)(kblocks * kPieceBytes) >> 4;
+      bool ok = mbar_wait(img_bar, 0, abort_flag);
+      for (int it = a; it < n_tiles && ok; it += 2) {
+        const uint32_t aph = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(&acc_empty[a], aph ^ 1u, abort_flag)) break;
+        const uint32_t d_tmem = tmem_base + (uint32_t)a * 128u;
+        int q = it * kblocks;
+        for (int kb = 0; kb < kblocks; ++kb, ++q) {
+          const int s = q % p.pieces;
+          const uint32_t ph = (uint32_t)(q / p.pieces) & 1u;
+          if (!mbar_wait(&full[s], ph, abort_flag)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint64_t tile_desc = umma_desc_sw128(smem_u32(ring + (size_t)s * kPieceBytes));
+          const uint64_t cq_desc = img_desc0 + (uint64_t)((uint32_t)(kb * kPieceBytes) >> 4);
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {
+              const uint64_t td = tile_desc + (uint64_t)(k4 * 2);
+              const uint64_t cd = cq_desc + (uint64_t)(t * term_step + k4 * 2);
+              if (PASS == 0)
+                umma_bf16(d_tmem, cd, td, idesc, (kb | t | k4) != 0);  // rows = window rows, columns = tokens
+              else
+                umma_bf16(d_tmem, td, cd, idesc, (kb | t | k4) != 0);  // rows = tokens, columns = window rows
+            }
+          }
+          umma_commit(&empty[s]);  // the piece is free once these MMAs have read it
+        }
+        if (ok) umma_commit(&acc_full[a]);
+      }
+    }
+  } else {
+    // ---------------- epilogue: 8 warps, two per TMEM lane quadrant (column halves) ----------------
+    const int et = tid - 64;
+    const int quad = warp & 3, half = (warp - 2) >> 2;
+    const int lane_row = quad * 32 + lane;
+    const uint32_t lane_field = (uint32_t)(quad * 32) << 16;
+    const int first_limit = L - p.Wq;  // the oldest window row sees tokens l <= L - W_q
+    if (PASS == 0) {
+      if (p.qo.qimg != nullptr) build_query_operand(p.qo, b, j, p.cps, L, et, kEpiThreads);
+      // window row lane_row: tokens l <= lim are visible; padding rows compute on everything and are ignored
+      const int gl = lane_row / p.Wq;
+      const int lim = lane_row < R ? L - p.Wq + (lane_row - gl * p.Wq) : L - 1;
+      for (int it = 0; it < n_tiles; ++it) {
+        const int a = it & 1;
+        const uint32_t aph = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(&acc_full[a], aph, abort_flag)) break;
+        tc_fence_after();
+        const int tile_base = (t_begin + it) * kTileRows;
+        const uint32_t t_addr = tmem_base + (uint32_t)a * 128u + lane_field;
+        // this warp's half of the accumulator row at once, so that the tensor cores get the buffer back early
+        uint32_t v0[32], v1[32];
+        tmem_ld32(t_addr + (uint32_t)(half * 64), v0);
+        tmem_ld32(t_addr + (uint32_t)(half * 64 + 32), v1);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[a]);
+        if (tile_base + kTileRows - 1 <= first_limit) {
+          stats_chunk_fast(v0, p.scale2, m_row, s_row);
+          stats_chunk_fast(v1, p.scale2, m_row, s_row);
+        } else {
+          const int nvis = lim - (tile_base + half * 64) + 1;  // visible columns of this half of the tile
+          stats_chunk_masked(v0, p.scale2, nvis, m_row, s_row);
+          stats_chunk_masked(v1, p.scale2, nvis - 32, m_row, s_row);
+        }
+      }
+    } else {
+      {
+        // Eq. 9 normalisers: merge the CTAs' partials of window row et (empty partials are (-inf, 0))
+        const float2 *pp = p.wpart + (size_t)b * p.cps * 2 * kRows + (et & (kRows - 1));
+        float m = -INFINITY, s = 0.f;
+        for (int c = 0; c < 2 * p.cps; ++c) {
+          const float2 v = __ldcg(pp + (size_t)c * kRows);
+          if (v.y > 0.f) {
+            const float mn = fmaxf(m, v.x);
+            s = s * fast_exp2(m - mn) + v.y * fast_exp2(v.x - mn);
+            m = mn;
+          }
+        }
+        if (et < kRows) mc[et] = (s > 0.f && et < R) ? m + log2f(s * (float)p.Wq) : INFINITY;  // +inf: contributes nothing
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+      }
+      // columns (window rows) of this warp: [c0, c0 + 32 n_chunks)
+      const int c0 = split ? half * 64 : 0;
+      const int n_chunks = (split || half == 0) ? min(split ? 2 : 4, (R - c0 + 31) >> 5) : 0;
+      const bool takes_part = split || half == 0;
+      for (int it = 0; it < n_tiles && takes_part; ++it) {
+        const int a = it & 1;
+        const uint32_t aph = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(&acc_full[a], aph, abort_flag)) break;
+        tc_fence_after();
+        const int tile_base = (t_begin + it) * kTileRows;
+        const bool fast = SEG > 0 && tile_base + kTileRows - 1 <= first_limit;
+        const int row = tile_base + lane_row;  // token index
+        const int age = row - first_limit;     // window row i sees this token iff i >= age
+        float *dst = p.zmean + ((size_t)b * p.G + p.g0 + c0 / p.Wq) * p.z_stride + row;
+        const uint32_t t_addr = tmem_base + (uint32_t)a * 128u + lane_field + (uint32_t)c0;
+        uint32_t v0[32], v1[32], v2[32], v3[32];
+        if (n_chunks > 0) tmem_ld32(t_addr, v0);
+        if (n_chunks > 1) tmem_ld32(t_addr + 32u, v1);
+        if (n_chunks > 2) tmem_ld32(t_addr + 64u, v2);
+        if (n_chunks > 3) tmem_ld32(t_addr + 96u, v3);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[a]);
+        float sum = 0.f;
+        int i = 0;
+        const float *mcw = mc + c0;
+        const int Rw = R - c0;  // columns left from c0 on
+        if (fast) {
+          constexpr int S = SEG == 0 ? 32 : SEG;
+          if (n_chunks > 0) mean_chunk_fast<S>(v0, mcw, p.scale2, min(32, Rw), sum, i, p.Wq, dst, p.z_stride);
+          if (n_chunks > 1) mean_chunk_fast<S>(v1, mcw + 32, p.scale2, min(32, Rw - 32), sum, i, p.Wq, dst, p.z_stride);
+          if (n_chunks > 2) mean_chunk_fast<S>(v2, mcw + 64, p.scale2, min(32, Rw - 64), sum, i, p.Wq, dst, p.z_stride);
+          if (n_chunks > 3) mean_chunk_fast<S>(v3, mcw + 96, p.scale2, min(32, Rw - 96), sum, i, p.Wq, dst, p.z_stride);
+        } else {
+          const bool in_cache = row < L;
+          if (n_chunks > 0)
+            mean_chunk_general(v0, mcw, p.scale2, min(32, Rw), age, in_cache, sum, i, p.Wq, dst, p.z_stride);
+          if (n_chunks > 1)
+            mean_chunk_general(v1, mcw + 32, p.scale2, min(32, Rw - 32), age, in_cache, sum, i, p.Wq, dst, p.z_stride);
+          if (n_chunks > 2)
+            mean_chunk_general(v2, mcw + 64, p.scale2, min(32, Rw - 64), age, in_cache, sum, i, p.Wq, dst, p.z_stride);
+          if (n_chunks > 3)
+            mean_chunk_general(v3, mcw + 96, p.scale2, min(32, Rw - 96), age, in_cache, sum, i, p.Wq, dst, p.z_stride);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (PASS == 0 && warp >= 2 && warp < 10)  // an epilogue thread owns window row (warp % 4) * 32 + lane, columns of its half
+    p.wpart[(((size_t)b * p.cps + j) * 2 + ((warp - 2) >> 2)) * kRows + (warp & 3) * 32 + lane] = make_float2(m_row, s_row);
+  if (tid == 0 && *abort_flag && p.dev_status) atomicOr(p.dev_status, S4R_DEV_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+template <int PASS, int SEG>
+cudaError_t launch_pass(const CUtensorMap &tmap, const WScanParams &p, int B, size_t smem, cudaStream_t st) {
+  static size_t smem_set = 0;
+  if (smem > smem_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_wscan<PASS, SEG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    smem_set = smem;
+  }
+  cudaError_t le = launch_chained(k_wscan<PASS, SEG>, dim3(p.cps, B), dim3(kThreads), smem, st, 1, tmap, p);
+  if (le != cudaSuccess) return le;
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// Groups scored by one launch pair: whole query groups, at most 128 window rows
+int wscan_groups_per_launch(const Layer &ly, int score_window) {
+  if (score_window < 1 || score_window > kRows) return 0;
+  const int gpl = kRows / score_window;
+  return gpl < ly.G ? gpl : ly.G;
+}
+
+size_t wscan_image_bytes(const Layer &ly) { return (size_t)2 * (ly.rk / 64) * kPieceBytes; }
+
+bool wscan_supported(const Layer &ly, int score_window) {
+  if (!scan_fast_supported(ly) || wscan_groups_per_launch(ly, score_window) < 1) return false;
+  return wscan_image_bytes(ly) + 2048 + 1024 + 3 * (size_t)kPieceBytes <= 226 * 1024;
+}
+
+// Scores groups g0 .. g0 + ng - 1 of the window: statistics pass, then mean pass.  wimg: the operand images of
+// this launch's groups, [B][wscan_image_bytes]; wpart: [B][cps][2][128] float2.
+cudaError_t launch_wscan(const StepArgs &a, const uint8_t *wimg, int score_window, int g0, int ng, float2 *wpart,
+                         float *zmean, float2 *unit, bool first) {
+  const Layer &ly = a.ly;
+  CUtensorMap tmap;
+  if (!make_tmap_bf16_2d(&tmap, a.coef_k, (uint64_t)ly.B * (uint64_t)ly.cap, (uint64_t)ly.rk, kTileRows))
+    return cudaErrorInvalidValue;
+  WScanParams p;
+  p.wimg = wimg; p.Wq = score_window; p.G = ly.G; p.g0 = g0; p.ng = ng;
+  p.coef_len = a.coef_len; p.wpart = wpart; p.zmean = zmean; p.unit = unit;
+  p.r = ly.rk; p.cps = a.plan.n_parts; p.cap = ly.cap; p.max_len = a.plan.max_len; p.z_stride = a.plan.z_stride;
+  p.scale2 = (float)(1.4426950408889634 / sqrt((double)ly.rk));
+  p.dev_status = a.dev_status;
+  p.qo.qimg = first && a.query_operand && ly.dh == 128 ? (uint8_t *)(a.ws + a.plan.off_qop) : nullptr;
+  if (a.query_operand && ly.dh != 128) return cudaErrorInvalidValue;
+  p.qo.q = (const __nv_bfloat16 *)a.q; p.qo.Hq = ly.Hq; p.qo.Hkv = ly.Hkv; p.qo.Gq = ly.G; p.qo.dh = ly.dh;
+  p.qo.sinks = ly.s; p.qo.theta = a.theta;
+  fill_rope_turns(p.qo.rope_turns, ly.dh, a.theta);
+  const size_t fixed = wscan_image_bytes(ly) + 2048 /*barriers, constants*/ + 1024 /*alignment*/;
+  int pieces = (int)((226 * 1024 - fixed) / kPieceBytes);
+  if (pieces > kMaxPieces) pieces = kMaxPieces;
+  if (pieces < 3) return cudaErrorInvalidValue;
+  p.pieces = pieces;
+  const size_t smem = fixed + (size_t)pieces * kPieceBytes;
+  cudaError_t e = launch_pass<0, 0>(tmap, p, ly.B, smem, a.stream);
+  if (e != cudaSuccess) return e;
+  const int Wq = score_window;
+  if (Wq % 32 == 0) return launch_pass<1, 32>(tmap, p, ly.B, smem, a.stream);
+  switch (Wq) {
+    case 1: return launch_pass<1, 1>(tmap, p, ly.B, smem, a.stream);
+    case 2: return launch_pass<1, 2>(tmap, p, ly.B, smem, a.stream);
+    case 4: return launch_pass<1, 4>(tmap, p, ly.B, smem, a.stream);
+    case 8: return launch_pass<1, 8>(tmap, p, ly.B, smem, a.stream);
+    case 16: return launch_pass<1, 16>(tmap, p, ly.B, smem, a.stream);
+    default: return launch_pass<1, 0>(tmap, p, ly.B, smem, a.stream);
+  }
+}
+
+}  // namespace s4r

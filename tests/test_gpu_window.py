@@ -77,17 +77,21 @@ def _run_case(cfg, Wq, steps=2, theta=None, cache_rows=None):
     return worst
 
 
-@pytest.mark.parametrize("Wq", [2, 4, 8])
+@pytest.mark.parametrize("Wq", [2, 4, 5, 8, 32])
 def test_windowed_scoring_llama_shape(Wq):
+    """G = 4: 8 to 128 window rows, all scored by one pair of passes (W_q = 32 fills the 128-row operand; W_q = 5
+    leaves group boundaries inside the 32-column chunks the epilogue reads)."""
     cfg = W.scaled_config(W.get_config(1), context=6000 + 4, batch=2)
     err = _run_case(cfg, Wq)
     print(f"W_q={Wq} (rows {Wq * cfg.group}): max rel err {err:.3e}")
 
 
-def test_windowed_scoring_qwen_shape_group7():
+@pytest.mark.parametrize("Wq", [4, 32])
+def test_windowed_scoring_qwen_shape_group7(Wq):
+    """G = 7: 28 window rows in one pair of passes; at W_q = 32 the 224 rows take two pairs (groups 0-3, 4-6)."""
     cfg = W.scaled_config(W.get_config(3), context=5000 + 4, batch=1)
-    err = _run_case(cfg, 4)                                                   # 28 window rows, four scan blocks
-    print(f"qwen W_q=4: max rel err {err:.3e}")
+    err = _run_case(cfg, Wq, steps=1 if Wq > 8 else 2)
+    print(f"qwen W_q={Wq}: max rel err {err:.3e}")
 
 
 def test_window_of_one_equals_the_plain_step():
@@ -118,9 +122,9 @@ def test_window_of_one_equals_the_plain_step():
 def test_window_longer_than_the_cache():
     """Window rows whose token index would be negative see nothing and add nothing (Eq. 9's mask)."""
     cfg = W.scaled_config(W.get_config(1), context=2000 + 4, batch=1, top_k=8, window=2)
-    for rows in (3, 1, 50):
-        err = _run_case(cfg, 4, steps=1, cache_rows=rows)
-        print(f"L={rows}, W_q=4: max rel err {err:.3e}")
+    for rows, Wq in ((3, 4), (1, 4), (50, 4), (20, 32), (130, 32)):
+        err = _run_case(cfg, Wq, steps=1, cache_rows=rows)
+        print(f"L={rows}, W_q={Wq}: max rel err {err:.3e}")
         assert err <= 1e-4            # every row is selected: what is left is the attention's own rounding
 
 
@@ -133,10 +137,10 @@ def test_windowed_entry_rejects_what_it_cannot_do():
     sel = torch.empty(1, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
     cnt = torch.empty(1, dtype=torch.int32, device="cuda")
     ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=8)
-    win = torch.zeros(1, 9, cfg.group, cfg.rank_k, dtype=torch.float32, device="cuda")     # 36 rows > 32
+    win = torch.zeros(1, 129, cfg.group, cfg.rank_k, dtype=torch.float32, device="cuda")   # W_q > 128
     with pytest.raises(s4r.S4RError) as e:
         s4r.decode_step_windowed(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
-                                 cfg.window, cfg.top_k, win, out, sel, cnt, ws, score_window=9)
+                                 cfg.window, cfg.top_k, win, out, sel, cnt, ws, score_window=129)
     assert e.value.status == -2
     with pytest.raises(s4r.S4RError) as e:                                                  # plain entry: W_q must be 1
         s4r.decode_step(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap, cfg.window,
