@@ -193,6 +193,15 @@ int s4r_decode_step_windowed(const s4r_layer_t *layer, const void *q, const void
                              int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
                              size_t workspace_bytes, int32_t *dev_status, void *stream);
 
+/* Initial query-coefficient window (Eq. 4: C^Q = Q~ B^K for the last prompt queries).
+ * queries       [B, n_queries, H_q, d_h] (device, layer dtype), oldest first, pre-RoPE; 0 <= n_queries <= W_q
+ * query_window  [B, W_q, G, rank_k] fp32 (device): rows W_q - n_queries .. W_q - 1 receive the coefficients of the
+ *               queries, the rows before them zeros.  The first s4r_decode_step_windowed then drops row 0 and
+ *               appends the first generated token's query.
+ * Any geometry s4r_decode_step accepts.  Errors as s4r_append. */
+int s4r_window_init(const s4r_layer_t *layer, const void *queries, int32_t n_queries, const void *key_basis,
+                    float *query_window, int32_t score_window, void *stream);
+
 /* s4r_append followed by s4r_decode_step as one call (Sec. 3.2.1 then 3.2.2-3.2.3): the new token's key and
  * value rows are projected in the same pass over the bases that projects the query (Eq. 5), appended
  * (Eq. 6), and the step then runs on the grown cache.  The new rows may differ from those of s4r_append by one

@@ -21,7 +21,7 @@ VALUE_AUTO, VALUE_RECONSTRUCT = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_workspace_bytes_windowed", "s4r_compress", "s4r_append", "s4r_decode_step",
-           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed",
+           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed", "s4r_window_init",
            "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
            "s4r_stage_times", "s4r_strerror", "s4r_last_cuda_error", "s4r_version")
 STAGES = ("query_projection", "latent_scoring", "selection", "reconstruct_attend", "merge")
@@ -80,6 +80,8 @@ def load(build_if_missing: bool = True):
     lib.s4r_workspace_bytes.argtypes = [lp, i64, i32, i32]
     lib.s4r_workspace_bytes_windowed.restype = sz
     lib.s4r_workspace_bytes_windowed.argtypes = [lp, i64, i32, i32, i32]
+    lib.s4r_window_init.restype = ctypes.c_int
+    lib.s4r_window_init.argtypes = [lp, vp, i32, vp, vp, i32, vp]
     lib.s4r_decode_step_windowed.restype = ctypes.c_int
     lib.s4r_decode_step_windowed.argtypes = [lp] + [vp] * 8 + [i64, i32, i32, ctypes.POINTER(_Score), ctypes.POINTER(_Rope),
                                              vp, vp, i32, vp, vp, vp, sz, vp, vp]
@@ -274,6 +276,22 @@ def decode_step_windowed(layer: Layer, q, sink_k, sink_v, coef_k, coef_v, coef_l
                                          _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream))
     if rc != 0:
         raise S4RError(rc, "s4r_decode_step_windowed")
+
+
+def window_init(layer: Layer, queries, key_basis, query_window, *, score_window: int, stream=None):
+    """s4r_window_init: `queries` [B, n, H_q, d_h] (n <= W_q, oldest first; None or n = 0: an all-zero window) fill the
+    last n rows of `query_window` [B, W_q, G, rank_k] fp32."""
+    _need_cuda(key_basis, query_window)
+    n = 0 if queries is None else int(queries.shape[1])
+    if queries is not None and (not queries.is_cuda or not queries.is_contiguous()):
+        raise ValueError("queries must be a contiguous CUDA tensor [B, n, H_q, d_h]")
+    if query_window.dtype != torch.float32 or tuple(query_window.shape) != (
+            layer.batch, score_window, layer.n_q_heads // layer.n_kv_heads, layer.rank_k) or not query_window.is_contiguous():
+        raise ValueError("query_window must be a contiguous fp32 tensor [B, W_q, G, rank_k]")
+    rc = load().s4r_window_init(ctypes.byref(layer.c()), _ptr(queries), n, _ptr(key_basis), _ptr(query_window),
+                                int(score_window), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_window_init")
 
 
 def decode_step_host(layer: Layer, q_host, q_dev, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,

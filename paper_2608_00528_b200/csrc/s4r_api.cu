@@ -330,6 +330,32 @@ int s4r_decode_step_windowed(const s4r_layer_t *layer, const void *q, const void
                      workspace_bytes, dev_status, stream, query_window);
 }
 
+int s4r_window_init(const s4r_layer_t *layer, const void *queries, int32_t n_queries, const void *key_basis,
+                    float *query_window, int32_t score_window, void *stream) {
+  launch_counter() = 0;
+  Layer ly;
+  if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
+  if (int rc = layer_supported(ly)) return rc;
+  if (!key_basis || !query_window || score_window < 1 || n_queries < 0 || n_queries > score_window ||
+      (n_queries > 0 && !queries))
+    return S4R_ERR_INVALID_ARG;
+  if (!aligned16(key_basis) || (n_queries > 0 && !aligned16(queries))) return S4R_ERR_INVALID_ARG;
+  if (int rc = check_arch()) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t row = (int64_t)ly.G * ly.rk, q_row = (int64_t)ly.Hq * ly.dh;
+  const size_t esz = ly.dtype == S4R_BF16 ? 2 : 4;
+  if (n_queries < score_window &&
+      cuda_failed(cudaMemsetAsync(query_window, 0, sizeof(float) * (size_t)ly.B * score_window * row, st)))
+    return S4R_ERR_CUDA;
+  for (int i = 0; i < n_queries; ++i) {  // query i lands in window row W_q - n + i
+    const char *q_i = (const char *)queries + (size_t)i * q_row * esz;
+    float *dst = query_window + (int64_t)(score_window - n_queries + i) * row;
+    if (cuda_failed(launch_project_queries(ly, q_i, (int64_t)n_queries * q_row, key_basis, dst, (int64_t)score_window * row, st)))
+      return S4R_ERR_CUDA;
+  }
+  return S4R_OK;
+}
+
 int s4r_append_decode_step(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,
                            const void *sink_k, const void *sink_v, void *coef_k, void *coef_v, int32_t *coef_len,
                            const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,

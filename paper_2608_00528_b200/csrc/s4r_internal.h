@@ -40,6 +40,8 @@ int &launch_counter();
 
 // generic (any supported geometry, fp32 or bf16 storage, CUDA-core arithmetic in fp32)
 cudaError_t launch_qproj(const StepArgs &a);
+cudaError_t launch_project_queries(const Layer &ly, const void *q, int64_t q_seq_stride, const void *basis_k, float *dst,
+                                   int64_t dst_seq_stride, cudaStream_t st);
 cudaError_t launch_scan_generic(const StepArgs &a);
 cudaError_t launch_relevance(const StepArgs &a);
 cudaError_t launch_select(const StepArgs &a);

@@ -36,8 +36,9 @@ struct ProjSet {
 struct ProjParams {
   ProjSet set[2];
   int n_sets;
-  const void *q;       // [B, Hq, dh]
-  float *cq;           // [B][G][r_k]
+  const void *q;       // [B, Hq, dh], q_seq_stride elements between sequences
+  float *cq;           // [B][G][r_k], cq_seq_stride floats between sequences
+  int64_t q_seq_stride, cq_seq_stride;
   unsigned *hist;      // cleared when non-null, [B][2048]
   int32_t *coef_len;   // read when a token vector is present
   int bump_len;
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(256) k_project(ProjParams p) {
           const int v = i / Ds, d = d0 + (i - v * Ds);
           float x;
           if (v < nq)
-            x = Store<T>::ld((const T *)p.q + ((size_t)b * p.Hq + (size_t)(d / p.dh) * p.G + v) * p.dh + (d % p.dh));
+            x = Store<T>::ld((const T *)p.q + (size_t)b * p.q_seq_stride + ((size_t)(d / p.dh) * p.G + v) * p.dh + (d % p.dh));
           else
             x = Store<T>::ld((const T *)st.x_tok + (size_t)b * p.D + d);
           xs[i] = x;
@@ -172,7 +173,7 @@ __global__ void __launch_bounds__(256) k_project(ProjParams p) {
         for (int rk = 0; rk < CL; ++rk) s += partial[((size_t)rk * 2 + si) * p.slot + i];  // rank order
         const int v = i / r, col = i - v * r;
         if (v < nq)
-          p.cq[((size_t)b * p.G + v) * r + col] = s;
+          p.cq[(size_t)b * p.cq_seq_stride + (size_t)v * r + col] = s;
         else if (len >= 0)
           Store<T>::st((T *)st.coef + ((size_t)b * p.cap + len) * r + col, s);
       }
@@ -390,6 +391,8 @@ cudaError_t launch_qproj(const StepArgs &a) {
   ProjParams p = {};
   p.q = a.q;
   p.cq = (float *)(a.ws + a.plan.off_cq);
+  p.q_seq_stride = (int64_t)ly.Hq * ly.dh;
+  p.cq_seq_stride = (int64_t)ly.G * ly.rk;
   p.hist = (unsigned *)(a.ws + a.plan.off_hist);
   p.D = ly.D; p.G = ly.G; p.dh = ly.dh; p.Hq = ly.Hq; p.cap = ly.cap; p.dev_status = a.dev_status;
   p.set[0].basis = a.basis_k; p.set[0].r = ly.rk; p.set[0].nq = ly.G;
@@ -416,6 +419,19 @@ cudaError_t launch_qproj(const StepArgs &a) {
   }
   p.slot = project_slot(p);
   return ly.dtype == S4R_BF16 ? project_launch<__nv_bfloat16>(p, ly.B, a.stream) : project_launch<float>(p, ly.B, a.stream);
+}
+
+// Eq. 4: coefficients of one query per sequence, read and written with the caller's strides (the initial
+// query-coefficient window is filled row by row).
+cudaError_t launch_project_queries(const Layer &ly, const void *q, int64_t q_seq_stride, const void *basis_k, float *dst,
+                                   int64_t dst_seq_stride, cudaStream_t st) {
+  ProjParams p = {};
+  p.q = q; p.cq = dst; p.q_seq_stride = q_seq_stride; p.cq_seq_stride = dst_seq_stride;
+  p.D = ly.D; p.G = ly.G; p.dh = ly.dh; p.Hq = ly.Hq; p.cap = ly.cap;
+  p.set[0].basis = basis_k; p.set[0].r = ly.rk; p.set[0].nq = ly.G;
+  p.n_sets = 1;
+  p.slot = project_slot(p);
+  return ly.dtype == S4R_BF16 ? project_launch<__nv_bfloat16>(p, ly.B, st) : project_launch<float>(p, ly.B, st);
 }
 
 cudaError_t launch_append(const Layer &ly, const void *k_t, const void *v_t, const void *basis_k,

@@ -128,6 +128,48 @@ def test_window_longer_than_the_cache():
         assert err <= 1e-4            # every row is selected: what is left is the attention's own rounding
 
 
+@pytest.mark.parametrize("n_init", [0, 3, 8])
+def test_window_initialised_from_prompt_queries(n_init):
+    """Eq. 4: the library projects the last prompt queries itself; the rows must equal the oracle's projections and
+    the first windowed step on that window must agree with the oracle's step on the same rows."""
+    s4r = _s4r()
+    Wq = 8
+    cfg = W.scaled_config(W.get_config(1), context=3000 + 4, batch=2)
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    B, G, r, s = cfg.batch, cfg.group, cfg.rank_k, cfg.sink_count
+    qs = [_queries(cfg, p, b, n_init + 1) for b in range(B)]
+    cq = [[O.project_query(to_np(q), p.BK[b], cfg.n_kv_heads) for q in qs[b]] for b in range(B)]
+    win = torch.full((B, Wq, G, r), 3.0, dtype=torch.float32, device="cuda")
+    prompt_q = torch.stack([torch.stack(qs[b][:n_init]) for b in range(B)]).to("cuda") if n_init else None
+    s4r.window_init(ly, prompt_q, p.d_BK, win, score_window=Wq)
+    torch.cuda.synchronize()
+    got = win.double().cpu().numpy()
+    for b in range(B):
+        assert np.all(got[b, :Wq - n_init] == 0.0)
+        for i in range(n_init):
+            ref = cq[b][i]
+            assert np.abs(got[b, Wq - n_init + i] - ref).max() <= 2e-5 * np.abs(ref).max()
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=Wq)
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(B, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(B, dtype=torch.int32, device="cuda")
+    d_q = torch.stack([qs[b][n_init].to("cuda") for b in range(B)])
+    s4r.decode_step_windowed(ly, d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap, cfg.window,
+                             cfg.top_k, win, out, sel, cnt, ws, score_window=Wq, rope_theta=cfg.rope_theta)
+    torch.cuda.synchronize()
+    for b in range(B):
+        rows = [np.zeros((G, r))] * (Wq - 1 - n_init) + cq[b][max(0, n_init - (Wq - 1)):n_init + 1]
+        window_rows = np.stack(rows[-Wq:], axis=1)                               # [G, W_q, r], oldest first
+        res = O.decode_step(to_np(qs[b][n_init]), to_np(p.K[b][:s]), to_np(p.V[b][:s]), p.CK[b], p.CV[b], p.BK[b], p.BV[b],
+                            cfg.window, cfg.top_k, kappa=cfg.pool_kernel, pool_mode=cfg.pool_mode,
+                            group_mode=cfg.group_mode, theta=cfg.rope_theta, CQ_window=window_rows)
+        n = int(cnt[b].item())
+        got_idx = sel[b, :n].cpu().numpy().astype(np.int64)
+        ok, msg = O.selection_agrees(res["score"], res["idx"], got_idx, res["W_eff"], res["k_eff"], BAND)
+        assert ok, f"seq {b}: {msg}"
+
+
 def test_windowed_entry_rejects_what_it_cannot_do():
     s4r = _s4r()
     cfg = W.scaled_config(W.get_config(1), context=1000 + 4, batch=1)
