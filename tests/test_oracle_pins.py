@@ -218,6 +218,28 @@ def test_relevance_rows_sum_to_one_and_mask_is_causal():
     assert np.allclose(O.relevance(Z[:, 3:4, :]), sp.softmax(Z[:, 3, :], axis=-1), atol=1e-15)
 
 
+def test_window_mean_against_plain_loops():
+    """Eq. 9-10 written out with scalar loops: per group and window row a masked softmax, then the mean over the
+    window (divided by W_q even when some rows see nothing)."""
+    import math
+    rng = _rng(71)
+    for G, Wq, L in ((2, 3, 7), (1, 4, 2), (3, 1, 5)):
+        Z = rng.standard_normal((G, Wq, L))
+        want = np.zeros((G, L))
+        for g in range(G):
+            for i in range(Wq):
+                last = L - Wq + i
+                if last < 0:
+                    continue
+                den = sum(math.exp(Z[g, i, l]) for l in range(last + 1))
+                for l in range(last + 1):
+                    want[g, l] += math.exp(Z[g, i, l]) / den / Wq
+        got = O.relevance(Z)
+        assert np.allclose(got, want, atol=1e-14)
+        seeing = sum(1 for i in range(Wq) if L - Wq + i >= 0)
+        assert np.allclose(got.sum(axis=1), seeing / Wq, atol=1e-13)
+
+
 def test_ranking_without_pooling_is_argsort_of_logits():
     rng = _rng(8)
     cq = rng.standard_normal((1, 1, 6))
