@@ -495,29 +495,21 @@ def main():
     s4r.stage_timing(False)
     stage_ms = {k_: v_ / n_prof for k_, v_ in stage_sum.items()}
 
-    # ---- end to end: q, k_t, v_t from pinned host memory every step, results read back every step
+    # ---- end to end through the host-buffer entry point: every step one packed block {q, k_t, v_t} goes from pinned
+    #      host memory to the device, the fused call runs, and one block {out, sel_idx, sel_count} comes back
     c["len"].fill_(cfg.cache_len)
-    q_h = [qs[j].cpu().pin_memory() for j in range(pool)]
-    kt_h = [kt[j].cpu().pin_memory() for j in range(pool)]
-    vt_h = [vt[j].cpu().pin_memory() for j in range(pool)]
-    out_h = torch.empty(B, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32).pin_memory()
-    sel_h = torch.empty(B, n_sel, dtype=torch.int32).pin_memory()
-    cnt_h = torch.empty(B, dtype=torch.int32).pin_memory()
-    q_d, kt_d, vt_d = torch.empty_like(qs[0]), torch.empty_like(kt[0]), torch.empty_like(vt[0])
+    hs = s4r.HostStep(ly, cfg.window, cfg.top_k, torch.float32, device)
+    in_blocks = []
+    for j in range(pool):
+        hs.q.copy_(qs[j].cpu()); hs.k_t.copy_(kt[j].cpu()); hs.v_t.copy_(vt[j].cpu())
+        in_blocks.append(hs.in_host.clone().pin_memory())
+    kw_host = {k_: v_ for k_, v_ in kw.items()}
 
     def step_e2e(i):
-        # the call a user makes for one generated token: inputs from pinned host memory, one fused library call
-        # (cache update + decode step), results read back to the host before the next token
-        j = i % pool
-        kt_d.copy_(kt_h[j], non_blocking=True)
-        vt_d.copy_(vt_h[j], non_blocking=True)
-        q_d.copy_(q_h[j], non_blocking=True)
-        s4r.append_decode_step(ly, kt_d, vt_d, q_d, c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"],
-                               capacity, cfg.window, cfg.top_k, out, sel, cnt, c["ws"], **kw)
-        out_h.copy_(out, non_blocking=True)
-        sel_h.copy_(sel, non_blocking=True)
-        cnt_h.copy_(cnt, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        # the call a user makes for one generated token; its results are valid in hs.out / hs.sel_idx / hs.sel_count
+        # when it returns
+        s4r.append_decode_step_host(hs, c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"], capacity,
+                                    c["ws"], in_host=in_blocks[i % pool], **kw_host)
 
     for i in range(3):
         step_e2e(i)
@@ -529,8 +521,9 @@ def main():
     e2e_s = time.perf_counter() - t0
     e2e_s = replicas.max_over_ranks(e2e_s, dist, device)
     esz = cfg.elem_bytes
-    h2d = B * (cfg.n_q_heads * cfg.head_dim + 2 * cfg.d_kv) * esz
-    d2h = B * (cfg.n_q_heads * cfg.head_dim * 4 + n_sel * 4 + 4)
+    h2d, d2h = hs.h2d_bytes, hs.d2h_bytes
+    e2e_checksum = float(hs.out.abs().sum()) + int(hs.sel_count.sum())      # the host block was really written
+    assert e2e_checksum > 0
     dev_flags = int(status.item())
 
     if rank != 0:

@@ -15,7 +15,8 @@
  *     DEVICE pointer owned by the caller.  The library never allocates or
  *     frees device memory, keeps no state between calls (except the opt-in
  *     stage timing below) and never synchronises the stream (except
- *     s4r_decode_step_host and s4r_stage_times, see there).
+ *     s4r_decode_step_host, s4r_append_decode_step_host and s4r_stage_times,
+ *     see there).
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *     work of a call is enqueued on it, in order.  The device-pointer calls
  *     may be captured into a CUDA graph (after one uncaptured call on the
@@ -227,6 +228,25 @@ int s4r_decode_step_host(const s4r_layer_t *layer, const void *q_host, void *q_d
                          void *out_dev, int32_t out_dtype, int32_t *sel_idx_host, int32_t *sel_idx_dev,
                          int32_t *sel_count_host, int32_t *sel_count_dev, void *workspace,
                          size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/* The fused step (s4r_append_decode_step) for callers whose per-step data lives in HOST memory, with ONE copy
+ * in each direction.  The inputs of a step are packed in one block {q, k_t, v_t} and the results in one block
+ * {out, sel_idx, sel_count}; s4r_host_step_layout gives the byte offsets (each a multiple of 16):
+ *   in_off [4] = offsets of q [B, H_q, d_h], k_t [B, D'], v_t [B, D'] (layer dtype) and the block size
+ *   out_off[4] = offsets of out [B, H_q, d_h] (out_dtype), sel_idx [B, W + k] int32, sel_count [B] int32 and
+ *                the block size
+ * in_host / out_host are HOST blocks (pinned memory makes the copies asynchronous), in_dev / out_dev device
+ * staging blocks of the same sizes, 16-byte aligned.  The call copies in_host to in_dev, runs the step, copies
+ * out_dev to out_host and waits for the stream, so out_host is valid on return.  Errors as
+ * s4r_append_decode_step. */
+int s4r_host_step_layout(const s4r_layer_t *layer, int32_t window, int32_t top_k, int32_t out_dtype, size_t *in_off,
+                         size_t *out_off);
+int s4r_append_decode_step_host(const s4r_layer_t *layer, const void *in_host, void *in_dev, const void *sink_k,
+                                const void *sink_v, void *coef_k, void *coef_v, int32_t *coef_len,
+                                const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                                int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out_host,
+                                void *out_dev, int32_t out_dtype, void *workspace, size_t workspace_bytes,
+                                int32_t *dev_status, void *stream);
 
 /* The decode step for callers that cannot allocate device memory.  (The paper has no counterpart; this is
  * a property of the library, not of the method.)  Some callers have nowhere to get a workspace from: code

@@ -21,7 +21,7 @@ VALUE_AUTO, VALUE_RECONSTRUCT = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_workspace_bytes_windowed", "s4r_compress", "s4r_append", "s4r_decode_step",
-           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed", "s4r_window_init",
+           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed", "s4r_window_init", "s4r_host_step_layout", "s4r_append_decode_step_host",
            "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
            "s4r_stage_times", "s4r_strerror", "s4r_last_cuda_error", "s4r_version")
 STAGES = ("query_projection", "latent_scoring", "selection", "reconstruct_attend", "merge")
@@ -95,6 +95,11 @@ def load(build_if_missing: bool = True):
     lib.s4r_decode_step_host.restype = ctypes.c_int
     lib.s4r_decode_step_host.argtypes = [lp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, sp, rp, vp, vp, i32,
                                          vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.s4r_host_step_layout.restype = ctypes.c_int
+    lib.s4r_host_step_layout.argtypes = [lp, i32, i32, i32, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+    lib.s4r_append_decode_step_host.restype = ctypes.c_int
+    lib.s4r_append_decode_step_host.argtypes = [lp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, sp, rp, vp, vp, i32,
+                                                vp, sz, vp, vp]
     lib.s4r_top_k_from_ratio.restype = i64
     lib.s4r_top_k_from_ratio.argtypes = [ctypes.c_double, i64, i32]
     lib.s4r_rank_for_ratio.restype = i32
@@ -311,6 +316,61 @@ def decode_step_host(layer: Layer, q_host, q_dev, sink_k, sink_v, coef_k, coef_v
         _stream(stream))
     if rc != 0:
         raise S4RError(rc, "s4r_decode_step_host")
+
+
+class HostStep:
+    """Packed per-step blocks of s4r_append_decode_step_host: one pinned host block and one device block for the
+    inputs {q, k_t, v_t}, one of each for the results {out, sel_idx, sel_count}, with typed views into them."""
+
+    def __init__(self, layer: Layer, window: int, top_k: int, out_dtype=torch.float32, device="cuda"):
+        self.layer, self.window, self.top_k = layer, int(window), int(top_k)
+        self.out_code = S4R_BF16 if out_dtype == torch.bfloat16 else S4R_F32
+        io, oo = (ctypes.c_size_t * 4)(), (ctypes.c_size_t * 4)()
+        rc = load().s4r_host_step_layout(ctypes.byref(layer.c()), self.window, self.top_k, self.out_code, io, oo)
+        if rc != 0:
+            raise S4RError(rc, "s4r_host_step_layout")
+        io, oo = list(io), list(oo)
+        st = torch.bfloat16 if layer.dtype == S4R_BF16 else torch.float32
+        B, Hq, dh = layer.batch, layer.n_q_heads, layer.head_dim
+        D = layer.n_kv_heads * dh
+        self.in_host = torch.empty(io[3], dtype=torch.uint8).pin_memory()
+        self.out_host = torch.empty(oo[3], dtype=torch.uint8).pin_memory()
+        self.in_dev = torch.empty(io[3], dtype=torch.uint8, device=device)
+        self.out_dev = torch.empty(oo[3], dtype=torch.uint8, device=device)
+        esz = 2 if st == torch.bfloat16 else 4
+        osz = 2 if out_dtype == torch.bfloat16 else 4
+
+        def view(block, off, n, dtype, shape):
+            return block[off:off + n].view(dtype).view(*shape)
+        self.q = view(self.in_host, io[0], B * Hq * dh * esz, st, (B, Hq, dh))
+        self.k_t = view(self.in_host, io[1], B * D * esz, st, (B, D))
+        self.v_t = view(self.in_host, io[2], B * D * esz, st, (B, D))
+        self.out = view(self.out_host, oo[0], B * Hq * dh * osz, out_dtype, (B, Hq, dh))
+        self.sel_idx = view(self.out_host, oo[1], B * (self.window + self.top_k) * 4, torch.int32,
+                            (B, self.window + self.top_k))
+        self.sel_count = view(self.out_host, oo[2], B * 4, torch.int32, (B,))
+        self.h2d_bytes, self.d2h_bytes = io[3], oo[3]
+
+
+def append_decode_step_host(hs: HostStep, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis, max_len: int,
+                            workspace, *, pool_kernel: int = 7, pool_mode: int = POOL_MAX, group_mode: int = GROUP_MEAN,
+                            rope_theta: float = 0.0, value_path: int = VALUE_AUTO, dev_status=None, stream=None,
+                            in_host=None):
+    """s4r_append_decode_step_host: the caller fills hs.q / hs.k_t / hs.v_t (pinned host views); on return hs.out /
+    hs.sel_idx / hs.sel_count hold the step's results.  `in_host`: another host block of the same layout to read
+    the inputs from instead of hs.in_host."""
+    _need_cuda(coef_k, coef_v, coef_len, key_basis, value_basis, workspace)
+    src = hs.in_host if in_host is None else in_host
+    if src.numel() != hs.in_host.numel() or src.is_cuda:
+        raise ValueError("in_host must be a host block of hs.h2d_bytes bytes")
+    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, 1, rope_theta, value_path)
+    rc = load().s4r_append_decode_step_host(
+        ctypes.byref(hs.layer.c()), _ptr(src), _ptr(hs.in_dev), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k),
+        _ptr(coef_v), _ptr(coef_len), _ptr(key_basis), _ptr(value_basis), int(max_len), hs.window, hs.top_k,
+        ctypes.byref(sc), ctypes.byref(rp), _ptr(hs.out_host), _ptr(hs.out_dev), hs.out_code, _ptr(workspace),
+        workspace.numel(), _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_append_decode_step_host")
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

@@ -400,6 +400,47 @@ int s4r_decode_step_host(const s4r_layer_t *layer, const void *q_host, void *q_d
   return S4R_OK;
 }
 
+static size_t round16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+int s4r_host_step_layout(const s4r_layer_t *layer, int32_t window, int32_t top_k, int32_t out_dtype, size_t *in_off,
+                         size_t *out_off) {
+  Layer ly;
+  if (!layer_ok(layer, &ly) || !in_off || !out_off || window < 0 || top_k < 0) return S4R_ERR_INVALID_ARG;
+  if (out_dtype != S4R_F32 && out_dtype != S4R_BF16) return S4R_ERR_INVALID_ARG;
+  const size_t esz = ly.dtype == S4R_BF16 ? 2 : 4, osz = out_dtype == S4R_BF16 ? 2 : 4;
+  in_off[0] = 0;                                                         // q   [B, H_q, d_h]
+  in_off[1] = round16(in_off[0] + (size_t)ly.B * ly.Hq * ly.dh * esz);   // k_t [B, D']
+  in_off[2] = round16(in_off[1] + (size_t)ly.B * ly.D * esz);            // v_t [B, D']
+  in_off[3] = round16(in_off[2] + (size_t)ly.B * ly.D * esz);            // total
+  out_off[0] = 0;                                                                      // out       [B, H_q, d_h]
+  out_off[1] = round16(out_off[0] + (size_t)ly.B * ly.Hq * ly.dh * osz);               // sel_idx   [B, W + k]
+  out_off[2] = round16(out_off[1] + sizeof(int32_t) * ly.B * ((size_t)window + top_k)); // sel_count [B]
+  out_off[3] = round16(out_off[2] + sizeof(int32_t) * ly.B);                           // total
+  return S4R_OK;
+}
+
+int s4r_append_decode_step_host(const s4r_layer_t *layer, const void *in_host, void *in_dev, const void *sink_k,
+                                const void *sink_v, void *coef_k, void *coef_v, int32_t *coef_len,
+                                const void *key_basis, const void *value_basis, int64_t max_len, int32_t window,
+                                int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope, void *out_host,
+                                void *out_dev, int32_t out_dtype, void *workspace, size_t workspace_bytes,
+                                int32_t *dev_status, void *stream) {
+  size_t io[4], oo[4];
+  if (int rc = s4r_host_step_layout(layer, window, top_k, out_dtype, io, oo)) return rc;
+  if (!in_host || !in_dev || !out_host || !out_dev || !aligned16(in_dev) || !aligned16(out_dev)) return S4R_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cuda_failed(cudaMemcpyAsync(in_dev, in_host, io[3], cudaMemcpyHostToDevice, st))) return S4R_ERR_CUDA;
+  char *in = (char *)in_dev, *od = (char *)out_dev;
+  int rc = s4r_append_decode_step(layer, in + io[1], in + io[2], in + io[0], sink_k, sink_v, coef_k, coef_v, coef_len,
+                                  key_basis, value_basis, max_len, window, top_k, score, rope, od + oo[0], out_dtype,
+                                  (int32_t *)(od + oo[1]), (int32_t *)(od + oo[2]), workspace, workspace_bytes,
+                                  dev_status, stream);
+  if (rc != S4R_OK) return rc;
+  if (cuda_failed(cudaMemcpyAsync(out_host, out_dev, oo[3], cudaMemcpyDeviceToHost, st))) return S4R_ERR_CUDA;
+  if (cuda_failed(cudaStreamSynchronize(st))) return S4R_ERR_CUDA;
+  return S4R_OK;
+}
+
 // ---- decode step with built-in scratch, for callers that may not allocate --------------------------------
 // The array below is the whole workspace of one decode step.  In host code its name is only a handle for the
 // runtime (not a device address), so the address the kernels get is looked up once per device with

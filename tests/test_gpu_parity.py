@@ -324,6 +324,42 @@ def test_fused_append_decode_agrees_with_separate_calls():
     assert err <= 1e-3
 
 
+def test_fused_step_with_packed_host_blocks():
+    """s4r_append_decode_step_host: one copy in, the fused step, one copy out; the results in the pinned host
+    block must equal those of the device-pointer call on an identical cache."""
+    s4r = _s4r()
+    cfg = _cfg(1, context=3000 + 3, batch=2)
+    res = []
+    for host in (False, True):
+        p = Problem(cfg, device="cuda", capacity=cfg.cache_len + 4).upload()
+        ly = p.layer_desc()
+        ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, device="cuda")
+        sel = torch.empty(cfg.batch, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+        cnt = torch.empty(cfg.batch, dtype=torch.int32, device="cuda")
+        hs = s4r.HostStep(ly, cfg.window, cfg.top_k)
+        assert hs.h2d_bytes == hs.in_host.numel() and hs.d2h_bytes == hs.out_host.numel()
+        for step in (1, 2):
+            kt = torch.stack([W.make_token(cfg, 0, b, "k", step, "cpu") for b in range(cfg.batch)])
+            vt = torch.stack([W.make_token(cfg, 0, b, "v", step, "cpu") for b in range(cfg.batch)])
+            if host:
+                hs.q.copy_(p.d_q.cpu()); hs.k_t.copy_(kt); hs.v_t.copy_(vt)
+                hs.out_host.fill_(0x55)
+                s4r.append_decode_step_host(hs, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                            ws, rope_theta=cfg.rope_theta, dev_status=status)
+                out, sel, cnt = hs.out.clone(), hs.sel_idx.clone(), hs.sel_count.clone()   # valid on return, no sync
+            else:
+                s4r.append_decode_step(ly, kt.cuda(), vt.cuda(), p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len,
+                                       p.d_BK, p.d_BV, p.cap, cfg.window, cfg.top_k, out, sel, cnt, ws,
+                                       rope_theta=cfg.rope_theta, dev_status=status)
+                torch.cuda.synchronize()
+        assert status.item() == 0
+        res.append((out.cpu(), sel.cpu(), cnt.cpu(), p.d_CK.cpu(), p.d_len.cpu()))
+    for x, y in zip(res[0], res[1]):
+        assert torch.equal(x, y)
+
+
 def test_decode_step_replayed_from_a_cuda_graph():
     """A captured step must give the same result on every replay (the per-call token of the fused projection
     cannot be used there, so the library falls back to the separate projection kernel while capturing)."""
