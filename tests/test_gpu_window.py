@@ -50,6 +50,9 @@ def _run_case(cfg, Wq, steps=2, theta=None, cache_rows=None):
         before = win.clone()
         s4r.decode_step_windowed(ly, d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
                                  cfg.window, cfg.top_k, win, out, sel, cnt, ws, score_window=Wq, rope_theta=th,
+                                 pool_kernel=cfg.pool_kernel,
+                                 pool_mode={"max": s4r.POOL_MAX, "avg": s4r.POOL_AVG}[cfg.pool_mode],
+                                 group_mode={"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode],
                                  dev_status=status)
         torch.cuda.synchronize()
         assert status.item() == 0
@@ -84,6 +87,21 @@ def test_windowed_scoring_llama_shape(Wq):
     cfg = W.scaled_config(W.get_config(1), context=6000 + 4, batch=2)
     err = _run_case(cfg, Wq)
     print(f"W_q={Wq} (rows {Wq * cfg.group}): max rel err {err:.3e}")
+
+
+@pytest.mark.parametrize("Wq", [3, 16, 64, 96, 128])
+def test_window_lengths_that_change_the_kernel_layout(Wq):
+    """W_q = 16: eight-warp epilogue with four groups per column half; 64: one group per half; 96 and 128: a group
+    straddles column 64, so four warps read all columns (one group per launch pair); 3: general chunk code."""
+    cfg = W.scaled_config(W.get_config(1), context=3000 + 4, batch=1)
+    err = _run_case(cfg, Wq, steps=1)
+    print(f"W_q={Wq}: max rel err {err:.3e}")
+
+
+def test_windowed_scoring_without_rope_and_with_average_pooling():
+    cfg = W.scaled_config(W.get_config(1), context=3000 + 4, batch=1, pool_mode="avg", group_mode="max")
+    err = _run_case(cfg, 8, steps=1, theta=0.0)
+    print(f"W_q=8, avg pooling, group max, no RoPE: max rel err {err:.3e}")
 
 
 @pytest.mark.parametrize("Wq", [4, 32])
