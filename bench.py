@@ -165,10 +165,24 @@ def build_cache(cfg, s4r, device, capacity, seq_ids, layer=0, ws=None):
     torch.cuda.synchronize()
     compress_ms = e0.elapsed_time(e1)
     compress_launches = s4r.last_launch_count()
+    # subspace construction on the GPU (Eq. 1-2), timed on the same prompt; the cache above keeps the bases it
+    # was built with, so the decode numbers do not depend on this step
+    basis_ms = None
+    if layer == 0 and cfg.rank_k + 32 <= min(cfg.n_sampled, D) and cfg.rank_k <= 200:
+        idx = torch.stack([(W.sample_rows(cfg, layer, sid, "k") - s).to(torch.int32) for sid in seq_ids]).to(device)
+        sig = torch.empty(B, cfg.rank_k, dtype=torch.float32, device=device)
+        s4r.build_basis(ly, K, idx, cfg.rank_k, sigma=sig)                          # warm-up
+        torch.cuda.synchronize()
+        e0.record()
+        s4r.build_basis(ly, K, idx, cfg.rank_k, sigma=sig)
+        e1.record()
+        torch.cuda.synchronize()
+        basis_ms = e0.elapsed_time(e1)
+        del idx, sig
     del K, V
     torch.cuda.empty_cache()
     return dict(ly=ly, BK=BK, BV=BV, q=q, sink_k=sink_k, sink_v=sink_v, CK=CK, CV=CV, len=ln, ws=ws,
-                compress_ms=compress_ms, compress_launches=compress_launches)
+                compress_ms=compress_ms, compress_launches=compress_launches, basis_ms=basis_ms)
 
 
 def run_all_layers(args, cfg, s4r, device):
@@ -560,6 +574,8 @@ def main():
         "stage_ms": stage_ms,
         "compress": {"ms": c["compress_ms"], "tokens_per_s": B * (cfg.context - cfg.sink_count) / (c["compress_ms"] * 1e-3),
                      "launches": c["compress_launches"]},
+        "basis_build": {"ms": c["basis_ms"], "what": "s4r_build_basis, one tensor of the whole batch "
+                        "(%d sampled rows, rank %d)" % (cfg.n_sampled, cfg.rank_k)},
         "e2e": {"value": replicas.whole_job_rate(K_steps, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": gpu_launches, "clocks": clocks, "dev_status": dev_flags,
     }

@@ -64,6 +64,7 @@ typedef enum {
 /* flags OR-ed into *dev_status by kernels */
 #define S4R_DEV_TIMEOUT 1  /* a bounded wait (mbarrier) expired; results of that call are invalid */
 #define S4R_DEV_BOUNDS 2   /* coef_len[b] outside [0, max_len] or cache full on append; clamped   */
+#define S4R_DEV_NUMERIC 4  /* s4r_build_basis met a pivot that was not positive (rank-deficient sample) */
 
 #define S4R_F32 0
 #define S4R_BF16 1
@@ -120,6 +121,33 @@ size_t s4r_workspace_bytes(const s4r_layer_t *layer, int64_t max_len, int32_t wi
 #define S4R_MAX_SCORE_WINDOW 128
 size_t s4r_workspace_bytes_windowed(const s4r_layer_t *layer, int64_t max_len, int32_t window, int32_t top_k,
                                     int32_t score_window);
+
+/* Subspace construction (Sec. 3.1.2; Eq. 1: sampled rows L2-normalised along the feature dimension, Eq. 2: the
+ * top-r right singular vectors of the normalised sample), per sequence b and for ONE tensor (call it for the keys
+ * with rank_k and for the values with rank_v):
+ *   S_n[t]   = X[b, s + sample_idx[b, t]] / ||X[b, s + sample_idx[b, t]]||        t = 0 .. n_samples - 1
+ *   basis[b] = [D', rank] the rank leading right singular vectors of S_n, column i scaled by the sign that makes
+ *              its largest-magnitude entry positive (lowest index on ties), rounded to the layer dtype
+ *   sigma[b] = [rank] fp32 singular values (optional, may be NULL)
+ * X          [B, T, D'] pre-RoPE rows INCLUDING the s sink rows (device, layer dtype)
+ * sample_idx [B, n_samples] int32 NON-SINK indices in [0, T - s) (device); out-of-range entries set
+ *            S4R_DEV_BOUNDS and are clamped.  s4r_hybrid_sample_indices writes the paper's sampling pattern.
+ * Method: block power iteration with r + 32 vectors on the Gram matrix S_n^T S_n, n_iter iterations (<= 0: 24),
+ * Rayleigh-Ritz at the end; vector i converges like (sigma_{r+33} / sigma_i)^(2 n_iter), so the result is the
+ * SVD's up to that error and fp32 rounding.  Singular vectors whose singular values are closer than that are
+ * determined only as a subspace (by this routine as by any SVD in finite precision).
+ * Requirements: rank % 8 == 0, rank + 32 <= min(D', n_samples), rank <= 200 (S4R_ERR_UNSUPPORTED otherwise).
+ * workspace_bytes >= s4r_basis_workspace_bytes(...).  Asynchronous on `stream`.  A rank-deficient sample sets
+ * S4R_DEV_NUMERIC (the basis is then not orthonormal). */
+size_t s4r_basis_workspace_bytes(const s4r_layer_t *layer, int32_t rank, int32_t n_samples);
+int s4r_build_basis(const s4r_layer_t *layer, const void *X, int64_t T, const int32_t *sample_idx, int32_t n_samples,
+                    int32_t rank, int32_t n_iter, void *basis, float *sigma, void *workspace, size_t workspace_bytes,
+                    int32_t *dev_status, void *stream);
+
+/* Host helper: the paper's hybrid sampling (Sec. 3.1.2) over n_nonsink positions: a contiguous block of the
+ * ceil(recent_frac * n_samples) most recent positions plus evenly spread early positions floor(j * early / n_u)
+ * (duplicates removed).  Writes ascending indices to out (HOST, room for n_samples) and returns how many. */
+int32_t s4r_hybrid_sample_indices(int64_t n_nonsink, int32_t n_samples, double recent_frac, int32_t *out);
 
 /* Prefill-side projection (Sec. 3.1.1 sink split + Eq. 3), per sequence b:
  *   sink_k[b] = K[b, 0:s], sink_v[b] = V[b, 0:s]            (verbatim copies)

@@ -21,7 +21,8 @@ VALUE_AUTO, VALUE_RECONSTRUCT = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_workspace_bytes_windowed", "s4r_compress", "s4r_append", "s4r_decode_step",
-           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed", "s4r_window_init", "s4r_host_step_layout", "s4r_append_decode_step_host",
+           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed", "s4r_window_init", "s4r_host_step_layout", "s4r_append_decode_step_host", "s4r_basis_workspace_bytes", "s4r_build_basis",
+           "s4r_hybrid_sample_indices",
            "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
            "s4r_stage_times", "s4r_strerror", "s4r_last_cuda_error", "s4r_version")
 STAGES = ("query_projection", "latent_scoring", "selection", "reconstruct_attend", "merge")
@@ -95,6 +96,12 @@ def load(build_if_missing: bool = True):
     lib.s4r_decode_step_host.restype = ctypes.c_int
     lib.s4r_decode_step_host.argtypes = [lp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, sp, rp, vp, vp, i32,
                                          vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.s4r_basis_workspace_bytes.restype = sz
+    lib.s4r_basis_workspace_bytes.argtypes = [lp, i32, i32]
+    lib.s4r_build_basis.restype = ctypes.c_int
+    lib.s4r_build_basis.argtypes = [lp, vp, i64, vp, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    lib.s4r_hybrid_sample_indices.restype = i32
+    lib.s4r_hybrid_sample_indices.argtypes = [i64, i32, ctypes.c_double, ctypes.POINTER(i32)]
     lib.s4r_host_step_layout.restype = ctypes.c_int
     lib.s4r_host_step_layout.argtypes = [lp, i32, i32, i32, ctypes.POINTER(sz), ctypes.POINTER(sz)]
     lib.s4r_append_decode_step_host.restype = ctypes.c_int
@@ -316,6 +323,35 @@ def decode_step_host(layer: Layer, q_host, q_dev, sink_k, sink_v, coef_k, coef_v
         _stream(stream))
     if rc != 0:
         raise S4RError(rc, "s4r_decode_step_host")
+
+
+def hybrid_sample_indices(n_nonsink: int, n_samples: int, recent_frac: float = 0.7) -> torch.Tensor:
+    """s4r_hybrid_sample_indices: the paper's sampling pattern as an int32 CPU tensor of ascending non-sink indices."""
+    buf = (ctypes.c_int32 * max(int(n_samples), 1))()
+    n = load().s4r_hybrid_sample_indices(int(n_nonsink), int(n_samples), float(recent_frac), buf)
+    return torch.tensor(list(buf[:n]), dtype=torch.int32)
+
+
+def build_basis(layer: Layer, X, sample_idx, rank: int, *, n_iter: int = 0, sigma=None, workspace=None,
+                dev_status=None, stream=None) -> torch.Tensor:
+    """s4r_build_basis: X [B, T, D'] (with the sink rows), sample_idx [B, n_samples] int32 non-sink indices ->
+    basis [B, D', rank] in the layer dtype (returned); `sigma` [B, rank] fp32 receives the singular values."""
+    _need_cuda(X, sample_idx)
+    if sample_idx.dtype != torch.int32 or sample_idx.dim() != 2 or sample_idx.shape[0] != layer.batch:
+        raise ValueError("sample_idx must be an int32 tensor [B, n_samples]")
+    n_s = int(sample_idx.shape[1])
+    if workspace is None:
+        n = int(load().s4r_basis_workspace_bytes(ctypes.byref(layer.c()), int(rank), n_s))
+        if n == 0:
+            raise S4RError(-2, "s4r_basis_workspace_bytes")
+        workspace = torch.empty(n, dtype=torch.uint8, device=X.device)
+    basis = torch.empty(layer.batch, layer.d_kv, int(rank), dtype=layer.torch_dtype, device=X.device)
+    rc = load().s4r_build_basis(ctypes.byref(layer.c()), _ptr(X), int(X.shape[1]), _ptr(sample_idx), n_s, int(rank),
+                                int(n_iter), _ptr(basis), _ptr(sigma), _ptr(workspace), workspace.numel(),
+                                _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_build_basis")
+    return basis
 
 
 class HostStep:

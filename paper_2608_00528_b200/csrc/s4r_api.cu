@@ -142,6 +142,50 @@ size_t s4r_workspace_bytes_windowed(const s4r_layer_t *layer, int64_t max_len, i
   return w.total;
 }
 
+size_t s4r_basis_workspace_bytes(const s4r_layer_t *layer, int32_t rank, int32_t n_samples) {
+  Layer ly;
+  if (!layer_ok(layer, &ly) || n_samples < 1 || !basis_supported(ly, rank, n_samples)) return 0;
+  return basis_workspace(ly, rank, n_samples);
+}
+
+int s4r_build_basis(const s4r_layer_t *layer, const void *X, int64_t T, const int32_t *sample_idx, int32_t n_samples,
+                    int32_t rank, int32_t n_iter, void *basis, float *sigma, void *workspace, size_t workspace_bytes,
+                    int32_t *dev_status, void *stream) {
+  launch_counter() = 0;
+  Layer ly;
+  if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
+  if (!X || !sample_idx || !basis || n_samples < 1 || rank < 1 || T <= ly.s) return S4R_ERR_INVALID_ARG;
+  if (n_samples > 65535 || ly.B > 65535) return S4R_ERR_UNSUPPORTED;
+  if (!basis_supported(ly, rank, n_samples)) return S4R_ERR_UNSUPPORTED;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < basis_workspace(ly, rank, n_samples))
+    return S4R_ERR_WORKSPACE;
+  if (int rc = check_arch()) return rc;
+  if (cuda_failed(launch_build_basis(ly, X, T, sample_idx, n_samples, rank, n_iter > 0 ? n_iter : 24, basis, sigma,
+                                     (char *)workspace, dev_status, (cudaStream_t)stream)))
+    return S4R_ERR_CUDA;
+  return S4R_OK;
+}
+
+int32_t s4r_hybrid_sample_indices(int64_t n_nonsink, int32_t n_samples, double recent_frac, int32_t *out) {
+  if (!out || n_nonsink < 0 || n_samples < 0 || n_nonsink > 0x7fffffffLL) return 0;
+  if ((int64_t)n_samples > n_nonsink) n_samples = (int32_t)n_nonsink;
+  int64_t n_recent = (int64_t)ceil(recent_frac * (double)n_samples);
+  if (n_recent > n_samples) n_recent = n_samples;
+  if (n_recent < 0) n_recent = 0;
+  const int64_t n_uniform = n_samples - n_recent, early = n_nonsink - n_recent;
+  int32_t n = 0;
+  if (n_uniform > 0 && early > 0) {
+    int64_t last = -1;
+    for (int64_t j = 0; j < n_uniform; ++j) {
+      const int64_t v = (int64_t)floor((double)j * ((double)early / (double)n_uniform));
+      if (v != last) out[n++] = (int32_t)v;
+      last = v;
+    }
+  }
+  for (int64_t v = early; v < n_nonsink; ++v) out[n++] = (int32_t)v;
+  return n;
+}
+
 int s4r_compress(const s4r_layer_t *layer, const void *K, const void *V, int64_t T, const void *key_basis,
                  const void *value_basis, const void *norm_stats, void *sink_k, void *sink_v, void *coef_k,
                  void *coef_v, int32_t *coef_len, void *workspace, size_t workspace_bytes, int32_t *dev_status,

@@ -1,0 +1,455 @@
+// Subspace construction (Sec. 3.1.2, Eq. 1-2): the top-r right singular vectors of the L2-normalised sampled
+// rows, computed on the GPU as the dominant eigenvectors of the Gram matrix G = S_n^T S_n by block power
+// (orthogonal) iteration with a final Rayleigh-Ritz step.
+//
+//   1. k_basis_rows      gather the sampled rows and divide each by its L2 norm (Eq. 1)         A [n_s, D'] fp32
+//   2. k_gemm            G = A^T A                                                               [D', D'] fp32
+//   3. iterate on a block of p = r + 32 row vectors Q [p, D'] (deterministic pseudo-random start):
+//        Y = Q G, then Q = orth(Y) by two rounds of Cholesky QR:  M = Y Y^T accumulated in fp64,
+//        M = L L^T and L^-1 in fp64 by one CTA (k_chol_inv), Q = L^-1 Y.
+//      One multiplication by G spreads the rows of Y over a condition number of lambda_1 / lambda_p (several
+//      thousand for the spectra of interest), whose square is beyond fp32: hence the fp64 Gram and factor.
+//   4. Rayleigh-Ritz: H = (Q G) Q^T, H = W diag(lambda) W^T by a cyclic Jacobi method in shared memory
+//      (k_jacobi_eig), Ritz vectors = W^T Q, ordered by lambda.
+//   5. k_basis_finish    the r leading vectors, each with the sign that makes its largest-magnitude entry
+//                        positive (the SVD leaves it free), transposed to [D', r] in the storage type;
+//                        sigma_i = sqrt(lambda_i).
+// The error of vector i after k iterations falls like (lambda_{p+1} / lambda_i)^k.  Everything is batched over the
+// sequences of the layer.  The products run on the CUDA cores in fp32 (the whole construction is some 10 GFLOP per
+// sequence and tensor, next to 550 GFLOP for the projection of a 128K prompt).
+#include "s4r_internal.h"
+
+namespace s4r {
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------------------
+// rows: A[b][t][:] = X[b][s + idx[b][t]][:] / max(||.||, 1e-12)
+template <typename T>
+__global__ void __launch_bounds__(256) k_basis_rows(const T *X, const int32_t *idx, float *A, int64_t t_rows, int D,
+                                                    int n_s, int sinks, int32_t *dev_status) {
+  const int t = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  __shared__ float red[8];
+  int64_t row = (int64_t)sinks + idx[(size_t)b * n_s + t];
+  if (row < sinks || row >= t_rows) {  // uniform over the CTA
+    if (dev_status && tid == 0) atomicOr(dev_status, S4R_DEV_BOUNDS);
+    row = row < sinks ? sinks : t_rows - 1;
+  }
+  const T *x = X + ((size_t)b * t_rows + row) * D;
+  float ss = 0.f;
+  for (int d = tid; d < D; d += 256) {
+    const float v = Store<T>::ld(x + d);
+    ss += v * v;
+  }
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((tid & 31) == 0) red[tid >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float inv = 1.f / fmaxf(sqrtf(tot), 1e-12f);
+  float *a = A + ((size_t)b * n_s + t) * D;
+  for (int d = tid; d < D; d += 256) a[d] = Store<T>::ld(x + d) * inv;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// C[m][n] = sum_k A(m, k) B(k, n), element (m, k) of A at A[m sam + k sak], (k, n) of B at B[k sbk + n sbn];
+// batched (blockIdx.z).  64 x 64 tiles, 16 deep, 256 threads with 4 x 4 results each.  OUT = double accumulates
+// the exact fp32 products in fp64.
+struct GemmParams {
+  const float *A, *B;
+  void *C;
+  int M, N, K;
+  int64_t sam, sak, sbk, sbn, ldc, batch_a, batch_b, batch_c;
+};
+
+template <typename OUT>
+__global__ void __launch_bounds__(256) k_gemm(GemmParams p) {
+  __shared__ float As[16][64 + 1], Bs[16][64 + 1];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const float *A = p.A + (size_t)blockIdx.z * p.batch_a, *B = p.B + (size_t)blockIdx.z * p.batch_b;
+  OUT acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = (OUT)0;
+  // the index that is contiguous in memory varies fastest over the threads
+  const bool a_m_fast = p.sam == 1, b_n_fast = p.sbn == 1;
+  for (int k0 = 0; k0 < p.K; k0 += 16) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int e = tid + i * 256;
+      const int mm = a_m_fast ? (e & 63) : (e >> 4), kk = a_m_fast ? (e >> 6) : (e & 15);
+      const int m = m0 + mm, k = k0 + kk;
+      As[kk][mm] = (m < p.M && k < p.K) ? __ldg(A + (int64_t)m * p.sam + (int64_t)k * p.sak) : 0.f;
+      const int nn = b_n_fast ? (e & 63) : (e >> 4), kb = b_n_fast ? (e >> 6) : (e & 15);
+      const int n = n0 + nn, k2 = k0 + kb;
+      Bs[kb][nn] = (n < p.N && k2 < p.K) ? __ldg(B + (int64_t)k2 * p.sbk + (int64_t)n * p.sbn) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      float a[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] += (OUT)a[i] * (OUT)bv[j];
+    }
+    __syncthreads();
+  }
+  OUT *C = (OUT *)p.C + (size_t)blockIdx.z * p.batch_c;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+      if (m < p.M && n < p.N) C[(int64_t)m * p.ldc + n] = acc[i][j];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// deterministic start block: entry (b, i, d) from a 64-bit mix of its index, uniform in (-1, 1)
+__global__ void __launch_bounds__(256) k_basis_start(float *Q, int64_t n_per_batch, unsigned long long seed) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n_per_batch) return;
+  unsigned long long z = seed + 0x9e3779b97f4a7c15ull * (unsigned long long)(i + 1 + (int64_t)blockIdx.y * n_per_batch);
+  z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ull;
+  z = (z ^ (z >> 27)) * 0x94d049bb133111ebull;
+  z ^= z >> 31;
+  Q[(size_t)blockIdx.y * n_per_batch + i] = (float)((double)(z >> 11) * (2.0 / 9007199254740992.0) - 1.0);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// M = L L^T (fp64, lower triangle packed in shared memory), then L^-1 in place and out as fp32 [p][p] (zeros
+// above the diagonal).  One CTA per matrix.  A pivot that is not positive raises S4R_DEV_NUMERIC and is replaced.
+__device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }  // i >= j
+
+__global__ void __launch_bounds__(256) k_chol_inv(double *M, float *Linv, int p, int32_t *dev_status) {
+  extern __shared__ double Ls[];  // packed lower triangle
+  const int tid = threadIdx.x, b = blockIdx.x;
+  double *Mb = M + (size_t)b * p * p;
+  for (int e = tid; e < p * p; e += 256) {
+    const int i = e / p, j = e - i * p;
+    if (j <= i) Ls[tri(i, j)] = 0.5 * (Mb[(size_t)i * p + j] + Mb[(size_t)j * p + i]);
+  }
+  __syncthreads();
+  double scale = 0.0;  // largest diagonal entry: the measure a pivot is compared with
+  for (int i = 0; i < p; ++i) scale = fmax(scale, Ls[tri(i, i)]);
+  __syncthreads();
+  for (int j = 0; j < p; ++j) {
+    double d = Ls[tri(j, j)];
+    if (!(d > scale * 1e-14)) {  // also catches NaN
+      if (tid == 0 && dev_status) atomicOr(dev_status, S4R_DEV_NUMERIC);
+      d = scale * 1e-14 + 1e-300;
+    }
+    const double dj = sqrt(d), inv = 1.0 / dj;
+    __syncthreads();  // everyone has read the pivot
+    for (int i = j + tid; i < p; i += 256) Ls[tri(i, j)] = (i == j) ? dj : Ls[tri(i, j)] * inv;
+    __syncthreads();
+    // trailing update: L[i][k] -= L[i][j] L[k][j] for j < k <= i
+    const int n = p - j - 1;
+    for (int e = tid; e < n * n; e += 256) {
+      const int ii = e / n, kk = e - ii * n;
+      if (kk <= ii) {
+        const int i = j + 1 + ii, k = j + 1 + kk;
+        Ls[tri(i, k)] -= Ls[tri(i, j)] * Ls[tri(k, j)];
+      }
+    }
+    __syncthreads();
+  }
+  // X = L^-1 in place, column by column from the right: X[i][j] = -(sum_{k=j+1..i} X[i][k] L[k][j]) / L[j][j]
+  double *col = Ls + (size_t)p * (p + 1) / 2;  // copy of column j of L
+  for (int j = p - 1; j >= 0; --j) {
+    for (int k = j + tid; k < p; k += 256) col[k] = Ls[tri(k, j)];
+    __syncthreads();
+    const double xjj = 1.0 / col[j];
+    for (int i = j + tid; i < p; i += 256) {
+      if (i == j) {
+        Ls[tri(j, j)] = xjj;
+      } else {
+        double sum = 0.0;
+        for (int k = j + 1; k <= i; ++k) sum += Ls[tri(i, k)] * col[k];
+        Ls[tri(i, j)] = -sum * xjj;
+      }
+    }
+    __syncthreads();
+  }
+  float *Lo = Linv + (size_t)b * p * p;
+  for (int e = tid; e < p * p; e += 256) {
+    const int i = e / p, j = e - i * p;
+    Lo[e] = j <= i ? (float)Ls[tri(i, j)] : 0.f;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Symmetric eigendecomposition H = W diag(lambda) W^T of a p x p matrix (p even) by the cyclic Jacobi method with
+// the round-robin ordering: p / 2 disjoint rotations per round, p - 1 rounds per sweep.  H sits in shared memory,
+// the eigenvectors (rows of Wt) in global memory.  One CTA per matrix.
+constexpr int kJacThreads = 1024;
+constexpr int kJacSweeps = 16;
+
+__global__ void __launch_bounds__(kJacThreads) k_jacobi_eig(const float *H, float *Wt, float *lam, int32_t *perm, int p) {
+  extern __shared__ float Hs[];  // [p][p + 1]
+  const int ld = p + 1, half = p >> 1;
+  int *pi = reinterpret_cast<int *>(Hs + (size_t)p * ld), *pj = pi + half;
+  float *pc = reinterpret_cast<float *>(pj + half), *psn = pc + half;
+  __shared__ unsigned s_off;  // largest |a_pq| / sqrt(a_pp a_qq) seen in a sweep, as float bits
+  const int tid = threadIdx.x, b = blockIdx.x;
+  const float *Hb = H + (size_t)b * p * p;
+  float *Wb = Wt + (size_t)b * p * p;
+  for (int e = tid; e < p * p; e += kJacThreads) {
+    const int i = e / p, j = e - i * p;
+    Hs[i * ld + j] = 0.5f * (Hb[e] + Hb[(size_t)j * p + i]);
+    Wb[e] = i == j ? 1.f : 0.f;
+  }
+  __syncthreads();
+  for (int sweep = 0; sweep < kJacSweeps; ++sweep) {
+    if (tid == 0) s_off = 0u;
+    __syncthreads();
+    for (int t = 0; t < p - 1; ++t) {
+      if (tid < half) {
+        const int k = tid;
+        int i = k == 0 ? t : (t + k) % (p - 1);
+        int j = k == 0 ? p - 1 : (t - k + (p - 1)) % (p - 1);
+        if (i > j) {
+          const int tmp = i;
+          i = j;
+          j = tmp;
+        }
+        const float app = Hs[i * ld + i], aqq = Hs[j * ld + j], apq = Hs[i * ld + j];
+        float c = 1.f, s = 0.f;
+        const float ref = sqrtf(fabsf(app * aqq));
+        if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * ref) {
+          const float theta = (aqq - app) / (2.f * apq);
+          const float tt = (theta >= 0.f ? 1.f : -1.f) / (fabsf(theta) + sqrtf(theta * theta + 1.f));
+          c = rsqrtf(tt * tt + 1.f);
+          s = tt * c;
+          atomicMax(&s_off, __float_as_uint(fabsf(apq) / fmaxf(ref, 1e-30f)));
+        }
+        pi[k] = i; pj[k] = j; pc[k] = c; psn[k] = s;
+      }
+      __syncthreads();
+      // columns i, j of H, all rows
+      for (int e = tid; e < half * p; e += kJacThreads) {
+        const int k = e / p, r = e - k * p;
+        const float c = pc[k], s = psn[k];
+        if (s != 0.f) {
+          float *hp = Hs + r * ld + pi[k], *hq = Hs + r * ld + pj[k];
+          const float a = *hp, q = *hq;
+          *hp = c * a - s * q;
+          *hq = s * a + c * q;
+        }
+      }
+      __syncthreads();
+      // rows i, j of H and of the eigenvector matrix, all columns
+      for (int e = tid; e < half * p; e += kJacThreads) {
+        const int k = e / p, col = e - k * p;
+        const float c = pc[k], s = psn[k];
+        if (s != 0.f) {
+          float *hp = Hs + pi[k] * ld + col, *hq = Hs + pj[k] * ld + col;
+          const float a = *hp, q = *hq;
+          *hp = c * a - s * q;
+          *hq = s * a + c * q;
+          float *wp = Wb + (size_t)pi[k] * p + col, *wq = Wb + (size_t)pj[k] * p + col;
+          const float wa = *wp, wb = *wq;
+          *wp = c * wa - s * wb;
+          *wq = s * wa + c * wb;
+        }
+      }
+      __syncthreads();
+    }
+    if (__uint_as_float(s_off) < 2e-7f) break;  // uniform: read after the round's last barrier
+    __syncthreads();
+  }
+  // eigenvalues and their descending order (ties: lower index first)
+  for (int i = tid; i < p; i += kJacThreads) {
+    const float li = Hs[i * ld + i];
+    int rank = 0;
+    for (int j = 0; j < p; ++j) {
+      const float lj = Hs[j * ld + j];
+      rank += (lj > li || (lj == li && j < i)) ? 1 : 0;
+    }
+    lam[(size_t)b * p + i] = li;
+    perm[(size_t)b * p + rank] = i;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// basis[b][:, c] = sign * Ritz vector perm[c]; sign makes the entry of largest magnitude (lowest index on ties)
+// positive.  sigma[b][c] = sqrt(lambda).  grid (r, B).
+template <typename T>
+__global__ void __launch_bounds__(256) k_basis_finish(const float *Rt, const float *lam, const int32_t *perm, T *basis,
+                                                      float *sigma, int p, int D, int r) {
+  const int c = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int src = perm[(size_t)b * p + c];
+  const float *v = Rt + ((size_t)b * p + src) * D;
+  __shared__ float s_val[256];
+  __shared__ int s_idx[256];
+  float best = -1.f;
+  int bi = 0x7fffffff;
+  for (int d = tid; d < D; d += 256) {
+    const float a = fabsf(v[d]);
+    if (a > best) {
+      best = a;
+      bi = d;
+    }
+  }
+  s_val[tid] = best;
+  s_idx[tid] = bi;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (tid < o) {
+      const float ov = s_val[tid + o];
+      const int oi = s_idx[tid + o];
+      if (ov > s_val[tid] || (ov == s_val[tid] && oi < s_idx[tid])) {
+        s_val[tid] = ov;
+        s_idx[tid] = oi;
+      }
+    }
+    __syncthreads();
+  }
+  const float sign = v[s_idx[0]] < 0.f ? -1.f : 1.f;
+  T *out = basis + (size_t)b * D * r + c;
+  for (int d = tid; d < D; d += 256) Store<T>::st(out + (size_t)d * r, sign * v[d]);
+  if (sigma && tid == 0) sigma[(size_t)b * r + c] = sqrtf(fmaxf(lam[(size_t)b * p + src], 0.f));
+}
+
+template <typename OUT>
+cudaError_t gemm(const float *A, const float *B, OUT *C, int M, int N, int K, int64_t sam, int64_t sak, int64_t sbk,
+                 int64_t sbn, int64_t ba, int64_t bb, int64_t bc, int batch, cudaStream_t st) {
+  GemmParams g;
+  g.A = A; g.B = B; g.C = C; g.M = M; g.N = N; g.K = K; g.sam = sam; g.sak = sak; g.sbk = sbk; g.sbn = sbn; g.ldc = N;
+  g.batch_a = ba; g.batch_b = bb; g.batch_c = bc;
+  k_gemm<OUT><<<dim3((N + 63) / 64, (M + 63) / 64, batch), 256, 0, st>>>(g);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int basis_block(int rank) { return rank + 32; }
+
+bool basis_supported(const Layer &ly, int rank, int n_samples) {
+  const int p = basis_block(rank);
+  if (rank < 1 || rank % 8 || p > ly.D || p > n_samples || (p & 1)) return false;
+  const size_t jac = sizeof(float) * (size_t)p * (p + 1) + sizeof(int) * 2 * (size_t)p + 64;
+  const size_t chol = sizeof(double) * ((size_t)p * (p + 1) / 2 + p);
+  return jac <= 226 * 1024 && chol <= 226 * 1024;
+}
+
+// Workspace layout (bytes, each part 256-byte aligned), in this order:
+//   A [B][n_s][D] f32 | G [B][D][D] f32 | Q, Y [B][p][D] f32 | M [B][p][p] f64 | Linv, H, Wt [B][p][p] f32 |
+//   lam [B][p] f32 | perm [B][p] i32
+size_t basis_workspace(const Layer &ly, int rank, int n_samples) {
+  const size_t p = basis_block(rank), B = ly.B, D = ly.D;
+  size_t off = 0;
+  auto add = [&](size_t bytes) { off = (off + bytes + 255) & ~(size_t)255; };
+  add(4 * B * n_samples * D);
+  add(4 * B * D * D);
+  add(4 * B * p * D);
+  add(4 * B * p * D);
+  add(8 * B * p * p);
+  add(4 * B * p * p);
+  add(4 * B * p * p);
+  add(4 * B * p * p);
+  add(4 * B * p);
+  add(4 * B * p);
+  return off;
+}
+
+cudaError_t launch_build_basis(const Layer &ly, const void *X, int64_t t_rows, const int32_t *sample_idx, int n_s,
+                               int rank, int n_iter, void *basis, float *sigma, char *ws, int32_t *dev_status,
+                               cudaStream_t st) {
+  const int B = ly.B, D = ly.D, p = basis_block(rank);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    char *ptr = ws + off;
+    off = (off + bytes + 255) & ~(size_t)255;
+    return ptr;
+  };
+  float *A = (float *)take(4ull * B * n_s * D);
+  float *G = (float *)take(4ull * B * D * D);
+  float *Q = (float *)take(4ull * B * p * D);
+  float *Y = (float *)take(4ull * B * p * D);
+  double *M = (double *)take(8ull * B * p * p);
+  float *Linv = (float *)take(4ull * B * p * p);
+  float *H = (float *)take(4ull * B * p * p);
+  float *Wt = (float *)take(4ull * B * p * p);
+  float *lam = (float *)take(4ull * B * p);
+  int32_t *perm = (int32_t *)take(4ull * B * p);
+  const int64_t pD = (int64_t)p * D, pp = (int64_t)p * p, DD = (int64_t)D * D;
+  cudaError_t e;
+#define S4R_TRY(x) do { e = (x); if (e != cudaSuccess) return e; } while (0)
+  // 1. normalised sampled rows
+  if (ly.dtype == S4R_BF16)
+    k_basis_rows<__nv_bfloat16><<<dim3(n_s, B), 256, 0, st>>>((const __nv_bfloat16 *)X, sample_idx, A, t_rows, D, n_s, ly.s, dev_status);
+  else
+    k_basis_rows<float><<<dim3(n_s, B), 256, 0, st>>>((const float *)X, sample_idx, A, t_rows, D, n_s, ly.s, dev_status);
+  ++launch_counter();
+  S4R_TRY(cudaGetLastError());
+  // 2. G = A^T A
+  S4R_TRY(gemm<float>(A, A, G, D, D, n_s, 1, D, D, 1, (int64_t)n_s * D, (int64_t)n_s * D, DD, B, st));
+  // 3. block iteration
+  static size_t chol_set = 0, jac_set = 0;
+  const size_t chol_smem = sizeof(double) * ((size_t)p * (p + 1) / 2 + p);
+  const size_t jac_smem = sizeof(float) * (size_t)p * (p + 1) + sizeof(int) * 2 * (size_t)p + 64;
+  if (chol_smem > chol_set) {
+    S4R_TRY(cudaFuncSetAttribute(k_chol_inv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem));
+    chol_set = chol_smem;
+  }
+  if (jac_smem > jac_set) {
+    S4R_TRY(cudaFuncSetAttribute(k_jacobi_eig, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jac_smem));
+    jac_set = jac_smem;
+  }
+  k_basis_start<<<dim3((unsigned)((pD + 255) / 256), B), 256, 0, st>>>(Y, pD, 0x5334523472ull);
+  ++launch_counter();
+  S4R_TRY(cudaGetLastError());
+  auto orthonormalise = [&](float *src, float *dst) -> cudaError_t {  // dst = orth(src); src is overwritten
+    float *in = src, *out = dst;
+    for (int round = 0; round < 2; ++round) {
+      cudaError_t e2 = gemm<double>(in, in, M, p, p, D, D, 1, 1, D, pD, pD, pp, B, st);  // M = in in^T
+      if (e2 != cudaSuccess) return e2;
+      k_chol_inv<<<B, 256, chol_smem, st>>>(M, Linv, p, dev_status);
+      ++launch_counter();
+      if ((e2 = cudaGetLastError()) != cudaSuccess) return e2;
+      e2 = gemm<float>(Linv, in, out, p, D, p, p, 1, D, 1, pp, pD, pD, B, st);  // out = L^-1 in
+      if (e2 != cudaSuccess) return e2;
+      float *tmp = in;
+      in = out;
+      out = tmp;
+    }
+    return cudaSuccess;  // after two rounds the result is back in `src`... see the caller
+  };
+  // two rounds ping-pong src -> dst -> src, so the orthonormal block ends in its first argument
+  S4R_TRY(orthonormalise(Y, Q));
+  float *Qc = Y, *Yc = Q;  // Qc: orthonormal block, Yc: scratch
+  for (int it = 0; it < n_iter; ++it) {
+    S4R_TRY(gemm<float>(Qc, G, Yc, p, D, D, D, 1, D, 1, pD, DD, pD, B, st));  // Yc = Qc G
+    S4R_TRY(orthonormalise(Yc, Qc));
+    float *tmp = Qc;
+    Qc = Yc;
+    Yc = tmp;
+  }
+  // 4. Rayleigh-Ritz
+  S4R_TRY(gemm<float>(Qc, G, Yc, p, D, D, D, 1, D, 1, pD, DD, pD, B, st));     // Z = Q G
+  S4R_TRY(gemm<float>(Yc, Qc, H, p, p, D, D, 1, 1, D, pD, pD, pp, B, st));     // H = Z Q^T
+  k_jacobi_eig<<<B, kJacThreads, jac_smem, st>>>(H, Wt, lam, perm, p);
+  ++launch_counter();
+  S4R_TRY(cudaGetLastError());
+  S4R_TRY(gemm<float>(Wt, Qc, Yc, p, D, p, p, 1, D, 1, pp, pD, pD, B, st));    // Ritz vectors = Wt Q
+  // 5. leading r vectors, sign convention, storage type
+  if (ly.dtype == S4R_BF16)
+    k_basis_finish<__nv_bfloat16><<<dim3(rank, B), 256, 0, st>>>(Yc, lam, perm, (__nv_bfloat16 *)basis, sigma, p, D, rank);
+  else
+    k_basis_finish<float><<<dim3(rank, B), 256, 0, st>>>(Yc, lam, perm, (float *)basis, sigma, p, D, rank);
+  ++launch_counter();
+  S4R_TRY(cudaGetLastError());
+#undef S4R_TRY
+  return cudaSuccess;
+}
+
+}  // namespace s4r

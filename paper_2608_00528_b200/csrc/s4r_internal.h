@@ -40,6 +40,11 @@ int &launch_counter();
 
 // generic (any supported geometry, fp32 or bf16 storage, CUDA-core arithmetic in fp32)
 cudaError_t launch_qproj(const StepArgs &a);
+bool basis_supported(const Layer &ly, int rank, int n_samples);
+size_t basis_workspace(const Layer &ly, int rank, int n_samples);
+cudaError_t launch_build_basis(const Layer &ly, const void *X, int64_t t_rows, const int32_t *sample_idx, int n_s,
+                               int rank, int n_iter, void *basis, float *sigma, char *ws, int32_t *dev_status,
+                               cudaStream_t st);
 cudaError_t launch_project_queries(const Layer &ly, const void *q, int64_t q_seq_stride, const void *basis_k, float *dst,
                                    int64_t dst_seq_stride, cudaStream_t st);
 cudaError_t launch_scan_generic(const StepArgs &a);
