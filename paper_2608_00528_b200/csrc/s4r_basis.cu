@@ -5,8 +5,8 @@
 //   1. k_basis_rows      gather the sampled rows and divide each by its L2 norm (Eq. 1)         A [n_s, D'] fp32
 //   2. k_gemm            G = A^T A                                                               [D', D'] fp32
 //   3. iterate on a block of p = r + 32 row vectors Q [p, D'] (deterministic pseudo-random start):
-//        Y = Q G, then Q = orth(Y) by two rounds of Cholesky QR:  M = Y Y^T accumulated in fp64,
-//        M = L L^T and L^-1 in fp64 by one CTA (k_chol_inv), Q = L^-1 Y.
+//        Y = Q G, then Q = orth(Y) by Cholesky QR:  M = Y Y^T accumulated in fp64, M = L L^T and L^-1 in
+//        fp64 by one CTA (k_chol_inv), Q = L^-1 Y; a second round before the Rayleigh-Ritz step.
 //      One multiplication by G spreads the rows of Y over a condition number of lambda_1 / lambda_p (several
 //      thousand for the spectra of interest), whose square is beyond fp32: hence the fp64 Gram and factor.
 //   4. Rayleigh-Ritz: H = (Q G) Q^T, H = W diag(lambda) W^T by a cyclic Jacobi method in shared memory
@@ -128,11 +128,13 @@ __global__ void __launch_bounds__(256) k_basis_start(float *Q, int64_t n_per_bat
 // above the diagonal).  One CTA per matrix.  A pivot that is not positive raises S4R_DEV_NUMERIC and is replaced.
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }  // i >= j
 
-__global__ void __launch_bounds__(256) k_chol_inv(double *M, float *Linv, int p, int32_t *dev_status) {
-  extern __shared__ double Ls[];  // packed lower triangle
-  const int tid = threadIdx.x, b = blockIdx.x;
+constexpr int kCholThreads = 1024;
+
+__global__ void __launch_bounds__(kCholThreads) k_chol_inv(double *M, float *Linv, int p, int32_t *dev_status) {
+  extern __shared__ double Ls[];  // packed lower triangle, then one column
+  const int tid = threadIdx.x, b = blockIdx.x, lane = tid & 31, warp = tid >> 5;
   double *Mb = M + (size_t)b * p * p;
-  for (int e = tid; e < p * p; e += 256) {
+  for (int e = tid; e < p * p; e += kCholThreads) {
     const int i = e / p, j = e - i * p;
     if (j <= i) Ls[tri(i, j)] = 0.5 * (Mb[(size_t)i * p + j] + Mb[(size_t)j * p + i]);
   }
@@ -148,38 +150,33 @@ __global__ void __launch_bounds__(256) k_chol_inv(double *M, float *Linv, int p,
     }
     const double dj = sqrt(d), inv = 1.0 / dj;
     __syncthreads();  // everyone has read the pivot
-    for (int i = j + tid; i < p; i += 256) Ls[tri(i, j)] = (i == j) ? dj : Ls[tri(i, j)] * inv;
+    for (int i = j + tid; i < p; i += kCholThreads) Ls[tri(i, j)] = (i == j) ? dj : Ls[tri(i, j)] * inv;
     __syncthreads();
-    // trailing update: L[i][k] -= L[i][j] L[k][j] for j < k <= i
-    const int n = p - j - 1;
-    for (int e = tid; e < n * n; e += 256) {
-      const int ii = e / n, kk = e - ii * n;
-      if (kk <= ii) {
-        const int i = j + 1 + ii, k = j + 1 + kk;
-        Ls[tri(i, k)] -= Ls[tri(i, j)] * Ls[tri(k, j)];
-      }
+    // trailing update: L[i][k] -= L[i][j] L[k][j] for j < k <= i; a warp takes rows, its lanes take columns
+    for (int i = j + 1 + warp; i < p; i += kCholThreads / 32) {
+      const double lij = Ls[tri(i, j)];
+      for (int k = j + 1 + lane; k <= i; k += 32) Ls[tri(i, k)] -= lij * Ls[tri(k, j)];
     }
     __syncthreads();
   }
-  // X = L^-1 in place, column by column from the right: X[i][j] = -(sum_{k=j+1..i} X[i][k] L[k][j]) / L[j][j]
+  // X = L^-1 in place, column by column from the right: X[i][j] = -(sum_{k=j+1..i} X[i][k] L[k][j]) / L[j][j];
+  // a warp takes rows, its lanes split the sum
   double *col = Ls + (size_t)p * (p + 1) / 2;  // copy of column j of L
   for (int j = p - 1; j >= 0; --j) {
-    for (int k = j + tid; k < p; k += 256) col[k] = Ls[tri(k, j)];
+    for (int k = j + tid; k < p; k += kCholThreads) col[k] = Ls[tri(k, j)];
     __syncthreads();
     const double xjj = 1.0 / col[j];
-    for (int i = j + tid; i < p; i += 256) {
-      if (i == j) {
-        Ls[tri(j, j)] = xjj;
-      } else {
-        double sum = 0.0;
-        for (int k = j + 1; k <= i; ++k) sum += Ls[tri(i, k)] * col[k];
-        Ls[tri(i, j)] = -sum * xjj;
-      }
+    if (tid == 0) Ls[tri(j, j)] = xjj;
+    for (int i = j + 1 + warp; i < p; i += kCholThreads / 32) {
+      double sum = 0.0;
+      for (int k = j + 1 + lane; k <= i; k += 32) sum += Ls[tri(i, k)] * col[k];
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) Ls[tri(i, j)] = -sum * xjj;
     }
     __syncthreads();
   }
   float *Lo = Linv + (size_t)b * p * p;
-  for (int e = tid; e < p * p; e += 256) {
+  for (int e = tid; e < p * p; e += kCholThreads) {
     const int i = e / p, j = e - i * p;
     Lo[e] = j <= i ? (float)Ls[tri(i, j)] : 0.f;
   }
@@ -197,8 +194,9 @@ __global__ void __launch_bounds__(kJacThreads) k_jacobi_eig(const float *H, floa
   const int ld = p + 1, half = p >> 1;
   int *pi = reinterpret_cast<int *>(Hs + (size_t)p * ld), *pj = pi + half;
   float *pc = reinterpret_cast<float *>(pj + half), *psn = pc + half;
-  __shared__ unsigned s_off;  // largest |a_pq| / sqrt(a_pp a_qq) seen in a sweep, as float bits
-  const int tid = threadIdx.x, b = blockIdx.x;
+  __shared__ unsigned s_off;  // largest |a_pq| seen in a sweep, as float bits
+  __shared__ float s_dmax;    // largest diagonal entry at the start: H carries absolute errors of eps * that
+  const int tid = threadIdx.x, b = blockIdx.x, lane = tid & 31, warp = tid >> 5;
   const float *Hb = H + (size_t)b * p * p;
   float *Wb = Wt + (size_t)b * p * p;
   for (int e = tid; e < p * p; e += kJacThreads) {
@@ -207,6 +205,13 @@ __global__ void __launch_bounds__(kJacThreads) k_jacobi_eig(const float *H, floa
     Wb[e] = i == j ? 1.f : 0.f;
   }
   __syncthreads();
+  if (tid == 0) {
+    float m = 0.f;
+    for (int i = 0; i < p; ++i) m = fmaxf(m, fabsf(Hs[i * ld + i]));
+    s_dmax = m;
+  }
+  __syncthreads();
+  const float dmax = s_dmax;
   for (int sweep = 0; sweep < kJacSweeps; ++sweep) {
     if (tid == 0) s_off = 0u;
     __syncthreads();
@@ -222,47 +227,50 @@ __global__ void __launch_bounds__(kJacThreads) k_jacobi_eig(const float *H, floa
         }
         const float app = Hs[i * ld + i], aqq = Hs[j * ld + j], apq = Hs[i * ld + j];
         float c = 1.f, s = 0.f;
-        const float ref = sqrtf(fabsf(app * aqq));
-        if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * ref) {
+        atomicMax(&s_off, __float_as_uint(fabsf(apq)));
+        if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * dmax) {
           const float theta = (aqq - app) / (2.f * apq);
           const float tt = (theta >= 0.f ? 1.f : -1.f) / (fabsf(theta) + sqrtf(theta * theta + 1.f));
           c = rsqrtf(tt * tt + 1.f);
           s = tt * c;
-          atomicMax(&s_off, __float_as_uint(fabsf(apq) / fmaxf(ref, 1e-30f)));
         }
         pi[k] = i; pj[k] = j; pc[k] = c; psn[k] = s;
       }
       __syncthreads();
-      // columns i, j of H, all rows
-      for (int e = tid; e < half * p; e += kJacThreads) {
-        const int k = e / p, r = e - k * p;
+      // columns i, j of H, all rows: a warp takes pairs, its lanes take rows
+      for (int k = warp; k < half; k += kJacThreads / 32) {
         const float c = pc[k], s = psn[k];
         if (s != 0.f) {
-          float *hp = Hs + r * ld + pi[k], *hq = Hs + r * ld + pj[k];
-          const float a = *hp, q = *hq;
-          *hp = c * a - s * q;
-          *hq = s * a + c * q;
+          const int i = pi[k], j = pj[k];
+          for (int r = lane; r < p; r += 32) {
+            float *hp = Hs + r * ld + i, *hq = Hs + r * ld + j;
+            const float a = *hp, q = *hq;
+            *hp = c * a - s * q;
+            *hq = s * a + c * q;
+          }
         }
       }
       __syncthreads();
       // rows i, j of H and of the eigenvector matrix, all columns
-      for (int e = tid; e < half * p; e += kJacThreads) {
-        const int k = e / p, col = e - k * p;
+      for (int k = warp; k < half; k += kJacThreads / 32) {
         const float c = pc[k], s = psn[k];
         if (s != 0.f) {
-          float *hp = Hs + pi[k] * ld + col, *hq = Hs + pj[k] * ld + col;
-          const float a = *hp, q = *hq;
-          *hp = c * a - s * q;
-          *hq = s * a + c * q;
-          float *wp = Wb + (size_t)pi[k] * p + col, *wq = Wb + (size_t)pj[k] * p + col;
-          const float wa = *wp, wb = *wq;
-          *wp = c * wa - s * wb;
-          *wq = s * wa + c * wb;
+          const int i = pi[k], j = pj[k];
+          float *wi = Wb + (size_t)i * p, *wj = Wb + (size_t)j * p;
+          for (int col = lane; col < p; col += 32) {
+            float *hp = Hs + i * ld + col, *hq = Hs + j * ld + col;
+            const float a = *hp, q = *hq;
+            *hp = c * a - s * q;
+            *hq = s * a + c * q;
+            const float wa = wi[col], wb = wj[col];
+            wi[col] = c * wa - s * wb;
+            wj[col] = s * wa + c * wb;
+          }
         }
       }
       __syncthreads();
     }
-    if (__uint_as_float(s_off) < 2e-7f) break;  // uniform: read after the round's last barrier
+    if (__uint_as_float(s_off) < 3e-7f * dmax) break;  // uniform: read after the round's last barrier
     __syncthreads();
   }
   // eigenvalues and their descending order (ties: lower index first)
@@ -408,28 +416,26 @@ cudaError_t launch_build_basis(const Layer &ly, const void *X, int64_t t_rows, c
   k_basis_start<<<dim3((unsigned)((pD + 255) / 256), B), 256, 0, st>>>(Y, pD, 0x5334523472ull);
   ++launch_counter();
   S4R_TRY(cudaGetLastError());
-  auto orthonormalise = [&](float *src, float *dst) -> cudaError_t {  // dst = orth(src); src is overwritten
-    float *in = src, *out = dst;
-    for (int round = 0; round < 2; ++round) {
-      cudaError_t e2 = gemm<double>(in, in, M, p, p, D, D, 1, 1, D, pD, pD, pp, B, st);  // M = in in^T
-      if (e2 != cudaSuccess) return e2;
-      k_chol_inv<<<B, 256, chol_smem, st>>>(M, Linv, p, dev_status);
-      ++launch_counter();
-      if ((e2 = cudaGetLastError()) != cudaSuccess) return e2;
-      e2 = gemm<float>(Linv, in, out, p, D, p, p, 1, D, 1, pp, pD, pD, B, st);  // out = L^-1 in
-      if (e2 != cudaSuccess) return e2;
-      float *tmp = in;
-      in = out;
-      out = tmp;
-    }
-    return cudaSuccess;  // after two rounds the result is back in `src`... see the caller
+  // dst = rows of src made orthonormal by one round of Cholesky QR (M = src src^T in fp64, dst = L^-1 src)
+  auto chol_qr = [&](const float *src, float *dst) -> cudaError_t {
+    cudaError_t e2 = gemm<double>(src, src, M, p, p, D, D, 1, 1, D, pD, pD, pp, B, st);
+    if (e2 != cudaSuccess) return e2;
+    k_chol_inv<<<B, kCholThreads, chol_smem, st>>>(M, Linv, p, dev_status);
+    ++launch_counter();
+    if ((e2 = cudaGetLastError()) != cudaSuccess) return e2;
+    return gemm<float>(Linv, src, dst, p, D, p, p, 1, D, 1, pp, pD, pD, B, st);
   };
-  // two rounds ping-pong src -> dst -> src, so the orthonormal block ends in its first argument
-  S4R_TRY(orthonormalise(Y, Q));
-  float *Qc = Y, *Yc = Q;  // Qc: orthonormal block, Yc: scratch
+  // One round leaves an orthogonality error of about eps32 * cond(src) (the fp32 product L^-1 src), some 1e-4
+  // after a multiplication by G: harmless between iterations, where the next round removes it again, so the
+  // second round is spent only on the start block and before the Rayleigh-Ritz step.
+  float *Qc = Q, *Yc = Y;  // Qc: current block, Yc: scratch
+  S4R_TRY(chol_qr(Y, Q));
   for (int it = 0; it < n_iter; ++it) {
     S4R_TRY(gemm<float>(Qc, G, Yc, p, D, D, D, 1, D, 1, pD, DD, pD, B, st));  // Yc = Qc G
-    S4R_TRY(orthonormalise(Yc, Qc));
+    S4R_TRY(chol_qr(Yc, Qc));
+  }
+  S4R_TRY(chol_qr(Qc, Yc));
+  {
     float *tmp = Qc;
     Qc = Yc;
     Yc = tmp;

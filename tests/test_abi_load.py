@@ -5,6 +5,8 @@ import math
 import os
 import re
 
+import numpy as np
+
 import pytest
 
 import paper_2608_00528_b200 as s4r
@@ -82,3 +84,16 @@ def test_host_helpers_match_closed_forms():
         r8 = s4r.rank_for_ratio(eta, L, s, Dp, G, Wq, 8)
         assert r8 % 8 == 0 and r - 8 < r8 <= r
     assert abs(s4r.rank_for_ratio(0.2, 10 ** 9, 4, 1024, 4, 32, 1) - math.floor(0.2 * 1024)) <= 1   # limit r / D'
+
+
+def test_hybrid_sampling_matches_the_oracle_and_its_definition():
+    """Sec. 3.1.2: evenly spread early positions plus a contiguous block of the most recent ones."""
+    from oracle import s4r_oracle as O
+    for n, m, frac in [(131068, 1024, 0.7), (1000, 64, 0.7), (50, 64, 0.7), (4092, 512, 0.3), (10, 0, 0.7), (300, 100, 1.0),
+                       (300, 100, 0.0)]:
+        got = s4r.hybrid_sample_indices(n, m, frac).numpy().astype(np.int64)
+        want = O.hybrid_sample_indices(n, m, frac)
+        assert np.array_equal(got, want), (n, m, frac)
+        assert np.all(np.diff(got) > 0) and (len(got) == 0 or (got[0] >= 0 and got[-1] < n))
+        n_recent = min(min(m, n), math.ceil(frac * min(m, n)))
+        assert np.array_equal(got[len(got) - n_recent:], np.arange(n - n_recent, n))        # the recent block
