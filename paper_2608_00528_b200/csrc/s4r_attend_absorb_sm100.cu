@@ -497,7 +497,6 @@ __device__ __forceinline__ void cp_async8(void *dst, const void *src) {
 constexpr int kMgTiles = 32;
 
 __global__ void __launch_bounds__(128) k_merge_absorb(const __grid_constant__ MergeAbsorbParams p) {
-  grid_dependency_sync();
   extern __shared__ __align__(16) uint8_t msm[];
   const int h = blockIdx.x, b = blockIdx.y, i = threadIdx.x;
   const int kv = h / p.G, lane = i & 31, warp = i >> 5;
@@ -512,13 +511,8 @@ __global__ void __launch_bounds__(128) k_merge_absorb(const __grid_constant__ Me
   float *red_s = ut_s + p.rv;                                                       // [4][64]
   float *slog_s = red_s + 4 * 64;                                                   // [64]
 
-  int L = p.coef_len[b];
-  L = L < 0 ? 0 : ((int64_t)L > p.max_len ? (int)p.max_len : L);
-  const int count = min(p.sel_count[b], p.sel_stride);
-  const int tiles = (count + kTok - 1) / kTok;
-  const float2 *ms = p.part_ms + ((size_t)b * p.Hq + h) * p.n_tiles;
-  const float *pu = p.part_u + ((size_t)b * p.Hq + h) * p.n_tiles * 2 * p.rv;
-  // ---- one wave of asynchronous copies
+  // ---- one wave of asynchronous copies.  The value basis, the query and the sinks are inputs of the step, so their
+  //      copies go out before the wait for the attend kernel; everything the step produced is read after it.
   {
     const int cpr = p.rv >> 3;
     const __nv_bfloat16 *bvp = p.basis_v + ((size_t)b * p.D + (size_t)kv * kDh) * p.rv;
@@ -534,6 +528,15 @@ __global__ void __launch_bounds__(128) k_merge_absorb(const __grid_constant__ Me
       cp_async16(sk_s + sj * kDh + cc * 8, p.sink_k + off);
       cp_async16(sv_s + sj * kDh + cc * 8, p.sink_v + off);
     }
+  }
+  grid_dependency_sync();
+  int L = p.coef_len[b];
+  L = L < 0 ? 0 : ((int64_t)L > p.max_len ? (int)p.max_len : L);
+  const int count = min(p.sel_count[b], p.sel_stride);
+  const int tiles = (count + kTok - 1) / kTok;
+  const float2 *ms = p.part_ms + ((size_t)b * p.Hq + h) * p.n_tiles;
+  const float *pu = p.part_u + ((size_t)b * p.Hq + h) * p.n_tiles * 2 * p.rv;
+  {
     const int nt0 = min(tiles, kMgTiles);
     if (i < nt0) cp_async8(ms_s + i, ms + i);
     for (int c = i; c < nt0 * (p.rv >> 1); c += 128) cp_async16(pu_s + c * 4, pu + c * 4);

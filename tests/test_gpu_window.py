@@ -188,6 +188,36 @@ def test_window_initialised_from_prompt_queries(n_init):
         assert ok, f"seq {b}: {msg}"
 
 
+@pytest.mark.parametrize("Wq", [4, 32])
+def test_many_windowed_steps_stay_in_step(Wq):
+    """The scoring kernels hand tiles between a producer, two issuing warps and eight epilogue warps through
+    phase-parity barriers; a role that fell out of step would wait out its bound and raise S4R_DEV_TIMEOUT.  With
+    the same query every step the window becomes constant after W_q steps, and so must every result bit."""
+    s4r = _s4r()
+    cfg = W.scaled_config(W.get_config(1), context=20000 + 4, batch=2)
+    p = Problem(cfg, device="cuda").upload()
+    ly = p.layer_desc()
+    B = cfg.batch
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=Wq)
+    win = torch.zeros(B, Wq, cfg.group, cfg.rank_k, dtype=torch.float32, device="cuda")
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(B, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(B, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ref = None
+    for t in range(Wq + 200):
+        s4r.decode_step_windowed(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                 cfg.window, cfg.top_k, win, out, sel, cnt, ws, score_window=Wq,
+                                 rope_theta=cfg.rope_theta, dev_status=status)
+        if t == Wq:
+            ref = (out.clone(), sel.clone(), cnt.clone())
+        elif t > Wq and t % 20 == 0:
+            assert torch.equal(out, ref[0]) and torch.equal(sel, ref[1]) and torch.equal(cnt, ref[2]), f"step {t}"
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert torch.equal(out, ref[0]) and torch.equal(sel, ref[1])
+
+
 def test_windowed_entry_rejects_what_it_cannot_do():
     s4r = _s4r()
     cfg = W.scaled_config(W.get_config(1), context=1000 + 4, batch=1)
