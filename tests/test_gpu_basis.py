@@ -102,6 +102,44 @@ def test_more_iterations_do_not_change_the_converged_part():
     assert np.abs(a[0]["sig"] - b[0]["sig"]).max() <= 1e-4 * a[0]["sv"][0]
 
 
+def test_prefill_chain_with_gpu_built_bases_reconstructs_as_well_as_the_oracles():
+    """Hybrid sampling (host helper) -> s4r_build_basis -> s4r_compress, all through the library, against the oracle's
+    own chain (its sampling, its SVD, its projection) on the same prompt: the low-rank reconstruction error of the
+    cached rows, a quantity that does not depend on which basis of the subspace was found, must agree."""
+    s4r = _s4r()
+    cfg = W.scaled_config(W.get_config(1), context=6000, batch=1)
+    s, r = cfg.sink_count, cfg.rank_k
+    K = W.make_kv(cfg, 0, 0, "k")
+    V = W.make_kv(cfg, 0, 0, "v")
+    T = K.shape[0]
+    ly = s4r.Layer(1, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rank_k, cfg.rank_v, s, s4r.S4R_BF16, T)
+    idx = s4r.hybrid_sample_indices(T - s, cfg.n_sampled)
+    assert np.array_equal(idx.numpy(), O.hybrid_sample_indices(T - s, cfg.n_sampled))
+    d_idx = idx.cuda()[None]
+    d_K, d_V = K.cuda()[None], V.cuda()[None]
+    BK = s4r.build_basis(ly, d_K, d_idx, cfg.rank_k)
+    BV = s4r.build_basis(ly, d_V, d_idx, cfg.rank_v)
+    sink_k = torch.empty(1, s, cfg.d_kv, dtype=torch.bfloat16, device="cuda")
+    sink_v = torch.empty_like(sink_k)
+    CK = torch.zeros(1, T, cfg.rank_k, dtype=torch.bfloat16, device="cuda")
+    CV = torch.zeros(1, T, cfg.rank_v, dtype=torch.bfloat16, device="cuda")
+    ln = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = s4r.alloc_workspace(ly, T, cfg.window, cfg.top_k)
+    s4r.compress(ly, d_K, d_V, BK, BV, sink_k, sink_v, CK, CV, ln, workspace=ws)
+    torch.cuda.synchronize()
+    assert ln.item() == T - s
+    for X, B_gpu, C_gpu, rank in ((K, BK, CK, cfg.rank_k), (V, BV, CV, cfg.rank_v)):
+        Xn = to_np(X)[s:]
+        rec_gpu = to_np(C_gpu[0, :T - s]) @ to_np(B_gpu[0]).T
+        err_gpu = np.linalg.norm(Xn - rec_gpu) / np.linalg.norm(Xn)
+        B_ref, _ = O.build_basis(Xn[O.hybrid_sample_indices(T - s, cfg.n_sampled)], rank)
+        B_ref = O.round_to_storage(B_ref, "bf16")
+        C_ref = O.round_to_storage(Xn @ B_ref, "bf16")
+        err_ref = np.linalg.norm(Xn - C_ref @ B_ref.T) / np.linalg.norm(Xn)
+        print(f"relative reconstruction error: library chain {err_gpu:.5f}, oracle chain {err_ref:.5f}")
+        assert abs(err_gpu - err_ref) <= 2e-3 * err_ref + 1e-5
+
+
 def test_basis_rejects_what_it_cannot_do():
     s4r = _s4r()
     cfg = W.scaled_config(W.get_config(1), context=4096, batch=1)
