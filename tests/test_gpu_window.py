@@ -140,7 +140,7 @@ def test_window_of_one_equals_the_plain_step():
 def test_window_longer_than_the_cache():
     """Window rows whose token index would be negative see nothing and add nothing (Eq. 9's mask)."""
     cfg = W.scaled_config(W.get_config(1), context=2000 + 4, batch=1, top_k=8, window=2)
-    for rows, Wq in ((3, 4), (1, 4), (50, 4), (20, 32), (130, 32)):
+    for rows, Wq in ((0, 4), (3, 4), (1, 4), (50, 4), (20, 32), (130, 32)):
         err = _run_case(cfg, Wq, steps=1, cache_rows=rows)
         print(f"L={rows}, W_q={Wq}: max rel err {err:.3e}")
         assert err <= 1e-4            # every row is selected: what is left is the attention's own rounding
