@@ -6,7 +6,8 @@
 //   2. k_gemm            G = A^T A                                                               [D', D'] fp32
 //   3. iterate on a block of p = r + 32 row vectors Q [p, D'] (deterministic pseudo-random start):
 //        Y = Q G, then Q = orth(Y) by Cholesky QR:  M = Y Y^T accumulated in fp64, M = L L^T and L^-1 in
-//        fp64 by one CTA (k_chol_inv), Q = L^-1 Y; a second round before the Rayleigh-Ritz step.
+//        fp64 by one CTA (k_chol), Q = L^-1 Y by forward substitution (k_trsm); a second round before
+//        the Rayleigh-Ritz step.
 //      One multiplication by G spreads the rows of Y over a condition number of lambda_1 / lambda_p (several
 //      thousand for the spectra of interest), whose square is beyond fp32: hence the fp64 Gram and factor.
 //   4. Rayleigh-Ritz: H = (Q G) Q^T, H = W diag(lambda) W^T by a cyclic Jacobi method in shared memory
@@ -124,16 +125,16 @@ __global__ void __launch_bounds__(256) k_basis_start(float *Q, int64_t n_per_bat
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// M = L L^T (fp64, lower triangle packed in shared memory), then L^-1 in place and out as fp32 [p][p] (zeros
-// above the diagonal).  One CTA per matrix.  A pivot that is not positive raises S4R_DEV_NUMERIC and is replaced.
+// M = L L^T (fp64, lower triangle packed in shared memory); L goes out as fp32 [p][p] (zeros above the diagonal).
+// One CTA per matrix.  A pivot that is not positive raises S4R_DEV_NUMERIC and is replaced.
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }  // i >= j
 
 constexpr int kCholThreads = 1024;
 
-__global__ void __launch_bounds__(kCholThreads) k_chol_inv(double *M, float *Linv, int p, int32_t *dev_status) {
-  extern __shared__ double Ls[];  // packed lower triangle, then one column
+__global__ void __launch_bounds__(kCholThreads) k_chol(const double *M, float *Lout, int p, int32_t *dev_status) {
+  extern __shared__ double Ls[];  // packed lower triangle
   const int tid = threadIdx.x, b = blockIdx.x, lane = tid & 31, warp = tid >> 5;
-  double *Mb = M + (size_t)b * p * p;
+  const double *Mb = M + (size_t)b * p * p;
   for (int e = tid; e < p * p; e += kCholThreads) {
     const int i = e / p, j = e - i * p;
     if (j <= i) Ls[tri(i, j)] = 0.5 * (Mb[(size_t)i * p + j] + Mb[(size_t)j * p + i]);
@@ -159,26 +160,46 @@ __global__ void __launch_bounds__(kCholThreads) k_chol_inv(double *M, float *Lin
     }
     __syncthreads();
   }
-  // X = L^-1 in place, column by column from the right: X[i][j] = -(sum_{k=j+1..i} X[i][k] L[k][j]) / L[j][j];
-  // a warp takes rows, its lanes split the sum
-  double *col = Ls + (size_t)p * (p + 1) / 2;  // copy of column j of L
-  for (int j = p - 1; j >= 0; --j) {
-    for (int k = j + tid; k < p; k += kCholThreads) col[k] = Ls[tri(k, j)];
-    __syncthreads();
-    const double xjj = 1.0 / col[j];
-    if (tid == 0) Ls[tri(j, j)] = xjj;
-    for (int i = j + 1 + warp; i < p; i += kCholThreads / 32) {
-      double sum = 0.0;
-      for (int k = j + 1 + lane; k <= i; k += 32) sum += Ls[tri(i, k)] * col[k];
-      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      if (lane == 0) Ls[tri(i, j)] = -sum * xjj;
-    }
-    __syncthreads();
-  }
-  float *Lo = Linv + (size_t)b * p * p;
+  float *Lo = Lout + (size_t)b * p * p;
   for (int e = tid; e < p * p; e += kCholThreads) {
     const int i = e / p, j = e - i * p;
     Lo[e] = j <= i ? (float)Ls[tri(i, j)] : 0.f;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Q = L^-1 Y by forward substitution: a thread owns one of the D columns, a CTA 128 of them; L (packed) and the
+// CTA's columns of Q sit in shared memory.  grid (D / 128, B).
+constexpr int kTrsmCols = 128;
+
+__global__ void __launch_bounds__(kTrsmCols) k_trsm(const float *L, const float *Y, float *Q, int p, int D) {
+  extern __shared__ float tsm[];
+  float *Lp = tsm;                                  // packed lower triangle
+  float *Qs = tsm + (size_t)p * (p + 1) / 2;        // [p][128]
+  const int tid = threadIdx.x, b = blockIdx.y, c = blockIdx.x * kTrsmCols + tid;
+  const float *Lb = L + (size_t)b * p * p;
+  for (int e = tid; e < p * p; e += kTrsmCols) {
+    const int i = e / p, j = e - i * p;
+    if (j <= i) Lp[tri(i, j)] = Lb[e];
+  }
+  __syncthreads();
+  if (c >= D) return;
+  const float *y = Y + (size_t)b * p * D + c;
+  float *q = Q + (size_t)b * p * D + c;
+  for (int i = 0; i < p; ++i) {
+    const float *li = Lp + tri(i, 0);
+    float a0 = y[(size_t)i * D], a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    int k = 0;
+    for (; k + 4 <= i; k += 4) {
+      a0 = fmaf(-li[k], Qs[k * kTrsmCols + tid], a0);
+      a1 = fmaf(-li[k + 1], Qs[(k + 1) * kTrsmCols + tid], a1);
+      a2 = fmaf(-li[k + 2], Qs[(k + 2) * kTrsmCols + tid], a2);
+      a3 = fmaf(-li[k + 3], Qs[(k + 3) * kTrsmCols + tid], a3);
+    }
+    for (; k < i; ++k) a0 = fmaf(-li[k], Qs[k * kTrsmCols + tid], a0);
+    const float v = ((a0 + a1) + (a2 + a3)) / li[i];
+    Qs[i * kTrsmCols + tid] = v;
+    q[(size_t)i * D] = v;
   }
 }
 
@@ -345,12 +366,13 @@ bool basis_supported(const Layer &ly, int rank, int n_samples) {
   const int p = basis_block(rank);
   if (rank < 1 || rank % 8 || p > ly.D || p > n_samples || (p & 1)) return false;
   const size_t jac = sizeof(float) * (size_t)p * (p + 1) + sizeof(int) * 2 * (size_t)p + 64;
-  const size_t chol = sizeof(double) * ((size_t)p * (p + 1) / 2 + p);
-  return jac <= 226 * 1024 && chol <= 226 * 1024;
+  const size_t chol = sizeof(double) * ((size_t)p * (p + 1) / 2);
+  const size_t trsm = sizeof(float) * ((size_t)p * (p + 1) / 2 + (size_t)p * 128);
+  return jac <= 226 * 1024 && chol <= 226 * 1024 && trsm <= 226 * 1024;
 }
 
 // Workspace layout (bytes, each part 256-byte aligned), in this order:
-//   A [B][n_s][D] f32 | G [B][D][D] f32 | Q, Y [B][p][D] f32 | M [B][p][p] f64 | Linv, H, Wt [B][p][p] f32 |
+//   A [B][n_s][D] f32 | G [B][D][D] f32 | Q, Y [B][p][D] f32 | M [B][p][p] f64 | L, H, Wt [B][p][p] f32 |
 //   lam [B][p] f32 | perm [B][p] i32
 size_t basis_workspace(const Layer &ly, int rank, int n_samples) {
   const size_t p = basis_block(rank), B = ly.B, D = ly.D;
@@ -384,7 +406,7 @@ cudaError_t launch_build_basis(const Layer &ly, const void *X, int64_t t_rows, c
   float *Q = (float *)take(4ull * B * p * D);
   float *Y = (float *)take(4ull * B * p * D);
   double *M = (double *)take(8ull * B * p * p);
-  float *Linv = (float *)take(4ull * B * p * p);
+  float *Lf = (float *)take(4ull * B * p * p);
   float *H = (float *)take(4ull * B * p * p);
   float *Wt = (float *)take(4ull * B * p * p);
   float *lam = (float *)take(4ull * B * p);
@@ -402,11 +424,16 @@ cudaError_t launch_build_basis(const Layer &ly, const void *X, int64_t t_rows, c
   // 2. G = A^T A
   S4R_TRY(gemm<float>(A, A, G, D, D, n_s, 1, D, D, 1, (int64_t)n_s * D, (int64_t)n_s * D, DD, B, st));
   // 3. block iteration
-  static size_t chol_set = 0, jac_set = 0;
-  const size_t chol_smem = sizeof(double) * ((size_t)p * (p + 1) / 2 + p);
+  static size_t chol_set = 0, jac_set = 0, trsm_set = 0;
+  const size_t chol_smem = sizeof(double) * ((size_t)p * (p + 1) / 2);
+  const size_t trsm_smem = sizeof(float) * ((size_t)p * (p + 1) / 2 + (size_t)p * kTrsmCols);
+  if (trsm_smem > trsm_set) {
+    S4R_TRY(cudaFuncSetAttribute(k_trsm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)trsm_smem));
+    trsm_set = trsm_smem;
+  }
   const size_t jac_smem = sizeof(float) * (size_t)p * (p + 1) + sizeof(int) * 2 * (size_t)p + 64;
   if (chol_smem > chol_set) {
-    S4R_TRY(cudaFuncSetAttribute(k_chol_inv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem));
+    S4R_TRY(cudaFuncSetAttribute(k_chol, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem));
     chol_set = chol_smem;
   }
   if (jac_smem > jac_set) {
@@ -416,14 +443,17 @@ cudaError_t launch_build_basis(const Layer &ly, const void *X, int64_t t_rows, c
   k_basis_start<<<dim3((unsigned)((pD + 255) / 256), B), 256, 0, st>>>(Y, pD, 0x5334523472ull);
   ++launch_counter();
   S4R_TRY(cudaGetLastError());
-  // dst = rows of src made orthonormal by one round of Cholesky QR (M = src src^T in fp64, dst = L^-1 src)
+  // dst = rows of src made orthonormal by one round of Cholesky QR (M = src src^T in fp64, dst = L^-1 src;
+  // Lf: the factor rounded to fp32)
   auto chol_qr = [&](const float *src, float *dst) -> cudaError_t {
     cudaError_t e2 = gemm<double>(src, src, M, p, p, D, D, 1, 1, D, pD, pD, pp, B, st);
     if (e2 != cudaSuccess) return e2;
-    k_chol_inv<<<B, kCholThreads, chol_smem, st>>>(M, Linv, p, dev_status);
+    k_chol<<<B, kCholThreads, chol_smem, st>>>(M, Lf, p, dev_status);
     ++launch_counter();
     if ((e2 = cudaGetLastError()) != cudaSuccess) return e2;
-    return gemm<float>(Linv, src, dst, p, D, p, p, 1, D, 1, pp, pD, pD, B, st);
+    k_trsm<<<dim3((D + kTrsmCols - 1) / kTrsmCols, B), kTrsmCols, trsm_smem, st>>>(Lf, src, dst, p, D);
+    ++launch_counter();
+    return cudaGetLastError();
   };
   // One round leaves an orthogonality error of about eps32 * cond(src) (the fp32 product L^-1 src), some 1e-4
   // after a multiplication by G: harmless between iterations, where the next round removes it again, so the
