@@ -125,8 +125,8 @@ __global__ void __launch_bounds__(256) k_basis_start(float *Q, int64_t n_per_bat
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// M = L L^T (fp64, lower triangle packed in shared memory); L goes out as fp32 [p][p] (zeros above the diagonal).
-// One CTA per matrix.  A pivot that is not positive raises S4R_DEV_NUMERIC and is replaced.
+// M = L L^T (fp64, lower triangle packed in shared memory); L goes out as fp32 packed by columns: element (i, k),
+// i >= k, at k (p - 1) - k (k - 1) / 2 + i of the matrix's p (p + 1) / 2 values.  One CTA per matrix.  A pivot that is not positive raises S4R_DEV_NUMERIC and is replaced.
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }  // i >= j
 
 constexpr int kCholThreads = 1024;
@@ -160,46 +160,75 @@ __global__ void __launch_bounds__(kCholThreads) k_chol(const double *M, float *L
     }
     __syncthreads();
   }
-  float *Lo = Lout + (size_t)b * p * p;
+  float *Lo = Lout + (size_t)b * ((size_t)p * (p + 1) / 2);
   for (int e = tid; e < p * p; e += kCholThreads) {
-    const int i = e / p, j = e - i * p;
-    Lo[e] = j <= i ? (float)Ls[tri(i, j)] : 0.f;
+    const int i = e / p, k = e - i * p;
+    if (k <= i) Lo[k * (p - 1) - k * (k - 1) / 2 + i] = (float)Ls[tri(i, k)];
   }
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Q = L^-1 Y by forward substitution: a thread owns one of the D columns, a CTA 128 of them; L (packed) and the
-// CTA's columns of Q sit in shared memory.  grid (D / 128, B).
+// Q = L^-1 Y by forward substitution: a thread owns one of the D columns, a CTA 128 of them; L (packed by columns)
+// and the CTA's columns of Q sit in shared memory.  Rows are solved 32 at a time: first the contributions of all
+// rows solved before are subtracted from the block's 32 right-hand sides (32 independent multiply-adds per solved
+// value), then the 32 x 32 triangle is solved in registers.  grid (D / 128, B).
 constexpr int kTrsmCols = 128;
 
 __global__ void __launch_bounds__(kTrsmCols) k_trsm(const float *L, const float *Y, float *Q, int p, int D) {
   extern __shared__ float tsm[];
-  float *Lp = tsm;                                  // packed lower triangle
+  float *Lc = tsm;                                  // element (i, k), i >= k, at cb(k) + i
   float *Qs = tsm + (size_t)p * (p + 1) / 2;        // [p][128]
   const int tid = threadIdx.x, b = blockIdx.y, c = blockIdx.x * kTrsmCols + tid;
-  const float *Lb = L + (size_t)b * p * p;
-  for (int e = tid; e < p * p; e += kTrsmCols) {
-    const int i = e / p, j = e - i * p;
-    if (j <= i) Lp[tri(i, j)] = Lb[e];
+  {
+    // the factor arrives packed; p (p + 1) / 2 is a multiple of 4, eight 16-byte loads in flight per thread
+    const int n4 = p * (p + 1) / 8;
+    const float4 *src = reinterpret_cast<const float4 *>(L + (size_t)b * ((size_t)p * (p + 1) / 2));
+    float4 *dst = reinterpret_cast<float4 *>(Lc);
+    for (int base = 0; base < n4; base += 8 * kTrsmCols) {
+      float4 t[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + u * kTrsmCols + tid;
+        t[u] = e < n4 ? __ldcg(src + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + u * kTrsmCols + tid;
+        if (e < n4) dst[e] = t[u];
+      }
+    }
   }
   __syncthreads();
   if (c >= D) return;
   const float *y = Y + (size_t)b * p * D + c;
   float *q = Q + (size_t)b * p * D + c;
-  for (int i = 0; i < p; ++i) {
-    const float *li = Lp + tri(i, 0);
-    float a0 = y[(size_t)i * D], a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    int k = 0;
-    for (; k + 4 <= i; k += 4) {
-      a0 = fmaf(-li[k], Qs[k * kTrsmCols + tid], a0);
-      a1 = fmaf(-li[k + 1], Qs[(k + 1) * kTrsmCols + tid], a1);
-      a2 = fmaf(-li[k + 2], Qs[(k + 2) * kTrsmCols + tid], a2);
-      a3 = fmaf(-li[k + 3], Qs[(k + 3) * kTrsmCols + tid], a3);
+  for (int i0 = 0; i0 < p; i0 += 32) {
+    const int nb = min(32, p - i0);
+    float acc[32];
+#pragma unroll
+    for (int r = 0; r < 32; ++r) acc[r] = r < nb ? y[(size_t)(i0 + r) * D] : 0.f;
+    int cb = i0;  // cb(k) + i0 for k = 0
+    for (int k = 0; k < i0; ++k) {
+      const float qk = Qs[k * kTrsmCols + tid];
+      const float *lk = Lc + cb;
+#pragma unroll
+      for (int r = 0; r < 32; ++r)
+        if (r < nb) acc[r] = fmaf(-lk[r], qk, acc[r]);
+      cb += p - 1 - k;  // cb(k + 1) = cb(k) + p - 1 - k
     }
-    for (; k < i; ++k) a0 = fmaf(-li[k], Qs[k * kTrsmCols + tid], a0);
-    const float v = ((a0 + a1) + (a2 + a3)) / li[i];
-    Qs[i * kTrsmCols + tid] = v;
-    q[(size_t)i * D] = v;
+#pragma unroll
+    for (int r = 0; r < 32; ++r) {
+      if (r < nb) {
+        const int k = i0 + r;
+        const float *lk = Lc + (k * (p - 1) - k * (k - 1) / 2) + i0;  // column k of L from row i0 on
+        const float v = acc[r] / lk[r];
+        Qs[k * kTrsmCols + tid] = v;
+        q[(size_t)k * D] = v;
+#pragma unroll
+        for (int r2 = r + 1; r2 < 32; ++r2)
+          if (r2 < nb) acc[r2] = fmaf(-lk[r2], v, acc[r2]);
+      }
+    }
   }
 }
 
