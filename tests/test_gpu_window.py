@@ -98,6 +98,18 @@ def test_window_lengths_that_change_the_kernel_layout(Wq):
     print(f"W_q={Wq}: max rel err {err:.3e}")
 
 
+@pytest.mark.parametrize("over,Wq", [
+    (dict(context=700 + 4, batch=16), 8),                                  # nine scan CTAs per sequence
+    (dict(context=3000 + 4, batch=5, rank_k=64, rank_v=64), 6),            # one 64-column block, general chunk code
+    (dict(context=3000 + 4, batch=2, rank_k=256, rank_v=128), 16),         # four blocks, five ring pieces
+    (dict(context=3000 + 4, batch=2, rank_k=320, rank_v=64), 4),           # the largest supported key rank
+])
+def test_windowed_scoring_other_geometries(over, Wq):
+    cfg = W.scaled_config(W.get_config(1), **over)
+    err = _run_case(cfg, Wq, steps=1)
+    print(f"{over} W_q={Wq}: max rel err {err:.3e}")
+
+
 def test_windowed_scoring_without_rope_and_with_average_pooling():
     cfg = W.scaled_config(W.get_config(1), context=3000 + 4, batch=1, pool_mode="avg", group_mode="max")
     err = _run_case(cfg, 8, steps=1, theta=0.0)
