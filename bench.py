@@ -273,7 +273,7 @@ def run_windowed(args, cfg, s4r, device):
     Wq = args.score_window
     K_steps, Wm = args.steps, max(args.warmup, 3, Wq + 2)
     B = cfg.batch
-    capacity = cfg.cache_len + 8
+    capacity = cfg.cache_len + 2 * (K_steps + Wm) + 40
     c = build_cache(cfg, s4r, device, capacity, list(range(B)))
     ly = c["ly"]
     st = W.storage_dtype(cfg)
@@ -286,14 +286,17 @@ def run_windowed(args, cfg, s4r, device):
     win = torch.zeros(B, Wq, cfg.group, cfg.rank_k, dtype=torch.float32, device=device)
     pool = 4
     qs = torch.stack([c["q"] * (1.0 + 0.01 * i) for i in range(pool)]).to(st)
+    kt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "k", i + 1, device) for b in range(B)]) for i in range(pool)])
+    vt = torch.stack([torch.stack([W.make_token(cfg, 0, b, "v", i + 1, device) for b in range(B)]) for i in range(pool)])
     kw = dict(pool_kernel=cfg.pool_kernel, pool_mode={"max": s4r.POOL_MAX, "avg": s4r.POOL_AVG}[cfg.pool_mode],
               group_mode={"mean": s4r.GROUP_MEAN, "max": s4r.GROUP_MAX}[cfg.group_mode], rope_theta=cfg.rope_theta,
               dev_status=status, score_window=Wq)
     launches = [0]
 
     def step(i):
-        s4r.decode_step_windowed(ly, qs[i % pool], c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"], c["BK"], c["BV"],
-                                 capacity, cfg.window, cfg.top_k, win, out, sel, cnt, ws, **kw)
+        j = i % pool
+        s4r.append_decode_step_windowed(ly, kt[j], vt[j], qs[j], c["sink_k"], c["sink_v"], c["CK"], c["CV"], c["len"],
+                                        c["BK"], c["BV"], capacity, cfg.window, cfg.top_k, win, out, sel, cnt, ws, **kw)
         launches[0] += s4r.last_launch_count()
 
     for i in range(Wm):
@@ -314,6 +317,7 @@ def run_windowed(args, cfg, s4r, device):
     s4r.stage_timing(True)
     stage_sum = {}
     for i in range(20):
+        c["len"].fill_(cfg.cache_len + Wm + K_steps)      # keep the cache length of the timed region
         step(i)
         for k_, v_ in s4r.stage_times().items():
             stage_sum[k_] = stage_sum.get(k_, 0.0) + v_ / 20
@@ -330,7 +334,7 @@ def run_windowed(args, cfg, s4r, device):
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": f"{cfg.name}_wq{Wq}", "batch": B, "context": cfg.context, "rank": cfg.rank_k,
                    "window": cfg.window, "top_k": cfg.top_k, "score_window": Wq, "scored_rows": rows,
-                   "step": "s4r_decode_step_windowed (no cache update)",
+                   "step": "s4r_append_decode_step_windowed (cache update + windowed decode step)",
                    "l2": "inputs larger than L2 (key coefficients %.0f MB per pass)" % (scan_bytes / 1e6)},
         "roofline": {"bound": "hbm", "kernel": "windowed latent scoring (all passes over C^K)",
                      "achieved": scan_bytes / (scan_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",

@@ -222,6 +222,17 @@ int s4r_decode_step_windowed(const s4r_layer_t *layer, const void *q, const void
                              int32_t out_dtype, int32_t *sel_idx, int32_t *sel_count, void *workspace,
                              size_t workspace_bytes, int32_t *dev_status, void *stream);
 
+/* s4r_append followed by s4r_decode_step_windowed as one call: the projection kernel that produces c^Q also projects
+ * and appends the new token's rows (Eq. 5-6) and bumps coef_len, then the windowed step runs on the grown cache.
+ * k_t, v_t [B, D'] pre-RoPE; coef_k, coef_v, coef_len are updated; max_len must bound coef_len[b] + 1. */
+int s4r_append_decode_step_windowed(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,
+                                    const void *sink_k, const void *sink_v, void *coef_k, void *coef_v,
+                                    int32_t *coef_len, const void *key_basis, const void *value_basis, int64_t max_len,
+                                    int32_t window, int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope,
+                                    float *query_window, void *out, int32_t out_dtype, int32_t *sel_idx,
+                                    int32_t *sel_count, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                    void *stream);
+
 /* Initial query-coefficient window (Eq. 4: C^Q = Q~ B^K for the last prompt queries).
  * queries       [B, n_queries, H_q, d_h] (device, layer dtype), oldest first, pre-RoPE; 0 <= n_queries <= W_q
  * query_window  [B, W_q, G, rank_k] fp32 (device): rows W_q - n_queries .. W_q - 1 receive the coefficients of the

@@ -21,7 +21,7 @@ VALUE_AUTO, VALUE_RECONSTRUCT = 0, 1
 DEV_TIMEOUT, DEV_BOUNDS = 1, 2
 
 EXPORTS = ("s4r_workspace_bytes", "s4r_workspace_bytes_windowed", "s4r_compress", "s4r_append", "s4r_decode_step",
-           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed", "s4r_window_init", "s4r_host_step_layout", "s4r_append_decode_step_host", "s4r_basis_workspace_bytes", "s4r_build_basis",
+           "s4r_decode_step_host", "s4r_decode_step_static", "s4r_append_decode_step", "s4r_decode_step_windowed", "s4r_append_decode_step_windowed", "s4r_window_init", "s4r_host_step_layout", "s4r_append_decode_step_host", "s4r_basis_workspace_bytes", "s4r_build_basis",
            "s4r_hybrid_sample_indices",
            "s4r_top_k_from_ratio", "s4r_rank_for_ratio", "s4r_last_launch_count", "s4r_stage_timing",
            "s4r_stage_times", "s4r_strerror", "s4r_last_cuda_error", "s4r_version")
@@ -81,6 +81,9 @@ def load(build_if_missing: bool = True):
     lib.s4r_workspace_bytes.argtypes = [lp, i64, i32, i32]
     lib.s4r_workspace_bytes_windowed.restype = sz
     lib.s4r_workspace_bytes_windowed.argtypes = [lp, i64, i32, i32, i32]
+    lib.s4r_append_decode_step_windowed.restype = ctypes.c_int
+    lib.s4r_append_decode_step_windowed.argtypes = [lp] + [vp] * 10 + [i64, i32, i32, ctypes.POINTER(_Score),
+                                                    ctypes.POINTER(_Rope), vp, vp, i32, vp, vp, vp, sz, vp, vp]
     lib.s4r_window_init.restype = ctypes.c_int
     lib.s4r_window_init.argtypes = [lp, vp, i32, vp, vp, i32, vp]
     lib.s4r_decode_step_windowed.restype = ctypes.c_int
@@ -288,6 +291,28 @@ def decode_step_windowed(layer: Layer, q, sink_k, sink_v, coef_k, coef_v, coef_l
                                          _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream))
     if rc != 0:
         raise S4RError(rc, "s4r_decode_step_windowed")
+
+
+def append_decode_step_windowed(layer: Layer, k_t, v_t, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis,
+                                value_basis, max_len: int, window: int, top_k: int, query_window, out, sel_idx,
+                                sel_count, workspace, *, score_window: int, pool_kernel: int = 7,
+                                pool_mode: int = POOL_MAX, group_mode: int = GROUP_MEAN, rope_theta: float = 0.0,
+                                value_path: int = VALUE_AUTO, dev_status=None, stream=None):
+    """s4r_append_decode_step_windowed: the cache update and the windowed decode step as one call."""
+    _need_cuda(k_t, v_t, q, coef_k, coef_v, coef_len, key_basis, value_basis, query_window, out, sel_idx, sel_count,
+               workspace)
+    if query_window.dtype != torch.float32 or tuple(query_window.shape) != (
+            layer.batch, score_window, layer.n_q_heads // layer.n_kv_heads, layer.rank_k) or not query_window.is_contiguous():
+        raise ValueError("query_window must be a contiguous fp32 tensor [B, W_q, G, rank_k]")
+    sc, rp = _score_rope(pool_kernel, pool_mode, group_mode, score_window, rope_theta, value_path)
+    out_dtype = S4R_BF16 if out.dtype == torch.bfloat16 else S4R_F32
+    rc = load().s4r_append_decode_step_windowed(
+        ctypes.byref(layer.c()), _ptr(k_t), _ptr(v_t), _ptr(q), _ptr(sink_k), _ptr(sink_v), _ptr(coef_k), _ptr(coef_v),
+        _ptr(coef_len), _ptr(key_basis), _ptr(value_basis), int(max_len), int(window), int(top_k), ctypes.byref(sc),
+        ctypes.byref(rp), _ptr(query_window), _ptr(out), out_dtype, _ptr(sel_idx), _ptr(sel_count), _ptr(workspace),
+        workspace.numel(), _ptr(dev_status), _stream(stream))
+    if rc != 0:
+        raise S4RError(rc, "s4r_append_decode_step_windowed")
 
 
 def window_init(layer: Layer, queries, key_basis, query_window, *, score_window: int, stream=None):

@@ -265,7 +265,7 @@ static int decode_impl(const s4r_layer_t *layer, const void *k_t, const void *v_
   if (!plan_decode(ly, max_len, window, top_k, &a.plan)) return S4R_ERR_INVALID_ARG;
   WindowPlan wp = {};
   if (query_window) {
-    if (k_t || !wscan_supported(ly, sc.score_window)) return S4R_ERR_UNSUPPORTED;  // bf16 caches, rank % 64 == 0, W_q <= 128
+    if (!wscan_supported(ly, sc.score_window)) return S4R_ERR_UNSUPPORTED;  // bf16 caches, rank % 64 == 0, W_q <= 128
     if (!plan_window(ly, a.plan, sc.score_window, &wp)) return S4R_ERR_INVALID_ARG;
   }
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
@@ -372,6 +372,19 @@ int s4r_decode_step_windowed(const s4r_layer_t *layer, const void *q, const void
   return decode_impl(layer, nullptr, nullptr, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis,
                      max_len, window, top_k, score, rope, out, out_dtype, sel_idx, sel_count, workspace,
                      workspace_bytes, dev_status, stream, query_window);
+}
+
+int s4r_append_decode_step_windowed(const s4r_layer_t *layer, const void *k_t, const void *v_t, const void *q,
+                                    const void *sink_k, const void *sink_v, void *coef_k, void *coef_v,
+                                    int32_t *coef_len, const void *key_basis, const void *value_basis, int64_t max_len,
+                                    int32_t window, int32_t top_k, const s4r_score_t *score, const s4r_rope_t *rope,
+                                    float *query_window, void *out, int32_t out_dtype, int32_t *sel_idx,
+                                    int32_t *sel_count, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                    void *stream) {
+  if (!k_t || !v_t || !query_window || !score) return S4R_ERR_INVALID_ARG;
+  return decode_impl(layer, k_t, v_t, q, sink_k, sink_v, coef_k, coef_v, coef_len, key_basis, value_basis, max_len,
+                     window, top_k, score, rope, out, out_dtype, sel_idx, sel_count, workspace, workspace_bytes,
+                     dev_status, stream, query_window);
 }
 
 int s4r_window_init(const s4r_layer_t *layer, const void *queries, int32_t n_queries, const void *key_basis,

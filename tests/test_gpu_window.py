@@ -230,6 +230,44 @@ def test_many_windowed_steps_stay_in_step(Wq):
     assert torch.equal(out, ref[0]) and torch.equal(sel, ref[1])
 
 
+def test_fused_append_and_windowed_step_agrees_with_separate_calls():
+    s4r = _s4r()
+    Wq = 8
+    cfg = W.scaled_config(W.get_config(1), context=4000 + 3, batch=2)
+    res = []
+    for fused in (False, True):
+        p = Problem(cfg, device="cuda", capacity=cfg.cache_len + 4).upload()
+        ly = p.layer_desc()
+        ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=Wq)
+        win = torch.zeros(cfg.batch, Wq, cfg.group, cfg.rank_k, dtype=torch.float32, device="cuda")
+        out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, device="cuda")
+        sel = torch.empty(cfg.batch, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+        cnt = torch.empty(cfg.batch, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for step in (1, 2, 3):
+            kt = torch.stack([W.make_token(cfg, 0, b, "k", step, "cuda") for b in range(cfg.batch)])
+            vt = torch.stack([W.make_token(cfg, 0, b, "v", step, "cuda") for b in range(cfg.batch)])
+            kw = dict(score_window=Wq, rope_theta=cfg.rope_theta, dev_status=status)
+            if fused:
+                s4r.append_decode_step_windowed(ly, kt, vt, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK,
+                                                p.d_BV, p.cap, cfg.window, cfg.top_k, win, out, sel, cnt, ws, **kw)
+            else:
+                s4r.append(ly, kt, vt, p.d_BK, p.d_BV, p.d_CK, p.d_CV, p.d_len)
+                s4r.decode_step_windowed(ly, p.d_q, p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                         cfg.window, cfg.top_k, win, out, sel, cnt, ws, **kw)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        res.append((out.clone(), sel.clone(), cnt.clone(), p.d_CK.clone(), p.d_len.clone(), win.clone()))
+    (out_a, sel_a, cnt_a, ck_a, len_a, win_a), (out_b, sel_b, cnt_b, ck_b, len_b, win_b) = res
+    assert len_a.tolist() == len_b.tolist() == [cfg.cache_len + 3] * cfg.batch
+    assert torch.equal(cnt_a, cnt_b) and torch.equal(win_a, win_b)
+    xf, yf = ck_a.float(), ck_b.float()
+    assert torch.all((xf - yf).abs() <= 2.0 ** -7 * torch.maximum(xf.abs(), yf.abs()) + 1e-30)
+    same = sum(len(set(sel_a[b].tolist()) & set(sel_b[b].tolist())) for b in range(cfg.batch))
+    assert same >= cfg.batch * (cfg.window + cfg.top_k) - 2 * cfg.batch
+    assert ((out_a - out_b).abs().amax() / out_a.abs().amax()).item() <= 1e-3
+
+
 def test_windowed_entry_rejects_what_it_cannot_do():
     s4r = _s4r()
     cfg = W.scaled_config(W.get_config(1), context=1000 + 4, batch=1)
