@@ -1,12 +1,14 @@
 // Prefill projection (Eq. 3) for bf16 on sm_100a: C[T - s, r] = S[s:T, D'] B[D', r] per sequence, as a
 // persistent tcgen05 GEMM.
 //
-// A work item is 256 consecutive token rows of one sequence.  For each 64-wide block of D' a pipeline stage
-// holds two [128 x 64] row blocks of S and one [r x 64] block of B^T (all TMA, 128-byte swizzle); one thread
-// issues 2 x 4 tcgen05.mma (M = 128, N = r, K = 16) per stage into two fp32 accumulators in tensor memory, so
-// every block of B^T that crosses L2 -> SM is used for 256 rows.  Four epilogue warps read the accumulators
-// back, round once to bf16 and store whole 16-byte pieces of the coefficient rows.  B^T ([r, D'], K-major for
-// the tensor core) is produced once per call by a small transpose kernel into the workspace.
+// A work item is 128 consecutive token rows of one sequence.  For each 64-wide block of D' a pipeline stage
+// holds one [128 x 64] row block of S and one [r x 64] block of B^T (all TMA, 128-byte swizzle); one thread
+// issues 4 tcgen05.mma (M = 128, N = r, K = 16) per stage into one of TWO fp32 accumulators in tensor memory,
+// which alternate between items: while eight epilogue warps read item n back, round once to bf16 and store whole
+// 16-byte pieces of the coefficient rows, the products of item n + 1 already run.  (Items of 256 rows with both
+// accumulators in use at once halve the basis traffic from L2, but then every item ends with the tensor cores
+// and the loads waiting for the read-back: measured 8 % slower.)  B^T ([r, D'], K-major for the tensor core) is
+// needed only when r is not a multiple of 64 and is then produced once per call by a small transpose kernel.
 // Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-5 = epilogue.  grid = number of SMs.
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
@@ -17,8 +19,8 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kMTile = 256;
-constexpr int kStages = 3;
+constexpr int kMTile = 128;
+constexpr int kStages = 5;
 constexpr int kCmpEpiWarps = 8;  // two warps per tensor-memory lane quadrant: even / odd chunks of 32 columns
 constexpr int kCmpThreads = 64 + 32 * kCmpEpiWarps;
 
@@ -53,10 +55,10 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.r * 128;
-  const uint32_t stage_bytes = 2 * a_bytes + ((b_bytes + 1023u) & ~1023u);
+  const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kStages * stage_bytes);
-  uint64_t *full = bars, *empty = bars + kStages, *acc_full = bars + 2 * kStages, *acc_empty = acc_full + 1;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 1);
+  uint64_t *full = bars, *empty = bars + kStages, *acc_full = bars + 2 * kStages, *acc_empty = acc_full + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -69,8 +71,10 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], 1);
     }
-    mbar_init(acc_full, 1);
-    mbar_init(acc_empty, kCmpEpiWarps);  // one arrival per epilogue warp
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&acc_full[i], 1);
+      mbar_init(&acc_empty[i], kCmpEpiWarps);  // one arrival per epilogue warp
+    }
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tmap_x);
@@ -94,14 +98,13 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
           const int s = it % kStages;
           if (!mbar_wait(&empty[s], ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t *st = smem + (size_t)s * stage_bytes;
-          mbar_expect_tx(&full[s], 2 * a_bytes + b_bytes);
+          mbar_expect_tx(&full[s], a_bytes + b_bytes);
           tma_load_2d_hint(st, &tmap_x, kb * 64, y0, &full[s], pol);
-          tma_load_2d_hint(st + a_bytes, &tmap_x, kb * 64, y0 + 128, &full[s], pol);
           if (p.mn_major) {
             for (int g = 0; g < (p.r >> 6); ++g)  // [64 rows of D' x 64 columns] boxes, one per 64 columns of r
-              tma_load_2d(st + 2 * a_bytes + g * 8192, &tmap_bt, g * 64, b * p.D + kb * 64, &full[s]);
+              tma_load_2d(st + a_bytes + g * 8192, &tmap_bt, g * 64, b * p.D + kb * 64, &full[s]);
           } else {
-            tma_load_2d(st + 2 * a_bytes, &tmap_bt, kb * 64, b * p.r, &full[s]);
+            tma_load_2d(st + a_bytes, &tmap_bt, kb * 64, b * p.r, &full[s]);
           }
           issued = it + 1;
         }
@@ -121,51 +124,49 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
       int it = 0, n_done = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
-        if (!mbar_wait(acc_empty, ((uint32_t)n_done & 1u) ^ 1u, abort_flag)) break;
+        const int acc = n_done & 1;
+        if (!mbar_wait(&acc_empty[acc], (((uint32_t)n_done >> 1) & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * 256u;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % kStages;
           if (!mbar_wait(&full[s], (uint32_t)(it / kStages) & 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
-          const uint64_t a0 = umma_desc_sw128(st), a1 = umma_desc_sw128(st + a_bytes);
-          const uint64_t bd = p.mn_major ? umma_desc_mn_sw128(st + 2 * a_bytes, 8192) : umma_desc_sw128(st + 2 * a_bytes);
+          const uint64_t a0 = umma_desc_sw128(st);
+          const uint64_t bd = p.mn_major ? umma_desc_mn_sw128(st + a_bytes, 8192) : umma_desc_sw128(st + a_bytes);
 #pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4) {
-            umma_bf16(tmem_base, a0 + (uint64_t)(k4 * 2), bd + b_kstep * k4, idesc, (kb | k4) != 0);
-            umma_bf16(tmem_base + 256u, a1 + (uint64_t)(k4 * 2), bd + b_kstep * k4, idesc, (kb | k4) != 0);
-          }
+          for (int k4 = 0; k4 < 4; ++k4) umma_bf16(d_tmem, a0 + (uint64_t)(k4 * 2), bd + b_kstep * k4, idesc, (kb | k4) != 0);
           umma_commit(&empty[s]);
         }
-        if (ok) umma_commit(acc_full);
+        if (ok) umma_commit(&acc_full[acc]);
       }
     }
   } else {
-    // The accumulators are single-buffered (two of 192 columns fill tensor memory), so the next item's products
-    // wait for this read-back: it is spread over eight warps and hands the accumulators back as soon as the last
-    // values are in registers.
+    // Two warps per lane quadrant split the 32-column chunks by parity and hand the accumulator back as soon as
+    // their last values are in registers.
     const int quad = warp & 3, chunk_par = (warp - 2) >> 2;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     int n_done = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n_done) {
       const int b = item / p.n_mtiles, mt = item - b * p.n_mtiles;
-      if (ok) ok = mbar_wait(acc_full, (uint32_t)n_done & 1u, abort_flag);
+      const int acc = n_done & 1;
+      if (ok) ok = mbar_wait(&acc_full[acc], ((uint32_t)n_done >> 1) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
-        const int64_t row = (int64_t)mt * kMTile + half * 128 + quad * 32 + lane;
+      {
+        const int64_t row = (int64_t)mt * kMTile + quad * 32 + lane;
         __nv_bfloat16 *dst = p.coef + ((size_t)b * p.cap + (size_t)row) * p.r;
         for (int c0 = chunk_par * 32; c0 < p.r; c0 += 64) {
           uint32_t v[32];
-          tmem_ld32(tmem_base + (uint32_t)half * 256u + lane_addr + (uint32_t)c0, v);
+          tmem_ld32(tmem_base + (uint32_t)acc * 256u + lane_addr + (uint32_t)c0, v);
           tmem_ld_wait();
-          if (half == 1 && c0 + 64 >= p.r) {  // last read of this warp for the item
+          if (c0 + 64 >= p.r) {  // last read of this warp for the item
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty);
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);
           }
           if (row < n_rows) {
 #pragma unroll
@@ -189,7 +190,7 @@ __global__ void __launch_bounds__(kCmpThreads, 1) k_compress_sm100(const __grid_
       if (chunk_par * 32 >= p.r) {  // a warp without columns (r <= 32) still owes its arrival
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty);
+        if (lane == 0) mbar_arrive(&acc_empty[acc]);
       }
     }
   }
@@ -241,7 +242,7 @@ cudaError_t launch_compress_sm100(const Layer &ly, const void *X, const void *ba
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return cudaErrorInvalidValue;
   }
-  const uint32_t stage_bytes = 2 * 128 * 128 + (((uint32_t)r * 128 + 1023u) & ~1023u);
+  const uint32_t stage_bytes = 128 * 128 + (((uint32_t)r * 128 + 1023u) & ~1023u);
   const size_t smem = 1024 + (size_t)kStages * stage_bytes + 256;
   static size_t smem_set = 0;
   if (smem > smem_set) {
