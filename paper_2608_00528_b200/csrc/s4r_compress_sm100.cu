@@ -9,7 +9,7 @@
 // accumulators in use at once halve the basis traffic from L2, but then every item ends with the tensor cores
 // and the loads waiting for the read-back: measured 8 % slower.)  B^T ([r, D'], K-major for the tensor core) is
 // needed only when r is not a multiple of 64 and is then produced once per call by a small transpose kernel.
-// Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-5 = epilogue.  grid = number of SMs.
+// Warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-9 = epilogue.  grid = number of SMs.
 #include "s4r_internal.h"
 #include "s4r_sm100.cuh"
 
