@@ -323,7 +323,10 @@ __global__ void __launch_bounds__(kJacThreads) k_jacobi_eig(const float *H, floa
     if (__uint_as_float(s_off) < 3e-7f * dmax) break;  // uniform: read after the round's last barrier
     __syncthreads();
   }
-  // eigenvalues and their descending order (ties: lower index first)
+  // eigenvalues and their descending order (ties: lower index first).  The order starts as the identity so that
+  // every entry is a valid index even if a degenerate input left NaNs behind, whose ranks collide.
+  for (int i = tid; i < p; i += kJacThreads) perm[(size_t)b * p + i] = i;
+  __syncthreads();
   for (int i = tid; i < p; i += kJacThreads) {
     const float li = Hs[i * ld + i];
     int rank = 0;
@@ -343,7 +346,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) k_basis_finish(const float *Rt, const float *lam, const int32_t *perm, T *basis,
                                                       float *sigma, int p, int D, int r) {
   const int c = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-  const int src = perm[(size_t)b * p + c];
+  const int src = min(max(perm[(size_t)b * p + c], 0), p - 1);
   const float *v = Rt + ((size_t)b * p + src) * D;
   __shared__ float s_val[256];
   __shared__ int s_idx[256];
@@ -370,7 +373,7 @@ __global__ void __launch_bounds__(256) k_basis_finish(const float *Rt, const flo
     }
     __syncthreads();
   }
-  const float sign = v[s_idx[0]] < 0.f ? -1.f : 1.f;
+  const float sign = v[min(max(s_idx[0], 0), D - 1)] < 0.f ? -1.f : 1.f;  // (all-NaN vectors leave the start index)
   T *out = basis + (size_t)b * D * r + c;
   for (int d = tid; d < D; d += 256) Store<T>::st(out + (size_t)d * r, sign * v[d]);
   if (sigma && tid == 0) sigma[(size_t)b * r + c] = sqrtf(fmaxf(lam[(size_t)b * p + src], 0.f));

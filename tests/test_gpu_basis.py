@@ -140,6 +140,24 @@ def test_prefill_chain_with_gpu_built_bases_reconstructs_as_well_as_the_oracles(
         assert abs(err_gpu - err_ref) <= 2e-3 * err_ref + 1e-5
 
 
+def test_rank_deficient_sample_is_reported_not_fatal():
+    """All sampled rows equal: the Gram matrix has rank one, the Cholesky factorisation meets pivots that are not
+    positive.  The call must come back with S4R_DEV_NUMERIC in the status word (and a valid context)."""
+    s4r = _s4r()
+    cfg = W.scaled_config(W.get_config(0), context=1024, batch=1)
+    ly = s4r.Layer(1, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rank_k, cfg.rank_v, cfg.sink_count,
+                   s4r.S4R_F32, 1024)
+    X = torch.ones(1, 1024, cfg.d_kv, dtype=torch.float32, device="cuda")
+    idx = torch.arange(512, dtype=torch.int32, device="cuda")[None]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    basis = s4r.build_basis(ly, X, idx, cfg.rank_k, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() & 4
+    assert tuple(basis.shape) == (1, cfg.d_kv, cfg.rank_k)
+    # the device is still usable
+    assert float(torch.ones(4, device="cuda").sum()) == 4.0
+
+
 def test_basis_rejects_what_it_cannot_do():
     s4r = _s4r()
     cfg = W.scaled_config(W.get_config(1), context=4096, batch=1)
