@@ -203,3 +203,68 @@ def test_config4_layers_and_decode_steps_at_full_shape():
               f"max rel output error {worst:.3e}")
         del p, ws
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("Wq", [32])
+def test_full_size_windowed_scoring_and_basis(Wq):
+    """The windowed estimator (Eq. 7, 9, 10) on config 2 at full size: W_q successive queries go through
+    s4r_decode_step_windowed, which fills the FIFO itself; the last step is compared with the oracle's step on the
+    window it builds from its own projections of the same queries."""
+    import paper_2608_00528_b200 as s4r
+    cfg = W.get_config(2)
+    checked = (5,)
+    p = FullSizeProblem(cfg, checked)
+    p.check_compress_and_adopt_oracle_coefficients()
+    B, s = cfg.batch, cfg.sink_count
+    queries = [torch.stack([W.make_query(cfg, p.d_K[b], 0, b, step=i) for b in range(B)]) for i in range(Wq)]
+    # while the prompt is still on the device: the subspace construction at the full batch and prompt length (it reads
+    # only the sampled rows), singular values and captured energy against the oracle's SVD for the checked sequence
+    idx = torch.stack([(W.sample_rows(cfg, 0, b, "k") - s).to(torch.int32) for b in range(B)]).cuda()
+    sigma = torch.zeros(B, cfg.rank_k, dtype=torch.float32, device="cuda")
+    bstatus = torch.zeros(1, dtype=torch.int32, device="cuda")
+    basis = s4r.build_basis(p.layer_desc(), p.d_K, idx, cfg.rank_k, sigma=sigma, dev_status=bstatus)
+    torch.cuda.synchronize()
+    assert bstatus.item() == 0
+    for b in checked:
+        rows = to_np(p.d_K[b][W.sample_rows(cfg, 0, b, "k").cuda()])
+        B_ref, sv = O.build_basis(rows, cfg.rank_k)
+        assert np.abs(sigma[b].double().cpu().numpy() - sv[:cfg.rank_k]).max() <= 2e-4 * sv[0]
+        Sn = O.normalize_rows(rows)
+        e_ref = np.linalg.norm(Sn @ O.round_to_storage(B_ref, "bf16")) ** 2
+        assert np.linalg.norm(Sn @ to_np(basis[b])) ** 2 >= (1.0 - 2e-4) * e_ref
+    del p.d_K, p.d_V, basis
+    torch.cuda.empty_cache()
+    ly = p.layer_desc()
+    ws = s4r.alloc_workspace(ly, p.cap, cfg.window, cfg.top_k, score_window=Wq)
+    win = torch.zeros(B, Wq, cfg.group, cfg.rank_k, dtype=torch.float32, device="cuda")
+    out = torch.empty(B, cfg.n_q_heads, cfg.head_dim, device="cuda")
+    sel = torch.empty(B, cfg.window + cfg.top_k, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(B, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for i in range(Wq):
+        s4r.decode_step_windowed(ly, queries[i], p.d_sink_k, p.d_sink_v, p.d_CK, p.d_CV, p.d_len, p.d_BK, p.d_BV, p.cap,
+                                 cfg.window, cfg.top_k, win, out, sel, cnt, ws, score_window=Wq,
+                                 rope_theta=cfg.rope_theta, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for b in checked:
+        qs = [to_np(queries[i][b]) for i in range(Wq)]
+        window_rows = np.stack([O.project_query(q, p.BK[b], cfg.n_kv_heads) for q in qs], axis=1)     # [G, W_q, r]
+        res = O.decode_step(qs[-1], to_np(p.K[b][:s]), to_np(p.V[b][:s]), p.CK[b][:p.L], p.CV[b][:p.L], p.BK[b], p.BV[b],
+                            cfg.window, cfg.top_k, kappa=cfg.pool_kernel, pool_mode=cfg.pool_mode,
+                            group_mode=cfg.group_mode, theta=cfg.rope_theta, CQ_window=window_rows)
+        n = int(cnt[b].item())
+        got = sel[b, :n].cpu().numpy().astype(np.int64)
+        assert n == res["W_eff"] + res["k_eff"]
+        ok, msg = O.selection_agrees(res["score"], res["idx"], got, res["W_eff"], res["k_eff"], 1e-3)
+        assert ok, f"seq {b}: {msg}"
+        if np.array_equal(np.sort(got), np.sort(np.asarray(res["idx"], dtype=np.int64))):
+            ref = res["out"]
+        else:
+            ref = O.sparse_attention(qs[-1], to_np(p.K[b][:s]), to_np(p.V[b][:s]), p.CK[b][:p.L], p.CV[b][:p.L], p.BK[b],
+                                     p.BV[b], np.sort(got), cfg.rope_theta)
+        err = O.output_error(to_np(out[b]), ref)
+        assert err <= 1e-2, f"seq {b}: output error {err:.3e}"
+        print(f"{cfg.name} W_q={Wq}: sequence {b} selection ok, max rel output error {err:.3e}")
+    for b in range(B):
+        _properties(p, out, sel, cnt, b, cfg.window, cfg.top_k)
