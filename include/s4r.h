@@ -132,7 +132,8 @@ size_t s4r_workspace_bytes_windowed(const s4r_layer_t *layer, int64_t max_len, i
  * X          [B, T, D'] pre-RoPE rows INCLUDING the s sink rows (device, layer dtype)
  * sample_idx [B, n_samples] int32 NON-SINK indices in [0, T - s) (device); out-of-range entries set
  *            S4R_DEV_BOUNDS and are clamped.  s4r_hybrid_sample_indices writes the paper's sampling pattern.
- * Method: block power iteration with r + 32 vectors on the Gram matrix S_n^T S_n, n_iter iterations (<= 0: 24),
+ * Method: block power iteration with r + 32 vectors on the Gram matrix S_n^T S_n, n_iter iterations (<= 0: 24; more
+ * than 4096: S4R_ERR_INVALID_ARG),
  * Rayleigh-Ritz at the end; vector i converges like (sigma_{r+33} / sigma_i)^(2 n_iter), so the result is the
  * SVD's up to that error and fp32 rounding.  Singular vectors whose singular values are closer than that are
  * determined only as a subspace (by this routine as by any SVD in finite precision).

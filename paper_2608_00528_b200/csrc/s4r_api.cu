@@ -154,7 +154,7 @@ int s4r_build_basis(const s4r_layer_t *layer, const void *X, int64_t T, const in
   launch_counter() = 0;
   Layer ly;
   if (!layer_ok(layer, &ly)) return S4R_ERR_INVALID_ARG;
-  if (!X || !sample_idx || !basis || n_samples < 1 || rank < 1 || T <= ly.s) return S4R_ERR_INVALID_ARG;
+  if (!X || !sample_idx || !basis || n_samples < 1 || rank < 1 || T <= ly.s || n_iter > 4096) return S4R_ERR_INVALID_ARG;
   if (n_samples > 65535 || ly.B > 65535) return S4R_ERR_UNSUPPORTED;
   if (!basis_supported(ly, rank, n_samples)) return S4R_ERR_UNSUPPORTED;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < basis_workspace(ly, rank, n_samples))
