@@ -29,10 +29,10 @@ import torch  # noqa: E402
 import workloads as W  # noqa: E402
 
 # DRAM bytes (read + write) of one latent-scoring launch per algorithmic byte, from an `ncu --set full` capture of
-# the same launch configuration at 64K context (207.84 MB read + 4.33 MB written for 201.33 MB of key
+# the same launch configuration at 64K context (207.85 MB read + 3.81 MB written for 201.33 MB of key
 # coefficients; the rest is the bases of the fused projections and the part of the logits that left L2).  The
 # traffic grows in proportion to the rows scanned, so the ratio carries to the 128K launch.
-SCAN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = (207.84 + 4.33) / 201.33
+SCAN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = (207.85 + 3.81) / 201.33
 
 METRIC = "decode steps/sec at 128K context (one layer, whole batch)"
 UNIT = "steps/s"
